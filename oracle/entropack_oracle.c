@@ -1,0 +1,872 @@
+/*
+ * EntroPack reference oracle  --  TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, scalar CPU restatement of the EntroPack weight codec, written
+ * from the paper's method section step by step so that it can be checked
+ * against the paper by eye.  It shares no code with the CUDA library; only the
+ * tests, the smoke check and the bench's cpu_baseline / reference arm call it.
+ *
+ * What it computes (paper passage beside each function):
+ *   row RMS normalisation            Sec. 3.2 "Normalization and nearest points"
+ *   E8 nearest point                 Eq. 2, Eq. 3 and the tie conventions below them
+ *   field representation + inverse   Eq. 4, Eq. 5
+ *   17 coset-conditioned tables      Eq. 6, b-bit frequencies, C_CE of Eq. 8
+ *   stored-size estimate             Eq. 10, Eq. 11
+ *   sampled geometric scale search   Eq. 12, Algorithm 1, App. "Scale-search settings"
+ *   row-scale refit                  Eq. 13
+ *   tiled 32-state rANS encode       Eq. 17, App. "Tiled rANS implementation"
+ *   rANS decode + reconstruction     Eq. 18, Eq. 5, Eq. 19
+ *   relative L2 error, stored rate   Eq. 1
+ *
+ * Pins (tests/test_oracle_*.py): brute-force E8 search, lattice invariants,
+ * second-moment constant 929/12960, hand-derived tie examples, field and rANS
+ * round trips, terminal-state/pointer invariants, the tile-metadata byte
+ * counts of the paper's tile-overhead table, Gibbs bound C_CE >= n*H, the
+ * conditioning-gain identity of Eq. 7, payload size against C_CE, sampled
+ * estimate against true stored size, least-squares optimality of Eq. 13,
+ * dtype rounding against library casts.
+ * Parity unpinned by the paper (fixed only by this build's stated readings):
+ * the coset tie rule, the integer frequency-normalisation rule, the row
+ * sampler, default tile size between the listed targets, the byte layout of
+ * tables and header.
+ *
+ * Parallelism: OpenMP over rows (quantisation) and over tiles (coding) only;
+ * the arithmetic of one row / one tile is untouched by it.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define EPO_NT 17          /* 1 coset table + 2 x 8 coordinate tables (Eq. 6) */
+#define EPO_J 32           /* interleaved rANS states per tile */
+#define EPO_L (1u << 15)   /* lower bound of the state interval [2^15, 2^31) */
+#define EPO_HEADER 64
+#define EPO_MAGIC 0x314B5045u /* "EPK1" little-endian */
+#define EPO_ETA 1e-12
+
+enum { EPO_BF16 = 0, EPO_FP16 = 1, EPO_E4M3 = 2, EPO_INT8 = 3, EPO_FP32 = 4 };
+
+typedef struct {
+    double bracket_lo, bracket_hi; /* scale bracket, default [1e-3, 8] */
+    int32_t search_steps;          /* I_s, default 12 */
+    uint32_t sample_vectors;       /* nominal sample budget, default 2^18 */
+    uint32_t tile_vectors;         /* V; 0 = default from the target rate */
+    int32_t b_start;               /* 0 = 11 for targets <= 7 bpp, else 12 */
+    int32_t b_max;                 /* default 15 */
+    double retained_bits;          /* constant of Eq. 10, default 16 */
+} epo_opts;
+
+typedef struct {
+    double s;            /* selected search scale (value of the fp32 used) */
+    int32_t b;           /* probability precision */
+    uint32_t V, n_tiles;
+    uint64_t total_words;
+    uint64_t bytes;      /* B_stored */
+    double stored_bpp;   /* Eq. 1 */
+    double est_bpp_sample; /* last sampled estimate of Eq. 12 at the chosen s */
+    double cce_bits;     /* C_CE of the final full-tensor tables */
+    double est_bytes_full; /* Eq. 10-11 evaluated on the full tensor */
+    uint32_t sample_rows;
+    int32_t coord_min, coord_max;
+} epo_report;
+
+typedef struct {
+    int32_t min;     /* smallest observed value (alphabet offset) */
+    uint32_t K;      /* max - min + 1, 0 if the table was never used */
+    uint64_t *n;     /* counts, K entries */
+    uint32_t *f;     /* b-bit frequencies, K entries */
+    uint32_t *F;     /* exclusive cumulative frequencies, K+1 entries */
+    uint64_t total;
+} epo_tab;
+
+/* ---------------------------------------------------------------- helpers */
+
+static inline uint32_t rd32(const uint8_t *p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
+static inline uint16_t rd16(const uint8_t *p) { return (uint16_t)(p[0] | (p[1] << 8)); }
+static inline void wr32(uint8_t *p, uint32_t v) { p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); p[2] = (uint8_t)(v >> 16); p[3] = (uint8_t)(v >> 24); }
+static inline void wr16(uint8_t *p, uint16_t v) { p[0] = (uint8_t)v; p[1] = (uint8_t)(v >> 8); }
+static inline uint64_t rd64(const uint8_t *p) { return (uint64_t)rd32(p) | ((uint64_t)rd32(p + 4) << 32); }
+static inline void wr64(uint8_t *p, uint64_t v) { wr32(p, (uint32_t)v); wr32(p + 4, (uint32_t)(v >> 32)); }
+
+void epo_default_opts(epo_opts *o) {
+    o->bracket_lo = 1e-3; o->bracket_hi = 8.0; o->search_steps = 12;
+    o->sample_vectors = 1u << 18; o->tile_vectors = 0; o->b_start = 0; o->b_max = 15;
+    o->retained_bits = 16.0;
+}
+
+void epo_free(void *p) { free(p); }
+
+int epo_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+void epo_set_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* table index: 0 = coset; field k (1..7 = z_k, 8 = m) under coset c -> 1 + 8c + (k-1) */
+static inline int tab_of(int c, int k) { return k == 0 ? 0 : 1 + 8 * c + (k - 1); }
+
+/* default tile size: the paper lists S = 32768, 16384, 8192, 4096 symbols at
+ * 2, 4, 7, 8 bpp; between them this build switches at 3, 5.5 and 7.5 bpp
+ * (reading; unpinned).  V = max(32, floor(S/9))  (App. "Tile layout and storage"). */
+uint32_t epo_default_tile_vectors(double target_bpp) {
+    uint32_t S = target_bpp < 3.0 ? 32768u : target_bpp < 5.5 ? 16384u : target_bpp < 7.5 ? 8192u : 4096u;
+    uint32_t V = S / 9u;
+    return V < 32u ? 32u : V;
+}
+
+/* ------------------------------------------------- Sec. 3.2: normalisation */
+
+/* mu_r = max(sqrt(mean_j x_rj^2), eta); sum in double in index order, rounded once to fp32 */
+float epo_row_rms(const float *x, uint32_t C) {
+    double acc = 0.0;
+    for (uint32_t j = 0; j < C; ++j) acc += (double)x[j] * (double)x[j];
+    double mu = sqrt(acc / (double)C);
+    if (!(mu > EPO_ETA)) mu = EPO_ETA;
+    return (float)mu;
+}
+
+/* ---------------------------------------------- Eq. 3: nearest point of D8 */
+static void nearest_d8(const float Y[8], int32_t z[8]) {
+    float d[8];
+    int64_t sum = 0;
+    for (int i = 0; i < 8; ++i) {
+        float f = rintf(Y[i]);          /* coordinate ties round to even */
+        z[i] = (int32_t)f;
+        d[i] = Y[i] - f;
+        sum += z[i];
+    }
+    int pi = (int)(((sum % 2) + 2) % 2);
+    if (pi) {
+        int js = 0;                     /* first coordinate of largest |d| */
+        float best = fabsf(d[0]);
+        for (int i = 1; i < 8; ++i) if (fabsf(d[i]) > best) { best = fabsf(d[i]); js = i; }
+        z[js] += (d[js] >= 0.0f) ? 1 : -1;   /* sign(0) = +1 */
+    }
+}
+
+/* Eq. 2: nearest point of E8 = D8 u (D8 + 1/2).  Output is the coset c and the
+ * integer part z (p = z + c/2).  Distances: residuals of the final candidates
+ * in fp32, squares summed in double in index order; the half coset wins only
+ * if strictly closer (reading; the paper is silent on this tie). */
+void epo_e8_nearest(const float Y[8], int32_t *c_out, int32_t z_out[8]) {
+    int32_t a[8], bz[8];
+    float Yh[8];
+    nearest_d8(Y, a);
+    for (int i = 0; i < 8; ++i) Yh[i] = Y[i] - 0.5f;
+    nearest_d8(Yh, bz);
+    double da = 0.0, db = 0.0;
+    for (int i = 0; i < 8; ++i) {
+        float ea = Y[i] - (float)a[i];
+        float eb = Yh[i] - (float)bz[i];
+        da += (double)ea * (double)ea;
+        db += (double)eb * (double)eb;
+    }
+    if (db < da) { *c_out = 1; memcpy(z_out, bz, sizeof(bz)); }
+    else         { *c_out = 0; memcpy(z_out, a, sizeof(a)); }
+}
+
+/* Eq. 4: (c, z) -> (c, z1..z7, m) */
+void epo_fields_from_point(int32_t c, const int32_t z[8], int32_t fld[9]) {
+    int64_t s7 = 0;
+    fld[0] = c;
+    for (int i = 0; i < 7; ++i) { fld[1 + i] = z[i]; s7 += z[i]; }
+    int pi = (int)(((s7 % 2) + 2) % 2);
+    fld[8] = (z[7] - pi) / 2;           /* exact: z8 and pi have equal parity */
+}
+
+/* Eq. 5: fields -> doubled point q = 2p (integers; p = q/2) */
+void epo_point2_from_fields(const int32_t fld[9], int32_t q[8]) {
+    int64_t s7 = 0;
+    int32_t c = fld[0];
+    for (int i = 0; i < 7; ++i) { q[i] = 2 * fld[1 + i] + c; s7 += fld[1 + i]; }
+    int pi = (int)(((s7 % 2) + 2) % 2);
+    q[7] = 2 * (2 * fld[8] + pi) + c;
+}
+
+/* quantise one row: X = x/mu (fp32 division), Y = X/s (fp32 division), Eq. 2, Eq. 4 */
+static void quantise_row(const float *x, uint32_t C, float mu, float s, int32_t *fld /* C/8*9 */) {
+    for (uint32_t v = 0; v < C / 8; ++v) {
+        float Y[8];
+        int32_t c, z[8];
+        for (int i = 0; i < 8; ++i) {
+            float X = x[8 * v + i] / mu;
+            Y[i] = X / s;
+        }
+        epo_e8_nearest(Y, &c, z);
+        epo_fields_from_point(c, z, fld + 9 * (size_t)v);
+    }
+}
+
+/* exported for tests: quantise a whole matrix at a given scale */
+void epo_quantise(const float *W, uint32_t R, uint32_t C, float s, int32_t *fields, float *mu_out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < (int64_t)R; ++r) {
+        float mu = epo_row_rms(W + (size_t)r * C, C);
+        if (mu_out) mu_out[r] = mu;
+        quantise_row(W + (size_t)r * C, C, mu, s, fields + (size_t)r * (C / 8) * 9);
+    }
+}
+
+/* -------------------------------------------- Sec. 3.3: tables and C_CE */
+
+static void tabs_free(epo_tab *t) {
+    for (int i = 0; i < EPO_NT; ++i) { free(t[i].n); free(t[i].f); free(t[i].F); }
+    memset(t, 0, sizeof(epo_tab) * EPO_NT);
+}
+
+/* counts n_{t,z} of the 17 distributions from a list of field tuples */
+static void tabs_count(const int32_t *fld, size_t nvec, epo_tab *t) {
+    int32_t lo[EPO_NT], hi[EPO_NT];
+    int used[EPO_NT];
+    memset(t, 0, sizeof(epo_tab) * EPO_NT);
+    for (int i = 0; i < EPO_NT; ++i) { used[i] = 0; lo[i] = 0; hi[i] = 0; }
+    for (size_t v = 0; v < nvec; ++v) {
+        const int32_t *a = fld + 9 * v;
+        int c = a[0];
+        for (int k = 0; k < 9; ++k) {
+            int ti = tab_of(c, k);
+            if (!used[ti]) { used[ti] = 1; lo[ti] = hi[ti] = a[k]; }
+            else { if (a[k] < lo[ti]) lo[ti] = a[k]; if (a[k] > hi[ti]) hi[ti] = a[k]; }
+        }
+    }
+    for (int i = 0; i < EPO_NT; ++i) {
+        if (!used[i]) continue;
+        t[i].min = lo[i];
+        t[i].K = (uint32_t)((int64_t)hi[i] - lo[i] + 1);
+        t[i].n = (uint64_t *)calloc(t[i].K, sizeof(uint64_t));
+    }
+    for (size_t v = 0; v < nvec; ++v) {
+        const int32_t *a = fld + 9 * v;
+        int c = a[0];
+        for (int k = 0; k < 9; ++k) {
+            epo_tab *tb = &t[tab_of(c, k)];
+            tb->n[a[k] - tb->min]++;
+            tb->total++;
+        }
+    }
+}
+
+/* number of symbols with a positive count, per table; A_max over coordinate tables */
+static uint32_t tabs_observed(const epo_tab *t, int ti) {
+    uint32_t o = 0;
+    for (uint32_t j = 0; j < t[ti].K; ++j) o += t[ti].n[j] > 0;
+    return o;
+}
+
+/* Sec. 3.3: integer frequencies summing to 2^b, every observed symbol >= 1.
+ * Rule (reading; the paper fixes only the two properties above):
+ *   f = max(1, floor(n * 2^b / total)) for n > 0; the deficit goes to the
+ *   largest f (lowest index on ties); an excess is taken from the current
+ *   largest f, at most f-1 at a time. */
+void epo_normalise_freqs(const uint64_t *n, uint32_t K, int b, uint32_t *f) {
+    uint64_t total = 0, M = 1ull << b;
+    for (uint32_t j = 0; j < K; ++j) total += n[j];
+    if (total == 0) { for (uint32_t j = 0; j < K; ++j) f[j] = 0; return; }
+    uint64_t sum = 0;
+    for (uint32_t j = 0; j < K; ++j) {
+        if (n[j] == 0) { f[j] = 0; continue; }
+        uint64_t q = (n[j] * M) / total;
+        f[j] = (uint32_t)(q < 1 ? 1 : q);
+        sum += f[j];
+    }
+    if (sum < M) {
+        uint32_t jm = 0;
+        for (uint32_t j = 1; j < K; ++j) if (f[j] > f[jm]) jm = j;
+        f[jm] += (uint32_t)(M - sum);
+    }
+    while (sum > M) {
+        uint32_t jm = 0;
+        for (uint32_t j = 1; j < K; ++j) if (f[j] > f[jm]) jm = j;
+        uint64_t take = sum - M;
+        if (take > (uint64_t)f[jm] - 1) take = f[jm] - 1;
+        f[jm] -= (uint32_t)take;
+        sum -= take;
+    }
+}
+
+static void tabs_normalise(epo_tab *t, int b) {
+    for (int i = 0; i < EPO_NT; ++i) {
+        if (t[i].K == 0) continue;
+        t[i].f = (uint32_t *)calloc(t[i].K, sizeof(uint32_t));
+        t[i].F = (uint32_t *)calloc(t[i].K + 1, sizeof(uint32_t));
+        epo_normalise_freqs(t[i].n, t[i].K, b, t[i].f);
+        for (uint32_t j = 0; j < t[i].K; ++j) t[i].F[j + 1] = t[i].F[j] + t[i].f[j];
+    }
+}
+
+/* Eq. 8: C_CE = sum_t sum_{z: n>0} n (b - log2 f), tables 0..16, symbols ascending */
+static double tabs_cce(const epo_tab *t, int b) {
+    double acc = 0.0;
+    for (int i = 0; i < EPO_NT; ++i)
+        for (uint32_t j = 0; j < t[i].K; ++j)
+            if (t[i].n[j] > 0) acc += (double)t[i].n[j] * ((double)b - log2((double)t[i].f[j]));
+    return acc;
+}
+
+/* bytes of the stored table section: i32 min[17], u32 K[17], u16 freq[sum K], padded to 4 */
+static uint64_t tabs_bytes(const epo_tab *t) {
+    uint64_t k = 0;
+    for (int i = 0; i < EPO_NT; ++i) k += t[i].K;
+    uint64_t by = 8ull * EPO_NT + 2ull * k;
+    return (by + 3ull) & ~3ull;
+}
+
+/* Eq. 10-11: estimated stored bits for nvec vectors in `rows` rows coded with tables t */
+static double estimate_bits(const epo_tab *t, int b, uint64_t nvec, uint64_t rows, uint32_t V, double retained, double *cce_out) {
+    double cce = tabs_cce(t, b);
+    uint64_t n_tile = (nvec + V - 1) / V;
+    double rem = cce - retained * (double)EPO_J * (double)n_tile;
+    if (rem < 0.0) rem = 0.0;
+    double L_payload = 16.0 * ceil(rem / 16.0);
+    double L_restart = (double)n_tile * (32.0 * EPO_J + 32.0) + 32.0;
+    double L_tables = 8.0 * (double)tabs_bytes(t);
+    double L_scales = 32.0 * (double)rows;
+    double L_other = 8.0 * EPO_HEADER;
+    if (cce_out) *cce_out = cce;
+    return L_payload + L_restart + L_tables + L_scales + L_other;
+}
+
+/* exported for tests: C_CE, estimate and entropy figures of a field list */
+void epo_model_stats(const int32_t *fields, uint64_t nvec, uint64_t rows, int b, uint32_t V, double retained,
+                     double *cce, double *est_bits, double *ideal_cond_bits, double *ideal_pooled_bits,
+                     uint32_t *observed /*17*/) {
+    epo_tab t[EPO_NT];
+    tabs_count(fields, nvec, t);
+    tabs_normalise(t, b);
+    double e = estimate_bits(t, b, nvec, rows, V, retained, cce);
+    if (est_bits) *est_bits = e;
+    if (ideal_cond_bits) {   /* sum n * H under the 17 empirical distributions */
+        double h = 0.0;
+        for (int i = 0; i < EPO_NT; ++i)
+            for (uint32_t j = 0; j < t[i].K; ++j)
+                if (t[i].n[j]) h -= (double)t[i].n[j] * log2((double)t[i].n[j] / (double)t[i].total);
+        *ideal_cond_bits = h;
+    }
+    if (ideal_pooled_bits) { /* coset table + 8 pooled coordinate tables (left side of Eq. 7) */
+        double h = 0.0;
+        for (uint32_t j = 0; j < t[0].K; ++j)
+            if (t[0].n[j]) h -= (double)t[0].n[j] * log2((double)t[0].n[j] / (double)t[0].total);
+        for (int k = 1; k <= 8; ++k) {
+            const epo_tab *a = &t[tab_of(0, k)], *bb = &t[tab_of(1, k)];
+            if (a->K == 0 && bb->K == 0) continue;
+            int64_t lo = a->K ? a->min : bb->min, hi = a->K ? (int64_t)a->min + a->K - 1 : (int64_t)bb->min + bb->K - 1;
+            if (bb->K) { if (bb->min < lo) lo = bb->min; if ((int64_t)bb->min + bb->K - 1 > hi) hi = (int64_t)bb->min + bb->K - 1; }
+            uint64_t tot = a->total + bb->total;
+            for (int64_t z = lo; z <= hi; ++z) {
+                uint64_t n = 0;
+                if (a->K && z >= a->min && z < (int64_t)a->min + a->K) n += a->n[z - a->min];
+                if (bb->K && z >= bb->min && z < (int64_t)bb->min + bb->K) n += bb->n[z - bb->min];
+                if (n) h -= (double)n * log2((double)n / (double)tot);
+            }
+        }
+        *ideal_pooled_bits = h;
+    }
+    if (observed) for (int i = 0; i < EPO_NT; ++i) observed[i] = tabs_observed(t, i);
+    tabs_free(t);
+}
+
+/* ------------------------------- App. "Scale-search settings": row sample */
+
+static uint64_t splitmix64(uint64_t *s) {
+    uint64_t z = (*s += 0x9E3779B97F4A7C15ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+static int cmp_u32(const void *a, const void *b) { uint32_t x = *(const uint32_t *)a, y = *(const uint32_t *)b; return x < y ? -1 : x > y; }
+
+/* complete rows, about `budget` vectors, shape-dependent seed, sorted ascending */
+uint32_t epo_sample_rows(uint32_t R, uint32_t C, uint32_t budget, uint32_t *rows_out /* R entries */) {
+    uint32_t per_row = C / 8;
+    uint32_t n = budget / per_row;
+    if (n < 1) n = 1;
+    if (n > R) n = R;
+    uint32_t *idx = (uint32_t *)malloc(sizeof(uint32_t) * R);
+    for (uint32_t i = 0; i < R; ++i) idx[i] = i;
+    uint64_t st = ((uint64_t)R << 32) + (uint64_t)C;
+    for (uint32_t i = 0; i < n; ++i) {      /* partial Fisher-Yates */
+        uint32_t j = i + (uint32_t)(splitmix64(&st) % (uint64_t)(R - i));
+        uint32_t tmp = idx[i]; idx[i] = idx[j]; idx[j] = tmp;
+    }
+    qsort(idx, n, sizeof(uint32_t), cmp_u32);
+    memcpy(rows_out, idx, sizeof(uint32_t) * n);
+    free(idx);
+    return n;
+}
+
+/* -------------------------------------------- App. tiled rANS: one tile */
+
+typedef struct { uint16_t *w; size_t n, cap; } wordbuf;
+static void wb_push(wordbuf *b, uint16_t v) {
+    if (b->n == b->cap) { b->cap = b->cap ? 2 * b->cap : 1024; b->w = (uint16_t *)realloc(b->w, b->cap * sizeof(uint16_t)); }
+    b->w[b->n++] = v;
+}
+
+/* Encode the nv vectors of one tile.  Decode order is: group g of 32 vectors,
+ * field k = 0 (coset) .. 8 (m), lane 0..31, vector g*32+lane on state `lane`;
+ * after each symbol a lane whose state fell below 2^15 takes the next 16-bit
+ * word.  The encoder walks that order backwards (so each vector's m, z7..z1
+ * and then its coset, as the paper states) and reverses its word list.
+ * Eq. 17 with renormalisation before the update: emit while xi >= f * 2^(31-b). */
+static void encode_tile(const int32_t *fld, uint32_t nv, const epo_tab *t, int b, uint32_t states[EPO_J], wordbuf *out) {
+    uint32_t xi[EPO_J];
+    for (int l = 0; l < EPO_J; ++l) xi[l] = EPO_L;
+    uint32_t G = (nv + 31) / 32;
+    size_t start = out->n;
+    for (int64_t g = (int64_t)G - 1; g >= 0; --g)
+        for (int k = 8; k >= 0; --k)
+            for (int l = EPO_J - 1; l >= 0; --l) {
+                uint64_t i = (uint64_t)g * 32 + (uint64_t)l;
+                if (i >= nv) continue;
+                const int32_t *a = fld + 9 * i;
+                const epo_tab *tb = &t[tab_of(a[0], k)];
+                uint32_t sym = (uint32_t)(a[k] - tb->min);
+                uint32_t f = tb->f[sym], F = tb->F[sym];
+                uint64_t lim = (uint64_t)f << (31 - b);
+                if ((uint64_t)xi[l] >= lim) { wb_push(out, (uint16_t)(xi[l] & 0xFFFFu)); xi[l] >>= 16; }
+                xi[l] = ((xi[l] / f) << b) + (xi[l] % f) + F;
+            }
+    for (size_t i = start, j = out->n; i + 1 < j; ++i) { --j; uint16_t tmp = out->w[i]; out->w[i] = out->w[j]; out->w[j] = tmp; }
+    memcpy(states, xi, sizeof(xi));
+}
+
+/* parsed view of a stored representation */
+typedef struct {
+    uint32_t R, C, V, n_tiles, b;
+    int32_t coord_min, coord_max;
+    uint32_t off_tables, off_scales, off_tiles, off_payload;
+    uint64_t total_bytes, total_words;
+    int32_t tmin[EPO_NT];
+    uint32_t tK[EPO_NT];
+    const uint8_t *freq[EPO_NT];
+} epo_view;
+
+static int parse(const uint8_t *blob, size_t n, epo_view *v) {
+    if (n < EPO_HEADER || rd32(blob) != EPO_MAGIC || rd16(blob + 4) != 1 || blob[7] != EPO_J) return -1;
+    v->b = blob[6];
+    v->R = rd32(blob + 8); v->C = rd32(blob + 12); v->V = rd32(blob + 16); v->n_tiles = rd32(blob + 20);
+    v->coord_min = (int16_t)rd16(blob + 28); v->coord_max = (int16_t)rd16(blob + 30);
+    v->off_tables = rd32(blob + 32); v->off_scales = rd32(blob + 36); v->off_tiles = rd32(blob + 40); v->off_payload = rd32(blob + 44);
+    v->total_bytes = rd64(blob + 48); v->total_words = rd32(blob + 56);
+    if (v->b < 9 || v->b > 15 || v->C % 8 || v->V == 0 || v->total_bytes != n) return -2;
+    uint64_t nvec = (uint64_t)v->R * (v->C / 8);
+    if ((nvec + v->V - 1) / v->V != v->n_tiles) return -3;
+    if (v->off_tables != EPO_HEADER) return -4;
+    const uint8_t *p = blob + v->off_tables;
+    uint64_t ksum = 0;
+    for (int i = 0; i < EPO_NT; ++i) { v->tmin[i] = (int32_t)rd32(p + 4 * i); v->tK[i] = rd32(p + 4 * EPO_NT + 4 * i); ksum += v->tK[i]; }
+    uint64_t tb = (8ull * EPO_NT + 2ull * ksum + 3ull) & ~3ull;
+    if (v->off_scales != v->off_tables + tb) return -5;
+    if (v->off_tiles != v->off_scales + 4ull * v->R) return -6;
+    if (v->off_payload != v->off_tiles + 132ull * v->n_tiles + 4ull) return -7;
+    if (v->total_bytes != v->off_payload + 2ull * v->total_words) return -8;
+    const uint8_t *fq = p + 8 * EPO_NT;
+    for (int i = 0; i < EPO_NT; ++i) { v->freq[i] = fq; fq += 2ull * v->tK[i]; }
+    return 0;
+}
+
+/* ---------------------------------------------------- reconstruction side */
+
+/* round a finite double that came from an fp32 value to a binary format with
+ * `mbits` stored mantissa bits and minimum normal exponent `emin`, ties to even,
+ * subnormals included.  Returns the rounded value as a double. */
+static double round_to_format(double x, int mbits, int emin) {
+    if (x == 0.0 || !isfinite(x)) return x;
+    int e;
+    frexp(fabs(x), &e);        /* |x| = m * 2^e, m in [0.5, 1) -> floor(log2|x|) = e - 1 */
+    int ex = e - 1;
+    if (ex < emin) ex = emin;
+    double ulp = ldexp(1.0, ex - mbits);
+    return rint(x / ulp) * ulp;   /* division by a power of two is exact; rint ties to even */
+}
+
+static uint16_t snap_bf16(float v) {
+    if (isnan(v)) return 0x7FC0;
+    double r = round_to_format((double)v, 7, -126);
+    float fr = (float)r;          /* exact, or +-inf when the rounding left the fp32 range */
+    uint32_t u; memcpy(&u, &fr, 4);
+    return (uint16_t)(u >> 16);
+}
+
+static uint16_t snap_fp16(float v) {  /* RNE, saturating to +-65504 */
+    if (isnan(v)) return 0x7FFF;
+    double r = round_to_format((double)v, 10, -14);
+    uint16_t sign = signbit(v) ? 0x8000 : 0;
+    double a = fabs(r);
+    if (a > 65504.0) return (uint16_t)(sign | 0x7BFF);
+    if (a == 0.0) return sign;
+    int e; double m = frexp(a, &e);   /* a = m 2^e, m in [0.5,1) */
+    int ex = e - 1;
+    if (ex < -14) return (uint16_t)(sign | (uint16_t)(a / ldexp(1.0, -24)));      /* subnormal: multiples of 2^-24 */
+    uint16_t man = (uint16_t)((m * 2.0 - 1.0) * 1024.0);
+    return (uint16_t)(sign | ((ex + 15) << 10) | man);
+}
+
+static uint8_t snap_e4m3(float v) {   /* FP8 E4M3FN: RNE incl. subnormals (step 2^-9), saturating to +-448 */
+    if (isnan(v)) return 0x7F;
+    double r = round_to_format((double)v, 3, -6);
+    uint8_t sign = signbit(v) ? 0x80 : 0;
+    double a = fabs(r);
+    if (a > 448.0) return (uint8_t)(sign | 0x7E);
+    if (a == 0.0) return sign;
+    int e; double m = frexp(a, &e);
+    int ex = e - 1;
+    if (ex < -6) return (uint8_t)(sign | (uint8_t)(a / ldexp(1.0, -9)));
+    uint8_t man = (uint8_t)((m * 2.0 - 1.0) * 8.0);
+    return (uint8_t)(sign | ((ex + 7) << 3) | man);
+}
+
+static int8_t snap_int8(float v) {
+    if (isnan(v)) return 0;
+    double r = rint((double)v);
+    if (r > 127.0) r = 127.0;
+    if (r < -128.0) r = -128.0;
+    return (int8_t)r;
+}
+
+/* exported for tests: snap an fp32 array to a dtype (Eq. 19's snap_tau) */
+void epo_snap(const float *v, size_t n, int dtype, void *out) {
+    for (size_t i = 0; i < n; ++i) {
+        switch (dtype) {
+        case EPO_BF16: ((uint16_t *)out)[i] = snap_bf16(v[i]); break;
+        case EPO_FP16: ((uint16_t *)out)[i] = snap_fp16(v[i]); break;
+        case EPO_E4M3: ((uint8_t *)out)[i] = snap_e4m3(v[i]); break;
+        case EPO_INT8: ((int8_t *)out)[i] = snap_int8(v[i]); break;
+        default: ((float *)out)[i] = v[i]; break;
+        }
+    }
+}
+
+static size_t dtype_size(int dtype) { return dtype == EPO_FP32 ? 4 : (dtype == EPO_BF16 || dtype == EPO_FP16) ? 2 : 1; }
+
+/* Decode one tile (Eq. 18, Eq. 5, Eq. 19).  Writes weights to `out` (whole-
+ * tensor base, dtype tau) when out != NULL and the nine fields per vector to
+ * `fields` (whole-tensor base) when fields != NULL.  Returns 0, or a negative
+ * code if the stream is inconsistent (slot outside every interval, pointer
+ * beyond the tile, final states not 2^15, pointer not at the next offset). */
+static int decode_tile(const uint8_t *blob, const epo_view *v, uint32_t tile, const float *scales,
+                       const uint32_t *const *lut_sym, const uint32_t *const *tf, const uint32_t *const *tF,
+                       int dtype, void *out, int32_t *fields) {
+    const uint8_t *rec = blob + v->off_tiles + 132ull * tile;
+    uint32_t xi[EPO_J];
+    for (int l = 0; l < EPO_J; ++l) xi[l] = rd32(rec + 4 * l);
+    uint64_t ptr = rd32(rec + 128);
+    /* end of this tile's words: the next tile's offset, or the final boundary offset */
+    uint64_t end = (tile + 1 < v->n_tiles) ? rd32(rec + 132 + 128) : rd32(rec + 132);
+    const uint8_t *pay = blob + v->off_payload;
+    uint64_t nvec = (uint64_t)v->R * (v->C / 8);
+    uint64_t v0 = (uint64_t)tile * v->V;
+    uint32_t nv = (uint32_t)((nvec - v0) < v->V ? (nvec - v0) : v->V);
+    uint32_t M = 1u << v->b;
+    uint32_t per_row = v->C / 8;
+    uint32_t G = (nv + 31) / 32;
+    int32_t (*a)[9] = (int32_t (*)[9])malloc(sizeof(int32_t) * 9 * EPO_J);
+    int rc = 0;
+    for (uint32_t g = 0; g < G && !rc; ++g) {
+        for (int k = 0; k < 9 && !rc; ++k)
+            for (int l = 0; l < EPO_J; ++l) {
+                uint64_t i = (uint64_t)g * 32 + (uint64_t)l;
+                if (i >= nv) continue;
+                int ti = tab_of(k == 0 ? 0 : a[l][0], k);
+                if (v->tK[ti] == 0) { rc = -20; break; }
+                uint32_t u = xi[l] & (M - 1);
+                uint32_t sym = lut_sym[ti][u];
+                uint32_t f = tf[ti][sym], F = tF[ti][sym];
+                xi[l] = f * (xi[l] >> v->b) + u - F;          /* Eq. 18 */
+                if (xi[l] < EPO_L) {                          /* renormalise: one 16-bit word */
+                    if (ptr >= end) { rc = -21; break; }
+                    xi[l] = (xi[l] << 16) | rd16(pay + 2 * ptr);
+                    ++ptr;
+                }
+                a[l][k] = (int32_t)sym + v->tmin[ti];
+            }
+        if (rc) break;
+        for (int l = 0; l < EPO_J; ++l) {
+            uint64_t i = (uint64_t)g * 32 + (uint64_t)l;
+            if (i >= nv) continue;
+            uint64_t gv = v0 + i;                 /* flat row-major vector index */
+            if (fields) memcpy(fields + 9 * gv, a[l], sizeof(int32_t) * 9);
+            if (out) {
+                int32_t q[8];
+                float w[8];
+                epo_point2_from_fields(a[l], q);
+                float sig = scales[gv / per_row];
+                for (int j = 0; j < 8; ++j) {
+                    float p = (float)q[j] * 0.5f;         /* Eq. 5: half-integers are exact in fp32 */
+                    w[j] = sig * p;                       /* Eq. 19: one fp32 multiply */
+                }
+                epo_snap(w, 8, dtype, (uint8_t *)out + 8 * gv * dtype_size(dtype));
+            }
+        }
+    }
+    free(a);
+    if (!rc) {
+        for (int l = 0; l < EPO_J; ++l) if (xi[l] != EPO_L) rc = -22;
+        if (ptr != end) rc = -23;
+    }
+    return rc;
+}
+
+/* Decode tiles [t0, t1) of a stored representation.  `scales` overrides the
+ * stored row scales when not NULL.  Either of out / fields may be NULL. */
+int epo_decode_tiles(const uint8_t *blob, size_t n, uint32_t t0, uint32_t t1, const float *scales,
+                     int dtype, void *out, int32_t *fields) {
+    epo_view v;
+    int rc = parse(blob, n, &v);
+    if (rc) return rc;
+    if (t1 > v.n_tiles || t0 > t1) return -10;
+    uint32_t M = 1u << v.b;
+    uint32_t *lut[EPO_NT], *tf[EPO_NT], *tF[EPO_NT];
+    for (int i = 0; i < EPO_NT; ++i) {      /* slot -> symbol lookup from the stored frequencies */
+        lut[i] = NULL; tf[i] = NULL; tF[i] = NULL;
+        if (v.tK[i] == 0) continue;
+        tf[i] = (uint32_t *)malloc(sizeof(uint32_t) * v.tK[i]);
+        tF[i] = (uint32_t *)malloc(sizeof(uint32_t) * (v.tK[i] + 1));
+        lut[i] = (uint32_t *)malloc(sizeof(uint32_t) * M);
+        uint32_t acc = 0;
+        for (uint32_t j = 0; j < v.tK[i]; ++j) {
+            tf[i][j] = rd16(v.freq[i] + 2 * j);
+            tF[i][j] = acc;
+            for (uint32_t u = acc; u < acc + tf[i][j] && u < M; ++u) lut[i][u] = j;
+            acc += tf[i][j];
+        }
+        tF[i][v.tK[i]] = acc;
+        if (acc != M) rc = -11;
+    }
+    float *sc = NULL;
+    if (!scales) {
+        sc = (float *)malloc(sizeof(float) * v.R);
+        memcpy(sc, blob + v.off_scales, sizeof(float) * v.R);
+        scales = sc;
+    }
+    if (!rc) {
+        int err = 0;
+#pragma omp parallel for schedule(dynamic, 4)
+        for (int64_t t = t0; t < (int64_t)t1; ++t) {
+            int r = decode_tile(blob, &v, (uint32_t)t, scales, (const uint32_t *const *)lut, (const uint32_t *const *)tf,
+                                (const uint32_t *const *)tF, dtype, out, fields);
+            if (r) {
+#pragma omp critical
+                err = r;
+            }
+        }
+        rc = err;
+    }
+    for (int i = 0; i < EPO_NT; ++i) { free(lut[i]); free(tf[i]); free(tF[i]); }
+    free(sc);
+    return rc;
+}
+
+int epo_decode(const uint8_t *blob, size_t n, const float *scales, int dtype, void *out, int32_t *fields) {
+    epo_view v;
+    int rc = parse(blob, n, &v);
+    if (rc) return rc;
+    return epo_decode_tiles(blob, n, 0, v.n_tiles, scales, dtype, out, fields);
+}
+
+/* header fields for tests and drivers: R, C, V, n_tiles, b, coord_min, coord_max, offsets, words */
+int epo_info(const uint8_t *blob, size_t n, uint64_t out[16]) {
+    epo_view v;
+    int rc = parse(blob, n, &v);
+    if (rc) return rc;
+    out[0] = v.R; out[1] = v.C; out[2] = v.V; out[3] = v.n_tiles; out[4] = v.b;
+    out[5] = (uint64_t)(int64_t)v.coord_min; out[6] = (uint64_t)(int64_t)v.coord_max;
+    out[7] = v.off_tables; out[8] = v.off_scales; out[9] = v.off_tiles; out[10] = v.off_payload;
+    out[11] = v.total_bytes; out[12] = v.total_words;
+    float s; memcpy(&s, blob + 24, 4); out[13] = 0; memcpy(&out[13], &s, 4);
+    out[14] = out[15] = 0;
+    return 0;
+}
+
+/* --------------------------------------------- pack fields into a stream */
+
+/* Final tables from the full-tensor fields, tile encode, stored representation.
+ * fields: [nvec][9]; sigma: R fp32 row scales; s_info: search scale (header, informational). */
+int epo_pack(const int32_t *fields, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
+             uint8_t **blob_out, size_t *n_out, double *cce_out) {
+    uint64_t nvec = (uint64_t)R * (C / 8);
+    if (C % 8 || nvec == 0 || nvec >= (1ull << 32) || V == 0 || b < 9 || b > 15) return -1;
+    epo_tab t[EPO_NT];
+    tabs_count(fields, nvec, t);
+    for (int i = 0; i < EPO_NT; ++i) if (tabs_observed(t, i) > (1u << b)) { tabs_free(t); return -2; }
+    tabs_normalise(t, b);
+    if (cce_out) *cce_out = tabs_cce(t, b);
+    uint32_t n_tiles = (uint32_t)((nvec + V - 1) / V);
+    wordbuf *tw = (wordbuf *)calloc(n_tiles, sizeof(wordbuf));
+    uint32_t *states = (uint32_t *)malloc(sizeof(uint32_t) * EPO_J * (size_t)n_tiles);
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t tI = 0; tI < (int64_t)n_tiles; ++tI) {
+        uint64_t v0 = (uint64_t)tI * V;
+        uint32_t nv = (uint32_t)((nvec - v0) < V ? (nvec - v0) : V);
+        encode_tile(fields + 9 * v0, nv, t, b, states + EPO_J * (size_t)tI, &tw[tI]);
+    }
+    uint64_t words = 0;
+    for (uint32_t i = 0; i < n_tiles; ++i) words += tw[i].n;
+    /* coordinate range over z_1..z_8 (z_8 = 2m + parity lies in [2 m_min, 2 m_max + 1]) */
+    int64_t cmin = 0, cmax = 0; int any = 0;
+    for (int c = 0; c < 2; ++c) for (int k = 1; k <= 8; ++k) {
+        const epo_tab *tb = &t[tab_of(c, k)];
+        if (!tb->K) continue;
+        int64_t lo = tb->min, hi = (int64_t)tb->min + tb->K - 1;
+        if (k == 8) { lo = 2 * lo; hi = 2 * hi + 1; }
+        if (!any) { cmin = lo; cmax = hi; any = 1; } else { if (lo < cmin) cmin = lo; if (hi > cmax) cmax = hi; }
+    }
+    if (cmin < -32768) cmin = -32768;
+    if (cmax > 32767) cmax = 32767;
+    uint64_t tb_bytes = tabs_bytes(t);
+    uint64_t off_tables = EPO_HEADER, off_scales = off_tables + tb_bytes, off_tiles = off_scales + 4ull * R;
+    uint64_t off_payload = off_tiles + 132ull * n_tiles + 4ull, total = off_payload + 2ull * words;
+    if (total >= (1ull << 32) || words >= (1ull << 32)) { /* 32-bit offsets */
+        for (uint32_t i = 0; i < n_tiles; ++i) free(tw[i].w);
+        free(tw); free(states); tabs_free(t); return -3;
+    }
+    uint8_t *blob = (uint8_t *)calloc(1, total);
+    wr32(blob, EPO_MAGIC); wr16(blob + 4, 1); blob[6] = (uint8_t)b; blob[7] = EPO_J;
+    wr32(blob + 8, R); wr32(blob + 12, C); wr32(blob + 16, V); wr32(blob + 20, n_tiles);
+    memcpy(blob + 24, &s_info, 4);
+    wr16(blob + 28, (uint16_t)(int16_t)cmin); wr16(blob + 30, (uint16_t)(int16_t)cmax);
+    wr32(blob + 32, (uint32_t)off_tables); wr32(blob + 36, (uint32_t)off_scales);
+    wr32(blob + 40, (uint32_t)off_tiles); wr32(blob + 44, (uint32_t)off_payload);
+    wr64(blob + 48, total); wr32(blob + 56, (uint32_t)words); wr32(blob + 60, 0);
+    uint8_t *p = blob + off_tables;
+    for (int i = 0; i < EPO_NT; ++i) { wr32(p + 4 * i, (uint32_t)t[i].min); wr32(p + 4 * EPO_NT + 4 * i, t[i].K); }
+    uint8_t *fq = p + 8 * EPO_NT;
+    for (int i = 0; i < EPO_NT; ++i) for (uint32_t j = 0; j < t[i].K; ++j) { wr16(fq, (uint16_t)t[i].f[j]); fq += 2; }
+    memcpy(blob + off_scales, sigma, 4ull * R);
+    uint64_t w = 0;
+    for (uint32_t i = 0; i < n_tiles; ++i) {
+        uint8_t *rec = blob + off_tiles + 132ull * i;
+        for (int l = 0; l < EPO_J; ++l) wr32(rec + 4 * l, states[EPO_J * (size_t)i + l]);
+        wr32(rec + 128, (uint32_t)w);
+        for (size_t j = 0; j < tw[i].n; ++j) wr16(blob + off_payload + 2 * (w + j), tw[i].w[j]);
+        w += tw[i].n;
+        free(tw[i].w);
+    }
+    wr32(blob + off_tiles + 132ull * n_tiles, (uint32_t)w);   /* final boundary offset */
+    free(tw); free(states); tabs_free(t);
+    *blob_out = blob; *n_out = (size_t)total;
+    return 0;
+}
+
+/* -------------------------------------------------- Eq. 13: row-scale refit */
+void epo_refit(const float *W, uint32_t R, uint32_t C, const int32_t *fields, float s, const float *mu, float *sigma) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < (int64_t)R; ++r) {
+        double sxp = 0.0, spp = 0.0;
+        for (uint32_t v = 0; v < C / 8; ++v) {
+            int32_t q[8];
+            epo_point2_from_fields(fields + 9 * ((size_t)r * (C / 8) + v), q);
+            for (int j = 0; j < 8; ++j) {
+                double p = 0.5 * (double)q[j];
+                sxp += (double)W[(size_t)r * C + 8 * v + j] * p;
+                spp += p * p;
+            }
+        }
+        double sg;
+        if (spp > 0.0) { sg = sxp / spp; if (!(sg > EPO_ETA)) sg = EPO_ETA; }
+        else sg = (double)s * (double)mu[r];
+        sigma[r] = (float)sg;
+    }
+}
+
+/* --------------------------------- Algorithm 1 + packing: the whole encoder */
+int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const epo_opts *opts_in,
+               uint8_t **blob_out, size_t *n_out, epo_report *rep) {
+    epo_opts o;
+    if (opts_in) o = *opts_in; else epo_default_opts(&o);
+    if (!W || R == 0 || C == 0 || C % 8 || !(target_bpp > 0.0)) return -1;
+    uint64_t nvec = (uint64_t)R * (C / 8);
+    if (nvec >= (1ull << 32)) return -1;
+    uint32_t V = o.tile_vectors ? o.tile_vectors : epo_default_tile_vectors(target_bpp);
+    int b0 = o.b_start ? o.b_start : (target_bpp <= 7.0 ? 11 : 12);
+    float *mu = (float *)malloc(sizeof(float) * R);
+    for (uint32_t r = 0; r < R; ++r) mu[r] = epo_row_rms(W + (size_t)r * C, C);
+
+    uint32_t *srows = (uint32_t *)malloc(sizeof(uint32_t) * R);
+    uint32_t ns = epo_sample_rows(R, C, o.sample_vectors, srows);
+    uint64_t svec = (uint64_t)ns * (C / 8);
+    int32_t *sf = (int32_t *)malloc(sizeof(int32_t) * 9 * svec);
+    int32_t *fields = (int32_t *)malloc(sizeof(int32_t) * 9 * nvec);
+    float s32 = 0.0f;
+    double last_est = 0.0;
+    int b = b0, done = 0;
+    for (b = b0; b <= o.b_max && !done; ++b) {
+        double lo = o.bracket_lo, hi = o.bracket_hi;
+        for (int it = 0; it < o.search_steps; ++it) {
+            double s = sqrt(lo * hi);
+            float sq = (float)s;
+#pragma omp parallel for schedule(static)
+            for (int64_t i = 0; i < (int64_t)ns; ++i)
+                quantise_row(W + (size_t)srows[i] * C, C, mu[srows[i]], sq, sf + 9 * (size_t)i * (C / 8));
+            epo_tab t[EPO_NT];
+            tabs_count(sf, svec, t);
+            tabs_normalise(t, b);
+            double bits = estimate_bits(t, b, svec, ns, V, o.retained_bits, NULL);
+            tabs_free(t);
+            double rate = bits / (8.0 * (double)svec);   /* = 8 * B_sub / N_sub */
+            last_est = rate;
+            if (rate > target_bpp) lo = s; else hi = s;
+        }
+        s32 = (float)sqrt(lo * hi);
+        for (;;) {
+#pragma omp parallel for schedule(static)
+            for (int64_t r = 0; r < (int64_t)R; ++r)
+                quantise_row(W + (size_t)r * C, C, mu[r], s32, fields + 9 * (size_t)r * (C / 8));
+            epo_tab t[EPO_NT];
+            tabs_count(fields, nvec, t);
+            uint32_t amax = 0, worst = 0;
+            for (int i = 0; i < EPO_NT; ++i) {
+                uint32_t ob = tabs_observed(t, i);
+                if (ob > worst) worst = ob;
+                if (i > 0 && ob > amax) amax = ob;
+            }
+            tabs_free(t);
+            if (worst <= (1u << b)) { done = 1; break; }
+            if (b < o.b_max) break;                       /* raise b and search again */
+            s32 = (float)(1.05 * (double)s32 * (double)amax / (double)(1u << b));   /* coarsen */
+        }
+        if (done) break;
+    }
+    float *sigma = (float *)malloc(sizeof(float) * R);
+    epo_refit(W, R, C, fields, s32, mu, sigma);
+    double cce = 0.0;
+    int rc = epo_pack(fields, R, C, b, V, sigma, s32, blob_out, n_out, &cce);
+    if (!rc && rep) {
+        epo_view v; parse(*blob_out, *n_out, &v);
+        rep->s = (double)s32; rep->b = b; rep->V = V; rep->n_tiles = v.n_tiles; rep->total_words = v.total_words;
+        rep->bytes = *n_out; rep->stored_bpp = 8.0 * (double)*n_out / ((double)R * (double)C);
+        rep->est_bpp_sample = last_est; rep->cce_bits = cce; rep->sample_rows = ns;
+        rep->coord_min = v.coord_min; rep->coord_max = v.coord_max;
+        epo_tab t[EPO_NT];
+        tabs_count(fields, nvec, t); tabs_normalise(t, b);
+        rep->est_bytes_full = estimate_bits(t, b, nvec, R, V, o.retained_bits, NULL) / 8.0;
+        tabs_free(t);
+    }
+    free(mu); free(srows); free(sf); free(fields); free(sigma);
+    return rc;
+}
+
+/* Eq. 1: relative L2 error in double */
+double epo_rel_l2(const float *W, const float *What, size_t n) {
+    double num = 0.0, den = 0.0;
+    for (size_t i = 0; i < n; ++i) {
+        double d = (double)What[i] - (double)W[i];
+        num += d * d;
+        den += (double)W[i] * (double)W[i];
+    }
+    return sqrt(num / den);
+}
