@@ -1,0 +1,189 @@
+/*
+ * entropack.h -- C ABI of the B200-native EntroPack weight codec.
+ *
+ * EntroPack (arxiv 2609.34185) stores a weight matrix W[R][C] (C divisible by 8) as tiled,
+ * 32-way interleaved rANS streams of E8 lattice-coordinate fields under a coset-conditioned
+ * probability model, and reconstructs W-hat = snap_tau(sigma_r * p) on the GPU in one fused pass.
+ *
+ * Two halves:
+ *   host  : ep_encode() and friends build the stored representation ("blob") on the CPU
+ *           (paper Sec. 3.2-3.6, Algorithm 1, Eq. 13, Eq. 17).
+ *   device: ep_decode_tensor() / ep_decode_batch() enqueue the fused sm_100a decode kernel
+ *           (paper Sec. 3.7, Eq. 18, Eq. 5, Eq. 19).  There is no CPU decode path.
+ *
+ * Conventions
+ *   - every function returns 0 (EP_OK) or a negative ep_status; no exceptions cross the ABI;
+ *   - "host" pointers are ordinary memory, "device" pointers are CUDA global memory of the
+ *     current device; the library never allocates or frees device memory and never
+ *     synchronises inside a decode call: work is enqueued on the given stream;
+ *   - `stream` arguments are cudaStream_t handles passed as void* (NULL = default stream);
+ *   - all multi-byte stream fields are little-endian.
+ *
+ * Stored representation (all of it counts toward the stored rate of Eq. 1):
+ *   [header 64 B]   magic "EPK1", u16 version=1, u8 b, u8 J=32, u32 R, u32 C, u32 V, u32 n_tiles,
+ *                   f32 s (informational), i16 coord_min, i16 coord_max, u32 byte offsets of the four
+ *                   sections below, u64 total bytes, u32 total payload words, u32 zero
+ *   [tables]        i32 min[17], u32 K[17], then u16 freq[K_t] for t = 0..16, padded to 4 bytes.
+ *                   t = 0 is the coset table; field k (1..7 = z_k, 8 = m) under coset c is
+ *                   t = 1 + 8c + (k-1).  Frequencies of a non-empty table sum to 2^b.
+ *   [row scales]    R x f32
+ *   [tile index]    n_tiles x { u32 state[32], u32 word_offset }, then u32 final boundary offset
+ *                   (132 bytes per tile + 4, as in the paper's tile-overhead table)
+ *   [payload]       16-bit words of all tiles, concatenated, no padding
+ * Tile t holds vectors [t*V, min((t+1)*V, R*C/8)) of the row-major sequence of 8-weight blocks.
+ * Inside a tile, vector i uses rANS state i mod 32; decoding proceeds by groups of 32 vectors,
+ * within a group by field (coset first, then z1..z7, m), within a field by lane 0..31; after its
+ * symbol a lane whose state is below 2^15 takes the next payload word.
+ */
+#ifndef ENTROPACK_H
+#define ENTROPACK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EP_NUM_TABLES 17
+#define EP_MAX_BATCH 16
+
+typedef enum {
+    EP_OK = 0,
+    EP_ERR_BAD_ARG = -1,     /* NULL pointer, C % 8 != 0, size out of range, misaligned output */
+    EP_ERR_BAD_STREAM = -2,  /* blob fails structural validation, or the decoder found an inconsistency */
+    EP_ERR_UNSUPPORTED = -3, /* valid request this build cannot serve (e.g. offsets beyond 32 bits) */
+    EP_ERR_CUDA = -4,        /* a CUDA runtime call failed */
+    EP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out */
+    EP_ERR_NOMEM = -6,       /* host allocation failed */
+    EP_ERR_SCRATCH = -7      /* scratch buffer missing, misaligned or too small */
+} ep_status;
+
+/* Output element types of the decoder: snap_tau of Eq. 19. */
+typedef enum {
+    EP_BF16 = 0,        /* round to nearest even */
+    EP_FP16 = 1,        /* round to nearest even, saturating to +-65504 */
+    EP_FP8_E4M3 = 2,    /* E4M3FN, round to nearest even incl. subnormals, saturating to +-448 */
+    EP_INT8 = 3,        /* round to nearest even integer, saturating to [-128, 127] */
+    EP_FIELDS_I32 = 16  /* verification mode: the nine decoded fields (c, z1..z7, m) of Eq. 4 as
+                           int32[R*C/8][9]; row scales are not read */
+} ep_dtype;
+
+/* Encoder settings; ep_encode_opts_default() fills in the paper's values
+ * (App. "Scale-search settings", App. "Tile layout and storage"). */
+typedef struct {
+    double bracket_lo, bracket_hi; /* geometric search bracket for s: [1e-3, 8] */
+    int32_t search_steps;          /* I_s = 12 bisection steps */
+    uint32_t sample_vectors;       /* nominal row-sample budget: 2^18 eight-vectors */
+    uint32_t tile_vectors;         /* V; 0 = max(32, floor(S/9)) with S from the target rate */
+    int32_t b_start;               /* 0 = 11 for targets <= 7 bpp, 12 above */
+    int32_t b_max;                 /* 15 */
+    double retained_bits;          /* constant of Eq. 10 (bits assumed to stay in each state): 16 */
+    int32_t threads;               /* host worker threads; 0 = all hardware threads */
+} ep_encode_opts;
+
+/* What the encoder decided; filled by ep_blob_report(). */
+typedef struct {
+    double s;               /* selected search scale */
+    double stored_bpp;      /* Eq. 1: 8 * bytes / (R*C) */
+    double est_bpp_sample;  /* Eq. 12 at the last evaluated candidate of the chosen precision */
+    double cce_bits;        /* Eq. 8 on the final full-tensor tables */
+    uint64_t bytes;
+    uint32_t sample_rows;
+    int32_t b;
+} ep_encode_report;
+
+/* Host-side description of a blob: a copy of its header and table directory.  Obtained once from
+ * the host copy of the blob with ep_blob_info() and handed to the decode calls, which therefore
+ * never read device memory on the host. */
+typedef struct {
+    uint32_t R, C, V, n_tiles;
+    uint32_t b, J;
+    int32_t coord_min, coord_max;     /* range of the integer coordinates z_1..z_8 over the tensor */
+    float s;
+    uint32_t off_tables, off_scales, off_tiles, off_payload;  /* byte offsets inside the blob */
+    uint64_t total_bytes;
+    uint64_t total_words;
+    int32_t table_min[EP_NUM_TABLES];   /* alphabet offset of each table */
+    uint32_t table_K[EP_NUM_TABLES];    /* stored entries of each table (0 = table never used) */
+} ep_info;
+
+typedef struct ep_blob ep_blob;   /* host-owned stored representation */
+
+/* One tensor of a batched decode.  All pointers except `info` are device pointers. */
+typedef struct {
+    const ep_info *info;        /* host */
+    const void *d_stream;       /* device: the blob, or at least its header, table and payload sections,
+                                   at their blob offsets; 4-byte aligned */
+    const void *d_tile_index;   /* device: the tile-index section (132*n_tiles + 4 bytes); 4-byte aligned */
+    const float *d_row_scales;  /* device: R fp32 row scales (the blob's, or the caller's own) */
+    int32_t out_dtype;          /* ep_dtype */
+    void *d_out;                /* device: R*C elements of out_dtype, row-major; 16-byte aligned */
+    void *d_scratch;            /* device: ep_decode_scratch_bytes(info) bytes, 256-byte aligned; may be
+                                   NULL when that size is 0 */
+    size_t scratch_bytes;
+} ep_decode_job;
+
+/* ---- host encoder ------------------------------------------------------------------------- */
+
+/* Paper defaults for every field of *opts. */
+void ep_encode_opts_default(ep_encode_opts *opts);
+
+/* Compress W (host, row-major R x C fp32, C % 8 == 0, R*C/8 < 2^32) to about target_bpp stored
+ * bits per weight: row RMS normalisation, E8 nearest-point quantisation, sampled storage estimate,
+ * geometric scale search with precision escalation (Algorithm 1), row-scale refit (Eq. 13), final
+ * tables and tiled rANS encoding (Eq. 17).  opts may be NULL.  On success *out owns the blob;
+ * release it with ep_blob_free().  W is only read. */
+int ep_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts,
+              ep_blob **out);
+
+/* Encode given fields directly (final tables + tile coding only; Sec. 3.6).  fields is host
+ * int32[R*C/8][9] = (c, z1..z7, m) per block, row_scales host f32[R].  For tools and tests. */
+int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int32_t b, uint32_t V,
+                   const float *row_scales, float s_info, int32_t threads, ep_blob **out);
+
+const void *ep_blob_data(const ep_blob *blob);   /* host pointer valid until ep_blob_free */
+size_t ep_blob_bytes(const ep_blob *blob);       /* B_stored of Eq. 1 */
+int ep_blob_report(const ep_blob *blob, ep_encode_report *out);
+void ep_blob_free(ep_blob *blob);
+
+/* Parse header and table directory of a host copy of a blob (n bytes). */
+int ep_blob_info(const void *blob, size_t n, ep_info *out);
+
+/* Full structural check of a host copy of a blob: sizes and offsets consistent and monotone,
+ * frequencies of every used table sum to 2^b, states inside [2^15, 2^31).  A blob that passes can
+ * be given to the decoder without risk of out-of-range accesses. */
+int ep_validate(const void *blob, size_t n);
+
+/* ---- device decoder ----------------------------------------------------------------------- */
+
+/* Scratch bytes the decoder needs for this tensor: 0 when the symbol lookup tables fit shared
+ * memory (b <= 11 and coordinate range <= 512), else room for 17 tables of 2^b 8-byte entries. */
+size_t ep_decode_scratch_bytes(const ep_info *info);
+
+/* Fused decode of one tensor (Sec. 3.7): rANS symbol decode (Eq. 18) -> inverse field transform
+ * (Eq. 5) -> multiply by the fp32 row scale -> snap to out_dtype (Eq. 19) -> store.  Enqueues on
+ * `stream` and returns; see ep_decode_job for the pointer arguments. */
+int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                     const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
+                     size_t scratch_bytes, void *stream);
+
+/* The same for up to EP_MAX_BATCH tensors in one kernel launch (independent tiles of all tensors
+ * share the grid).  Jobs needing scratch get their lookup tables built by one extra launch first. */
+int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
+
+/* Device-side integrity word.  The kernel ORs in a flag when a tile does not end with every state
+ * at 2^15 and its word pointer at the next tile's offset (a damaged stream).  This call
+ * synchronises `stream`, returns EP_OK or EP_ERR_BAD_STREAM / EP_ERR_CUDA, and clears the word.
+ * For tests and debugging; not needed on the hot path. */
+int ep_last_device_status(void *stream);
+
+/* ---- misc --------------------------------------------------------------------------------- */
+const char *ep_strerror(int status);
+uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile-size defaults */
+int ep_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ENTROPACK_H */

@@ -1,0 +1,11 @@
+"""B200-native EntroPack codec: host encoder + fused sm_100a rANS/E8 weight decoder.
+
+The product is the C-ABI library declared in ``include/entropack.h``; this package is a thin
+ctypes binding with the same names.  PyTorch appears only as the owner of device memory and
+streams.
+"""
+from .binding import (  # noqa: F401
+    BF16, FP16, FP8_E4M3, INT8, FIELDS_I32, DTYPE_BYTES, EncodeOpts, EncodeReport, Info, DecodeJob, Blob,
+    EntroPackError, load, encode, pack_fields, blob_info, validate, decode_scratch_bytes, decode_tensor,
+    decode_batch, last_device_status, default_tile_vectors, strerror, DeviceBlob, upload, decode, decode_many,
+)

@@ -1,0 +1,547 @@
+// Host-side EntroPack encoder (paper Sec. 3.2-3.6): row normalisation, E8 nearest-point
+// quantisation, field representation, coset-conditioned model, sampled storage estimate,
+// geometric scale search with precision escalation (Algorithm 1), row-scale refit (Eq. 13),
+// final tables and tiled 32-state rANS encoding (Eq. 17).
+//
+// Numerical conventions (they decide which lattice point and which scale are chosen, so they are
+// part of the format's encoder contract):
+//   * row RMS: squares accumulated in double in index order, one rounding to fp32;
+//   * quantiser input: two fp32 divisions, (x / mu) / s, with s rounded once to fp32;
+//   * coordinate rounding ties to even; parity fix on the first coordinate of largest |residual|,
+//     sign(0) = +1; the half coset is taken only when strictly closer (distances: fp32 residuals
+//     of the final candidates, squares summed in double in index order);
+//   * frequencies: f = max(1, floor(n 2^b / total)); deficit to the largest f (lowest index),
+//     excess taken from the current largest f;
+//   * C_CE summed over tables 0..16 and symbols in ascending order, in double.
+// This file must be compiled without floating-point contraction.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <functional>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "stream.hpp"
+
+struct ep_blob {
+    std::vector<uint8_t> bytes;
+    ep_encode_report report{};
+};
+
+namespace ep {
+namespace {
+
+constexpr double kEta = 1e-12;
+
+// ---- small thread helper: static contiguous partition of [0, n) -------------------------------
+void parallel_for(uint64_t n, int threads, const std::function<void(uint64_t, uint64_t, int)> &body) {
+    if (threads <= 1 || n < 2) { body(0, n, 0); return; }
+    const uint64_t parts = std::min<uint64_t>(uint64_t(threads), n);
+    std::vector<std::thread> pool;
+    pool.reserve(parts);
+    for (uint64_t p = 0; p < parts; ++p) {
+        const uint64_t lo = n * p / parts, hi = n * (p + 1) / parts;
+        pool.emplace_back([=, &body] { body(lo, hi, int(p)); });
+    }
+    for (auto &t : pool) t.join();
+}
+
+int resolve_threads(int requested) {
+    if (requested > 0) return requested;
+    const unsigned hw = std::thread::hardware_concurrency();
+    return hw ? int(hw) : 1;
+}
+
+// ---- Sec. 3.2 ----------------------------------------------------------------------------------
+float row_rms(const float *x, uint32_t C) {
+    double acc = 0.0;
+    for (uint32_t j = 0; j < C; ++j) { const double v = x[j]; acc += v * v; }
+    double mu = std::sqrt(acc / double(C));
+    if (!(mu > kEta)) mu = kEta;
+    return float(mu);
+}
+
+// round to nearest integer, ties to even (default rounding mode); |y| < 2^22 uses the exact
+// add-and-subtract of 1.5 * 2^23, anything larger is handed to the library routine.
+inline float round_even(float y) {
+    if (std::fabs(y) < 4194304.0f) {
+        volatile float t = y + 12582912.0f;
+        return t - 12582912.0f;
+    }
+    return std::nearbyintf(y);
+}
+
+// Eq. 3 on one 8-vector; returns the integer point and keeps the fp32 residuals of that point.
+struct D8 {
+    int32_t z[8];
+    float res[8];
+};
+inline void nearest_d8(const float *y, D8 &o) {
+    int32_t sum = 0;
+    for (int i = 0; i < 8; ++i) {
+        const float f = round_even(y[i]);
+        o.z[i] = int32_t(f);
+        o.res[i] = y[i] - f;
+        sum += o.z[i];
+    }
+    if (sum & 1) {
+        int at = 0;
+        float big = std::fabs(o.res[0]);
+        for (int i = 1; i < 8; ++i) {
+            const float a = std::fabs(o.res[i]);
+            if (a > big) { big = a; at = i; }
+        }
+        const int step = (o.res[at] >= 0.0f) ? 1 : -1;
+        o.z[at] += step;
+        o.res[at] = y[at] - float(o.z[at]);
+    }
+}
+
+// Eq. 2 + Eq. 4: quantise one block x[0..8) of a row with RMS mu at scale s; writes (c, z1..z7, m).
+inline void quantise_block(const float *x, float mu, float s, int32_t *fld) {
+    float y[8], yh[8];
+    for (int i = 0; i < 8; ++i) {
+        const float X = x[i] / mu;
+        y[i] = X / s;
+        yh[i] = y[i] - 0.5f;
+    }
+    D8 a, h;
+    nearest_d8(y, a);
+    nearest_d8(yh, h);
+    double da = 0.0, dh = 0.0;
+    for (int i = 0; i < 8; ++i) {
+        da += double(a.res[i]) * double(a.res[i]);
+        dh += double(h.res[i]) * double(h.res[i]);
+    }
+    const D8 &w = (dh < da) ? h : a;
+    fld[0] = (dh < da) ? 1 : 0;
+    int32_t s7 = 0;
+    for (int i = 0; i < 7; ++i) { fld[1 + i] = w.z[i]; s7 += w.z[i]; }
+    const int32_t pi = s7 & 1;              // two's complement: (sum mod 2) in {0, 1}
+    fld[8] = (w.z[7] - pi) >> 1;            // exact: z8 - pi is even
+}
+
+void quantise_rows(const float *W, uint32_t C, const float *mu, const uint32_t *rows, uint64_t n_rows, float s,
+                   int32_t *fields, int threads) {
+    const uint32_t per_row = C / 8;
+    parallel_for(n_rows, threads, [&](uint64_t lo, uint64_t hi, int) {
+        for (uint64_t i = lo; i < hi; ++i) {
+            const uint64_t r = rows ? rows[i] : i;
+            const float *x = W + r * C;
+            int32_t *f = fields + i * per_row * 9;
+            for (uint32_t v = 0; v < per_row; ++v) quantise_block(x + 8 * v, mu[r], s, f + 9 * v);
+        }
+    });
+}
+
+// ---- Sec. 3.3: the seventeen categorical tables -------------------------------------------------
+struct Table {
+    int32_t lo = 0;
+    std::vector<uint64_t> n;   // counts over [lo, lo + K)
+    std::vector<uint32_t> f;   // b-bit frequencies
+    std::vector<uint32_t> F;   // exclusive prefix sums, K + 1 entries
+    uint64_t total = 0;
+    uint32_t K() const { return uint32_t(n.size()); }
+    uint32_t observed() const {
+        uint32_t o = 0;
+        for (uint64_t c : n) o += c != 0;
+        return o;
+    }
+};
+
+struct Model {
+    Table t[EP_NUM_TABLES];
+
+    // counts from field tuples; threads reduce private (min, max) first, then private histograms
+    void count(const int32_t *fld, uint64_t nvec, int threads) {
+        struct Range { int64_t lo[EP_NUM_TABLES], hi[EP_NUM_TABLES]; bool any[EP_NUM_TABLES]; };
+        const int T = std::max(1, threads);
+        std::vector<Range> rg(T);
+        for (auto &r : rg) for (int i = 0; i < EP_NUM_TABLES; ++i) { r.any[i] = false; r.lo[i] = r.hi[i] = 0; }
+        parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
+            Range &r = rg[id];
+            for (uint64_t v = a; v < b; ++v) {
+                const int32_t *q = fld + 9 * v;
+                for (int k = 0; k < 9; ++k) {
+                    const int ti = table_id(q[0], k);
+                    if (!r.any[ti]) { r.any[ti] = true; r.lo[ti] = r.hi[ti] = q[k]; }
+                    else { r.lo[ti] = std::min<int64_t>(r.lo[ti], q[k]); r.hi[ti] = std::max<int64_t>(r.hi[ti], q[k]); }
+                }
+            }
+        });
+        for (int i = 0; i < EP_NUM_TABLES; ++i) {
+            bool any = false;
+            int64_t lo = 0, hi = 0;
+            for (auto &r : rg) if (r.any[i]) {
+                if (!any) { lo = r.lo[i]; hi = r.hi[i]; any = true; }
+                else { lo = std::min(lo, r.lo[i]); hi = std::max(hi, r.hi[i]); }
+            }
+            t[i] = Table();
+            if (any) { t[i].lo = int32_t(lo); t[i].n.assign(size_t(hi - lo + 1), 0); }
+        }
+        std::vector<std::vector<uint64_t>> priv(size_t(T) * EP_NUM_TABLES);
+        parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
+            std::vector<uint64_t> *h = &priv[size_t(id) * EP_NUM_TABLES];
+            for (int i = 0; i < EP_NUM_TABLES; ++i) h[i].assign(t[i].n.size(), 0);
+            for (uint64_t v = a; v < b; ++v) {
+                const int32_t *q = fld + 9 * v;
+                for (int k = 0; k < 9; ++k) {
+                    const int ti = table_id(q[0], k);
+                    h[ti][size_t(q[k] - t[ti].lo)]++;
+                }
+            }
+        });
+        for (int id = 0; id < T; ++id)
+            for (int i = 0; i < EP_NUM_TABLES; ++i) {
+                const auto &h = priv[size_t(id) * EP_NUM_TABLES + i];
+                for (size_t j = 0; j < h.size(); ++j) { t[i].n[j] += h[j]; t[i].total += h[j]; }
+            }
+    }
+
+    // integer frequencies summing to 2^b, every observed symbol >= 1
+    void normalise(int b) {
+        const uint64_t M = 1ull << b;
+        for (auto &tb : t) {
+            const uint32_t K = tb.K();
+            tb.f.assign(K, 0);
+            tb.F.assign(K + 1, 0);
+            if (!K || !tb.total) continue;
+            uint64_t sum = 0;
+            for (uint32_t j = 0; j < K; ++j) {
+                if (!tb.n[j]) continue;
+                const uint64_t q = tb.n[j] * M / tb.total;
+                tb.f[j] = uint32_t(std::max<uint64_t>(q, 1));
+                sum += tb.f[j];
+            }
+            auto largest = [&] { return uint32_t(std::max_element(tb.f.begin(), tb.f.end()) - tb.f.begin()); };
+            if (sum < M) tb.f[largest()] += uint32_t(M - sum);
+            while (sum > M) {
+                const uint32_t j = largest();
+                const uint64_t take = std::min<uint64_t>(sum - M, uint64_t(tb.f[j]) - 1);
+                tb.f[j] -= uint32_t(take);
+                sum -= take;
+            }
+            for (uint32_t j = 0; j < K; ++j) tb.F[j + 1] = tb.F[j] + tb.f[j];
+        }
+    }
+
+    // Eq. 8
+    double cross_entropy_bits(int b) const {
+        double acc = 0.0;
+        for (const auto &tb : t)
+            for (uint32_t j = 0; j < tb.K(); ++j)
+                if (tb.n[j]) acc += double(tb.n[j]) * (double(b) - std::log2(double(tb.f[j])));
+        return acc;
+    }
+
+    uint64_t section_bytes() const {
+        uint32_t K[EP_NUM_TABLES];
+        for (int i = 0; i < EP_NUM_TABLES; ++i) K[i] = t[i].K();
+        return table_section_bytes(K);
+    }
+};
+
+// Eq. 10-11: estimated stored bits of nvec vectors in `rows` rows under model m
+double estimate_bits(const Model &m, int b, uint64_t nvec, uint64_t rows, uint32_t V, double retained, double *cce_out) {
+    const double cce = m.cross_entropy_bits(b);
+    const uint64_t n_tile = (nvec + V - 1) / V;
+    const double left = std::max(0.0, cce - retained * double(kStates) * double(n_tile));
+    const double payload = 16.0 * std::ceil(left / 16.0);
+    const double restart = double(n_tile) * (32.0 * kStates + 32.0) + 32.0;
+    const double tables = 8.0 * double(m.section_bytes());
+    const double scales = 32.0 * double(rows);
+    const double other = 8.0 * kHeaderBytes;
+    if (cce_out) *cce_out = cce;
+    return payload + restart + tables + scales + other;
+}
+
+// ---- App. "Scale-search settings": the fixed row sample -----------------------------------------
+inline uint64_t splitmix64(uint64_t &state) {
+    uint64_t z = (state += 0x9E3779B97F4A7C15ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+std::vector<uint32_t> sample_rows(uint32_t R, uint32_t C, uint32_t budget_vectors) {
+    const uint32_t per_row = C / 8;
+    uint32_t n = std::max<uint32_t>(1, budget_vectors / per_row);
+    n = std::min(n, R);
+    std::vector<uint32_t> idx(R);
+    for (uint32_t i = 0; i < R; ++i) idx[i] = i;
+    uint64_t st = (uint64_t(R) << 32) + uint64_t(C);
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t j = i + uint32_t(splitmix64(st) % uint64_t(R - i));
+        std::swap(idx[i], idx[j]);
+    }
+    idx.resize(n);
+    std::sort(idx.begin(), idx.end());
+    return idx;
+}
+
+// ---- Sec. 3.6 / App. "Tiled rANS implementation": one tile -------------------------------------
+// The decoder visits (group of 32 vectors, field 0..8, lane 0..31); the encoder walks that order
+// backwards, emits a word before the update whenever xi >= f * 2^(31-b), and finally reverses the
+// tile's words.
+void encode_tile(const int32_t *fld, uint32_t nv, const Model &m, int b, uint32_t *states, std::vector<uint16_t> &words) {
+    uint32_t xi[kStates];
+    for (auto &x : xi) x = kStateLow;
+    words.clear();
+    words.reserve(size_t(nv) * 5);
+    const uint32_t groups = (nv + kStates - 1) / kStates;
+    for (uint32_t g = groups; g-- > 0;) {
+        const uint32_t lanes = std::min<uint32_t>(kStates, nv - g * kStates);
+        for (int k = 8; k >= 0; --k)
+            for (uint32_t l = lanes; l-- > 0;) {
+                const int32_t *q = fld + 9ull * (uint64_t(g) * kStates + l);
+                const Table &tb = m.t[table_id(q[0], k)];
+                const uint32_t sym = uint32_t(q[k] - tb.lo);
+                const uint32_t f = tb.f[sym], F = tb.F[sym];
+                uint32_t x = xi[l];
+                if (uint64_t(x) >= (uint64_t(f) << (31 - b))) { words.push_back(uint16_t(x)); x >>= 16; }
+                xi[l] = ((x / f) << b) + (x % f) + F;
+            }
+    }
+    std::reverse(words.begin(), words.end());
+    std::copy(xi, xi + kStates, states);
+}
+
+// final tables -> tiles -> stored representation
+int pack(const int32_t *fields, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
+         int threads, ep_blob *out, double *cce_out) {
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    Model m;
+    m.count(fields, nvec, threads);
+    for (const auto &tb : m.t) if (tb.observed() > (1u << b)) return EP_ERR_UNSUPPORTED;
+    m.normalise(b);
+    if (cce_out) *cce_out = m.cross_entropy_bits(b);
+    const uint32_t n_tiles = uint32_t((nvec + V - 1) / V);
+    std::vector<std::vector<uint16_t>> words(n_tiles);
+    std::vector<uint32_t> states(size_t(n_tiles) * kStates);
+    parallel_for(n_tiles, threads, [&](uint64_t lo, uint64_t hi, int) {
+        for (uint64_t t = lo; t < hi; ++t) {
+            const uint64_t v0 = t * V;
+            const uint32_t nv = uint32_t(std::min<uint64_t>(V, nvec - v0));
+            encode_tile(fields + 9 * v0, nv, m, b, &states[t * kStates], words[t]);
+        }
+    });
+    uint64_t total_words = 0;
+    for (const auto &w : words) total_words += w.size();
+    // coordinate range of z_1..z_8 (z_8 = 2m + parity spans [2 m_lo, 2 m_hi + 1])
+    bool any = false;
+    int64_t cmin = 0, cmax = 0;
+    for (int c = 0; c < 2; ++c)
+        for (int k = 1; k <= 8; ++k) {
+            const Table &tb = m.t[table_id(c, k)];
+            if (!tb.K()) continue;
+            int64_t lo = tb.lo, hi = int64_t(tb.lo) + tb.K() - 1;
+            if (k == 8) { lo *= 2; hi = 2 * hi + 1; }
+            if (!any) { cmin = lo; cmax = hi; any = true; }
+            else { cmin = std::min(cmin, lo); cmax = std::max(cmax, hi); }
+        }
+    cmin = std::max<int64_t>(cmin, -32768);
+    cmax = std::min<int64_t>(cmax, 32767);
+    const uint64_t tb_bytes = m.section_bytes();
+    const uint64_t off_tables = kHeaderBytes, off_scales = off_tables + tb_bytes, off_tiles = off_scales + 4ull * R;
+    const uint64_t off_payload = off_tiles + uint64_t(kTileRecordBytes) * n_tiles + 4, total = off_payload + 2 * total_words;
+    if (total >= (1ull << 32)) return EP_ERR_UNSUPPORTED;   // section offsets are 32-bit
+    std::vector<uint8_t> &B = out->bytes;
+    B.assign(size_t(total), 0);
+    uint8_t *p = B.data();
+    store_le<uint32_t>(p, kMagic);
+    store_le<uint16_t>(p + 4, 1);
+    p[6] = uint8_t(b);
+    p[7] = uint8_t(kStates);
+    store_le<uint32_t>(p + 8, R);
+    store_le<uint32_t>(p + 12, C);
+    store_le<uint32_t>(p + 16, V);
+    store_le<uint32_t>(p + 20, n_tiles);
+    store_le<float>(p + 24, s_info);
+    store_le<int16_t>(p + 28, int16_t(cmin));
+    store_le<int16_t>(p + 30, int16_t(cmax));
+    store_le<uint32_t>(p + 32, uint32_t(off_tables));
+    store_le<uint32_t>(p + 36, uint32_t(off_scales));
+    store_le<uint32_t>(p + 40, uint32_t(off_tiles));
+    store_le<uint32_t>(p + 44, uint32_t(off_payload));
+    store_le<uint64_t>(p + 48, total);
+    store_le<uint32_t>(p + 56, uint32_t(total_words));
+    uint8_t *dir = p + off_tables;
+    uint8_t *fq = dir + 8 * EP_NUM_TABLES;
+    for (int i = 0; i < EP_NUM_TABLES; ++i) {
+        store_le<int32_t>(dir + 4 * i, m.t[i].lo);
+        store_le<uint32_t>(dir + 4 * EP_NUM_TABLES + 4 * i, m.t[i].K());
+        for (uint32_t j = 0; j < m.t[i].K(); ++j, fq += 2) store_le<uint16_t>(fq, uint16_t(m.t[i].f[j]));
+    }
+    std::memcpy(p + off_scales, sigma, 4ull * R);
+    uint64_t at = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) {
+        uint8_t *rec = p + off_tiles + uint64_t(kTileRecordBytes) * t;
+        std::memcpy(rec, &states[size_t(t) * kStates], 4 * kStates);
+        store_le<uint32_t>(rec + 4 * kStates, uint32_t(at));
+        if (!words[t].empty()) std::memcpy(p + off_payload + 2 * at, words[t].data(), 2 * words[t].size());
+        at += words[t].size();
+    }
+    store_le<uint32_t>(p + off_tiles + uint64_t(kTileRecordBytes) * n_tiles, uint32_t(at));
+    return EP_OK;
+}
+
+// Eq. 13
+void refit(const float *W, uint32_t R, uint32_t C, const int32_t *fields, float s, const float *mu, float *sigma, int threads) {
+    const uint32_t per_row = C / 8;
+    parallel_for(R, threads, [&](uint64_t lo, uint64_t hi, int) {
+        for (uint64_t r = lo; r < hi; ++r) {
+            double xp = 0.0, pp = 0.0;
+            const float *x = W + r * C;
+            for (uint32_t v = 0; v < per_row; ++v) {
+                const int32_t *q = fields + 9 * (r * per_row + v);
+                const double half = 0.5 * double(q[0]);
+                int32_t s7 = 0;
+                for (int j = 0; j < 7; ++j) {
+                    const double p = double(q[1 + j]) + half;
+                    xp += double(x[8 * v + j]) * p;
+                    pp += p * p;
+                    s7 += q[1 + j];
+                }
+                const double p8 = double(2 * q[8] + (s7 & 1)) + half;   // Eq. 5
+                xp += double(x[8 * v + 7]) * p8;
+                pp += p8 * p8;
+            }
+            double sg;
+            if (pp > 0.0) { sg = xp / pp; if (!(sg > kEta)) sg = kEta; }
+            else sg = double(s) * double(mu[r]);
+            sigma[r] = float(sg);
+        }
+    });
+}
+
+}  // namespace
+}  // namespace ep
+
+// ---- C ABI -----------------------------------------------------------------------------------------
+
+extern "C" void ep_encode_opts_default(ep_encode_opts *o) {
+    if (!o) return;
+    o->bracket_lo = 1e-3;
+    o->bracket_hi = 8.0;
+    o->search_steps = 12;
+    o->sample_vectors = 1u << 18;
+    o->tile_vectors = 0;
+    o->b_start = 0;
+    o->b_max = 15;
+    o->retained_bits = 16.0;
+    o->threads = 0;
+}
+
+extern "C" int ep_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts_in,
+                         ep_blob **out) {
+    using namespace ep;
+    if (!W || !out || R == 0 || C == 0 || C % 8 != 0 || !(target_bpp > 0.0)) return EP_ERR_BAD_ARG;
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    if (nvec >= (1ull << 32)) return EP_ERR_BAD_ARG;
+    ep_encode_opts o;
+    if (opts_in) o = *opts_in; else ep_encode_opts_default(&o);
+    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.b_max > 15 || o.b_max < 9 ||
+        (o.b_start != 0 && (o.b_start < 9 || o.b_start > o.b_max)))
+        return EP_ERR_BAD_ARG;
+    try {
+        const int threads = resolve_threads(o.threads);
+        const uint32_t V = o.tile_vectors ? o.tile_vectors : ep_default_tile_vectors(target_bpp);
+        int b = o.b_start ? o.b_start : (target_bpp <= 7.0 ? 11 : 12);
+        b = std::min(b, o.b_max);
+        std::vector<float> mu(R);
+        parallel_for(R, threads, [&](uint64_t lo, uint64_t hi, int) {
+            for (uint64_t r = lo; r < hi; ++r) mu[r] = row_rms(W + r * C, C);
+        });
+        const std::vector<uint32_t> rows = sample_rows(R, C, o.sample_vectors);
+        const uint64_t svec = uint64_t(rows.size()) * (C / 8);
+        std::vector<int32_t> sfields(size_t(svec) * 9), fields(size_t(nvec) * 9);
+        float s = 0.0f;
+        double last_rate = 0.0;
+        for (;; ++b) {
+            double lo = o.bracket_lo, hi = o.bracket_hi;
+            for (int it = 0; it < o.search_steps; ++it) {
+                const double mid = std::sqrt(lo * hi);
+                quantise_rows(W, C, mu.data(), rows.data(), rows.size(), float(mid), sfields.data(), threads);
+                Model m;
+                m.count(sfields.data(), svec, threads);
+                m.normalise(b);
+                const double bits = estimate_bits(m, b, svec, rows.size(), V, o.retained_bits, nullptr);
+                last_rate = bits / (8.0 * double(svec));
+                if (last_rate > target_bpp) lo = mid; else hi = mid;
+            }
+            s = float(std::sqrt(lo * hi));
+            bool fits = false;
+            for (;;) {
+                quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
+                Model m;
+                m.count(fields.data(), nvec, threads);
+                uint32_t worst = 0, amax = 0;
+                for (int i = 0; i < EP_NUM_TABLES; ++i) {
+                    const uint32_t ob = m.t[i].observed();
+                    worst = std::max(worst, ob);
+                    if (i > 0) amax = std::max(amax, ob);
+                }
+                if (worst <= (1u << b)) { fits = true; break; }
+                if (b < o.b_max) break;
+                s = float(1.05 * double(s) * double(amax) / double(1u << b));
+            }
+            if (fits) break;
+        }
+        std::vector<float> sigma(R);
+        refit(W, R, C, fields.data(), s, mu.data(), sigma.data(), threads);
+        ep_blob *blob = new ep_blob();
+        double cce = 0.0;
+        const int rc = pack(fields.data(), R, C, b, V, sigma.data(), s, threads, blob, &cce);
+        if (rc) { delete blob; return rc; }
+        blob->report.s = double(s);
+        blob->report.b = b;
+        blob->report.bytes = blob->bytes.size();
+        blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
+        blob->report.est_bpp_sample = last_rate;
+        blob->report.cce_bits = cce;
+        blob->report.sample_rows = uint32_t(rows.size());
+        *out = blob;
+        return EP_OK;
+    } catch (const std::bad_alloc &) {
+        return EP_ERR_NOMEM;
+    } catch (...) {
+        return EP_ERR_UNSUPPORTED;
+    }
+}
+
+extern "C" int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int32_t b, uint32_t V,
+                              const float *row_scales, float s_info, int32_t threads, ep_blob **out) {
+    using namespace ep;
+    if (!fields || !row_scales || !out || R == 0 || C == 0 || C % 8 != 0 || V == 0 || b < 9 || b > 15) return EP_ERR_BAD_ARG;
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    if (nvec >= (1ull << 32)) return EP_ERR_BAD_ARG;
+    for (uint64_t v = 0; v < nvec; ++v)
+        if (fields[9 * v] != 0 && fields[9 * v] != 1) return EP_ERR_BAD_ARG;
+    try {
+        ep_blob *blob = new ep_blob();
+        double cce = 0.0;
+        const int rc = pack(fields, R, C, b, V, row_scales, s_info, resolve_threads(threads), blob, &cce);
+        if (rc) { delete blob; return rc; }
+        blob->report.s = double(s_info);
+        blob->report.b = b;
+        blob->report.bytes = blob->bytes.size();
+        blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
+        blob->report.cce_bits = cce;
+        *out = blob;
+        return EP_OK;
+    } catch (const std::bad_alloc &) {
+        return EP_ERR_NOMEM;
+    } catch (...) {
+        return EP_ERR_UNSUPPORTED;
+    }
+}
+
+extern "C" const void *ep_blob_data(const ep_blob *b) { return b ? b->bytes.data() : nullptr; }
+extern "C" size_t ep_blob_bytes(const ep_blob *b) { return b ? b->bytes.size() : 0; }
+extern "C" int ep_blob_report(const ep_blob *b, ep_encode_report *out) {
+    if (!b || !out) return EP_ERR_BAD_ARG;
+    *out = b->report;
+    return EP_OK;
+}
+extern "C" void ep_blob_free(ep_blob *b) { delete b; }

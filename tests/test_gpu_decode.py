@@ -1,0 +1,171 @@
+"""GPU parity: the fused CUDA decoder against the oracle, element by element, through the C ABI.
+Both directions (library stream -> oracle decoder is covered on CPU; here library stream and oracle
+stream -> GPU decoder), all output types, ragged shapes, and the full-size benchmark configurations."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_34185_b200 as ep
+from paper_2609_34185_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+ORACLE_DT = {ep.BF16: oracle.BF16, ep.FP16: oracle.FP16, ep.FP8_E4M3: oracle.E4M3, ep.INT8: oracle.INT8}
+
+
+def _bits(t: torch.Tensor) -> np.ndarray:
+    if t.dtype in (torch.bfloat16, torch.float16):
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    if t.dtype == torch.float8_e4m3fn:
+        return t.view(torch.uint8).cpu().numpy()
+    return t.cpu().numpy()
+
+
+def _check_all_types(blob_bytes, scales=None):
+    d = ep.upload(blob_bytes)
+    sc_dev = None if scales is None else torch.from_numpy(scales).cuda()
+    ref_fields = None
+    for dt, odt in ORACLE_DT.items():
+        got = ep.decode(d, dt, row_scales=sc_dev)
+        ref, ref_fields = oracle.decode(blob_bytes, odt, scales=scales, want_fields=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(_bits(got), ref), f"dtype {dt}"
+    f = ep.decode(d, ep.FIELDS_I32)
+    assert np.array_equal(f.cpu().numpy(), ref_fields)
+    assert ep.last_device_status() == 0
+
+
+def test_config1_all_types_both_directions():
+    W = synth.config1()
+    lib_blob = ep.encode(W, 4.0, tile_vectors=4096)          # one tile per 64 rows
+    assert lib_blob.info.n_tiles == 8
+    _check_all_types(lib_blob.data)
+    ora_blob, rep = oracle.encode(W, 4.0, oracle.default_opts(tile_vectors=4096))
+    _check_all_types(ora_blob)
+    assert abs(rep["stored_bpp"] - 4.0) < 0.04
+    # weight error against the original matches the oracle's (same points, same scales)
+    got = ep.decode(ep.upload(lib_blob), ep.BF16).float().cpu().numpy()
+    ref, _ = oracle.decode(ora_blob, oracle.BF16)
+    ref = torch.from_numpy(ref.view(np.int16)).view(torch.bfloat16).float().numpy()
+    e_gpu, e_ref = oracle.rel_l2(W, got), oracle.rel_l2(W, ref)
+    assert abs(e_gpu - e_ref) <= 1e-6 * e_ref
+
+
+@pytest.mark.parametrize("R,C,V,bpp", [
+    (8, 8, 0, 4.0),          # a single vector per row, one tiny tile
+    (3, 40, 32, 3.0),        # 5 vectors per row: groups straddle rows
+    (33, 264, 100, 3.0),     # V not a multiple of 32, ragged last tile
+    (64, 2048, 455, 6.0),    # the paper's 8 bpp tile size
+    (96, 1024, 1820, 2.0),   # default 4 bpp tile size, low rate
+    (5, 4096, 3640, 5.0),
+    (256, 256, 33, 4.5),     # many tiny tiles
+])
+def test_ragged_shapes_all_types(R, C, V, bpp):
+    W = synth.laplace_rows(R, C, 1000 + R + C)
+    blob = ep.encode(W, bpp, tile_vectors=V)
+    _check_all_types(blob.data)
+
+
+def test_row_scale_edge_cases():
+    W = synth.gaussian_rows(16, 512, 31)
+    blob = ep.encode(W, 4.0, tile_vectors=100)
+    sc = np.array([0.0, -0.0, 1.0, -1.0, 1e30, -1e30, 3e38, 1e-30, 1e-38, 1e-42, 65504.0 / 8, 448.0 / 4, 127.0, 0.5,
+                   2.0 ** -20, 7.0], np.float32)
+    _check_all_types(blob.data, scales=sc)
+
+
+def test_single_symbol_tables_and_low_precision():
+    # every coordinate zero in coset 1, wide alphabets in coset 0, b = 9
+    rng = np.random.default_rng(5)
+    n = 4 * 80
+    fields = np.zeros((n, 9), np.int32)
+    fields[:, 0] = rng.integers(0, 2, n)
+    z = np.rint(rng.standard_normal((n, 8)) * 3).astype(np.int32)
+    fields[:, 1:] = np.where(fields[:, :1] == 0, z, 0)
+    blob = ep.pack_fields(fields, 4, 640, 9, 64, np.linspace(0.5, 2, 4).astype(np.float32))
+    _check_all_types(blob.data)
+    # only one coset ever used
+    fields[:, 0] = 0
+    fields[:, 1:] = z
+    blob = ep.pack_fields(fields, 4, 640, 10, 50, np.ones(4, np.float32))
+    _check_all_types(blob.data)
+
+
+def test_batch_decode_matches_single():
+    blobs = [ep.encode(synth.gaussian_rows(64 + 32 * i, 512 + 256 * i, 50 + i), 2.5 + 0.5 * i, tile_vectors=200 + 37 * i)
+             for i in range(5)]
+    devs = [ep.upload(b) for b in blobs]
+    outs = [torch.empty((b.info.R, b.info.C), dtype=torch.bfloat16, device="cuda") for b in blobs]
+    ep.decode_many(devs, ep.BF16, outs)
+    torch.cuda.synchronize()
+    for b, o in zip(blobs, outs):
+        ref, _ = oracle.decode(b.data, oracle.BF16)
+        assert np.array_equal(_bits(o), ref)
+    assert ep.last_device_status() == 0
+
+
+def test_damaged_payload_is_flagged_not_fatal():
+    W = synth.gaussian_rows(64, 1024, 9)
+    blob = ep.encode(W, 4.0, tile_vectors=128)
+    bad = blob.data.copy()
+    I = blob.info
+    bad[I.off_payload + 2 * (I.total_words // 2)] ^= 0x10       # structure still valid
+    bad[I.off_payload + 2 * I.total_words - 1] ^= 0x01          # and the very last word
+    assert ep.validate(bad) == 0
+    out = ep.decode(ep.upload(bad), ep.BF16)
+    assert ep.last_device_status() == -2
+    assert ep.last_device_status() == 0                          # the word is cleared after reading
+    # the context is still usable and a good stream decodes cleanly afterwards
+    good = ep.decode(ep.upload(blob), ep.BF16)
+    ref, _ = oracle.decode(blob.data, oracle.BF16)
+    assert np.array_equal(_bits(good), ref) and ep.last_device_status() == 0
+
+
+def test_decode_argument_checks():
+    blob = ep.encode(synth.gaussian_rows(16, 64, 1), 4.0)
+    d = ep.upload(blob)
+    out = torch.empty((16, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ep.EntroPackError):
+        ep.decode_tensor(d.info, d.d_stream, d.d_tile_index, d.d_row_scales, ep.BF16, out.data_ptr() + 2)
+    with pytest.raises(ep.EntroPackError):
+        ep.decode_tensor(d.info, d.d_stream, d.d_tile_index, d.d_row_scales, 7, out.data_ptr())
+    with pytest.raises(ep.EntroPackError):
+        ep.decode_tensor(d.info, 0, d.d_tile_index, d.d_row_scales, ep.BF16, out.data_ptr())
+
+
+# ---- full-size configurations, in the launch configuration the bench times -----------------------
+
+def _full_compare(W, bpp, dt, V=0):
+    blob = ep.encode(W, bpp, tile_vectors=V)
+    assert abs(blob.stored_bpp - bpp) < 0.01 * bpp, blob.stored_bpp
+    d = ep.upload(blob)
+    got = ep.decode(d, dt)
+    ref, _ = oracle.decode(blob.data, ORACLE_DT[dt])
+    torch.cuda.synchronize()
+    assert np.array_equal(_bits(got), ref)
+    assert ep.last_device_status() == 0
+    return blob
+
+
+def test_config2_full_size():
+    _full_compare(synth.config2(), 3.0, ep.BF16)
+
+
+def test_config4_full_size_two_rates():
+    W = synth.config4()
+    _full_compare(W, 4.0, ep.FP16)
+    _full_compare(W, 2.0, ep.FP16)
+
+
+def test_config3_one_wide_tensor_fp8_and_int8_containers():
+    # MLP-shaped tensor of the block bundle, pre-scaled to the FP8 / INT8 container as in the paper's
+    # low-precision route; decoded values must equal the oracle's in that container
+    W = synth.config3_tensor(4, shape=(2048, 17408))
+    for kind, dt, tdt in (("fp8", ep.FP8_E4M3, torch.float8_e4m3fn), ("int8", ep.INT8, None)):
+        a, Wc = synth.to_container(W, kind)
+        if tdt is not None:
+            Wc = torch.from_numpy(Wc).to(tdt).float().numpy()
+        else:
+            Wc = np.clip(np.rint(Wc), -128, 127).astype(np.float32)
+        _full_compare(Wc, 2.5, dt)

@@ -1,0 +1,110 @@
+"""CPU-side checks of the library: exported C ABI, host encoder against the oracle (byte-identical
+streams on the same inputs), library stream -> oracle decoder, structural validation."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2609_34185_b200 as ep
+from paper_2609_34185_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "entropack.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(ep_[a-z0-9_]+)\s*\(", hdr))
+    assert {"ep_encode", "ep_decode_tensor", "ep_decode_batch", "ep_blob_info", "ep_validate"} <= names
+    lib = ep.load()
+    for n in sorted(names):
+        assert hasattr(lib, n), n
+    assert lib.ep_version() == 1
+
+
+@pytest.mark.parametrize("shape,bpp,V", [((512, 512), 4.0, 4096), ((96, 1024), 2.0, 0), ((64, 2048), 6.0, 455),
+                                         ((33, 264), 3.0, 100), ((8, 8), 4.0, 0)])
+def test_host_encoder_matches_oracle_byte_for_byte(shape, bpp, V):
+    W = synth.gaussian_rows(shape[0], shape[1], 100 + shape[0])
+    lib_blob = ep.encode(W, bpp, tile_vectors=V)
+    ora_blob, rep = oracle.encode(W, bpp, oracle.default_opts(tile_vectors=V))
+    assert np.array_equal(lib_blob.data, ora_blob)
+    assert lib_blob.report["s"] == rep["s"] and lib_blob.report["b"] == rep["b"]
+    assert ep.validate(lib_blob.data) == 0
+
+
+def test_other_distributions_and_threads():
+    for W, bpp in ((synth.student_t_rows(256, 1024, 3), 3.0), (synth.laplace_rows(128, 2048, 4), 5.0),
+                   (synth.gaussian_rows(128, 1024, 5, outlier_p=0.001), 2.5)):
+        a = ep.encode(W, bpp, threads=1)
+        b = ep.encode(W, bpp, threads=5)
+        o, _ = oracle.encode(W, bpp)
+        assert np.array_equal(a.data, b.data) and np.array_equal(a.data, o)
+        assert abs(a.stored_bpp - bpp) < 0.02 * bpp
+
+
+def test_library_stream_decodes_with_the_oracle():
+    W = synth.laplace_rows(64, 1024, 8)
+    blob = ep.encode(W, 4.0, tile_vectors=77)
+    out, fields = oracle.decode(blob.data, oracle.FP32, want_fields=True)
+    qf, _ = oracle.quantise(W, blob.report["s"])
+    assert np.array_equal(fields, qf)
+    e = oracle.rel_l2(W, out)
+    assert 0.03 < e < 0.2
+    # pack_fields of the same fields and scales reproduces the stream
+    I = blob.info
+    sig = blob.data[I.off_scales:I.off_scales + 4 * I.R].view(np.float32)
+    again = ep.pack_fields(fields, I.R, I.C, I.b, I.V, sig, s_info=I.s)
+    assert np.array_equal(again.data, blob.data)
+
+
+def test_zero_matrix_and_constant_rows():
+    W = np.zeros((16, 64), np.float32)
+    blob = ep.encode(W, 4.0)
+    o, _ = oracle.encode(W, 4.0)
+    assert np.array_equal(blob.data, o)
+    out, _ = oracle.decode(blob.data, oracle.BF16)
+    assert not out.any()
+    W = np.tile(np.arange(1, 65, dtype=np.float32), (4, 1))
+    blob = ep.encode(W, 6.0)
+    assert np.array_equal(blob.data, oracle.encode(W, 6.0)[0])
+
+
+def test_bad_arguments():
+    lib = ep.load()
+    h = ctypes.c_void_p()
+    W = np.zeros((4, 12), np.float32)
+    assert lib.ep_encode(W.ctypes.data, 4, 12, 4.0, None, ctypes.byref(h)) == -1      # C % 8 != 0
+    assert lib.ep_encode(None, 4, 16, 4.0, None, ctypes.byref(h)) == -1
+    assert lib.ep_encode(W.ctypes.data, 4, 8, -1.0, None, ctypes.byref(h)) == -1
+    assert ep.strerror(-2).startswith("malformed")
+
+
+def test_validate_rejects_damaged_structure():
+    W = synth.gaussian_rows(32, 512, 6)
+    blob = ep.encode(W, 4.0, tile_vectors=64)
+    good = blob.data
+    I = blob.info
+    assert ep.validate(good) == 0
+
+    def broken(mut):
+        b = good.copy()
+        mut(b)
+        return ep.validate(b)
+
+    assert broken(lambda b: b.__setitem__(0, 0)) == -2                                  # magic
+    assert broken(lambda b: b.__setitem__(6, 16)) == -2                                 # b out of range
+    assert ep.validate(good[:-2]) == -2                                                 # truncated
+    assert broken(lambda b: b.__setitem__(I.off_tables + 8 * 17, b[I.off_tables + 8 * 17] ^ 1)) == -2  # freq sum
+    assert broken(lambda b: b[I.off_tiles:I.off_tiles + 4].fill(0)) == -2               # state below 2^15
+    assert broken(lambda b: b[I.off_tiles + 128:I.off_tiles + 132].fill(0xFF)) == -2    # offset beyond payload
+    def swap_offsets(b):
+        o1 = I.off_tiles + 132 + 128
+        o2 = I.off_tiles + 2 * 132 + 128
+        t = b[o1:o1 + 4].copy(); b[o1:o1 + 4] = b[o2:o2 + 4]; b[o2:o2 + 4] = t
+    assert broken(swap_offsets) == -2                                                   # offsets not monotone
+    with pytest.raises(ep.EntroPackError):
+        ep.blob_info(good[:40])
