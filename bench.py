@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Decode-throughput benchmark of the fused EntroPack decoder on B200.
+
+One "step" is one pass of the whole hot path (rANS decode -> E8 point -> row rescale -> dtype
+store) over one workload.  Default workload: the 8192x8192 Laplace tensor at 4.0 bpp decoded to
+FP16 (config 4 of the baseline).  Other workloads: --workload c2 | c3 | c4 | c5.
+
+  python bench.py [--gpus N --steps K --warmup W] [--workload c4 --bpp 4.0 --tile-vectors V]
+  python bench.py --impl reference       # the CPU oracle on the same workload (bounded sample per step)
+
+Prints ONE JSON line (rank 0).  Timing: CUDA events on the launching stream around each step, an
+L2 flush (512 MB write) between steps outside the events, max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+
+# dram bytes (read + write) per launch measured with ncu for the default workload, filled in from
+# profiles/ after a capture; None = not captured for this workload
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--bpp", type=float, default=None, help="target bits/param (default: the workload's)")
+    ap.add_argument("--tile-vectors", type=int, default=0, help="V; 0 = the paper's default for the target rate")
+    ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp8", "int8"])
+    ap.add_argument("--layers", type=int, default=48, help="c5: resident layers")
+    ap.add_argument("--distinct-layers", type=int, default=2, help="c5: distinct layers actually encoded")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+# ---- workloads ---------------------------------------------------------------------------------------
+
+def make_workload(args):
+    """Returns (name, dtype_name, target_bpp, list of layers; a layer is a list of fp32 matrices)."""
+    from paper_2609_34185_b200 import synth
+    w = args.workload
+    if w == "c4":
+        return "config4: 8192x8192 Laplace rows", args.dtype or "fp16", args.bpp or 4.0, [[synth.config4()]]
+    if w == "c2":
+        return "config2: 4096x4096 Student-t rows", args.dtype or "bf16", args.bpp or 3.0, [[synth.config2()]]
+    if w == "c3":
+        kind = args.dtype or "fp8"
+        mats = []
+        for i in range(7):
+            W = synth.config3_tensor(i)
+            if kind in ("fp8", "int8"):
+                import torch
+                a, Wc = synth.to_container(W, kind)
+                if kind == "fp8":
+                    Wc = torch.from_numpy(Wc).to(torch.float8_e4m3fn).float().numpy()
+                else:
+                    Wc = np.clip(np.rint(Wc), -128, 127).astype(np.float32)
+                W = Wc
+            mats.append(W)
+        return "config3: block bundle 4x5120^2 + 3x5120x17408, 0.1% outliers", kind, args.bpp or 2.5, [mats]
+    if w == "c5":
+        layers = [[synth.config5_tensor(l, i) for i in range(7)] for l in range(args.distinct_layers)]
+        return (f"config5: {args.layers}-layer stack of block bundles ({args.distinct_layers} distinct layers "
+                f"encoded, cycled)"), args.dtype or "bf16", args.bpp or 3.5, layers
+    raise ValueError(w)
+
+
+def encode_layers(layers, bpp, V):
+    import paper_2609_34185_b200 as ep
+    return [[ep.encode(W, bpp, tile_vectors=V) for W in mats] for mats in layers]
+
+
+# ---- clocks ------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            p = [t.strip() for t in ln.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---- CPU oracle legs -----------------------------------------------------------------------------------
+
+ORACLE_DT = {"bf16": 0, "fp16": 1, "fp8": 2, "int8": 3}
+
+
+def oracle_sample(blob, dtype_name, target_seconds=1.5):
+    """Times the oracle decoder, as it stands, on a leading tile range of one stream sized to take
+    about target_seconds; returns (params decoded, seconds, tiles, threads)."""
+    import oracle
+    I = blob.info
+    n_tiles = I.n_tiles
+    probe = max(1, min(n_tiles, 64))
+    t0 = time.perf_counter()
+    oracle.decode(blob.data, ORACLE_DT[dtype_name], tiles=(0, probe))
+    dt = max(time.perf_counter() - t0, 1e-4)
+    tiles = int(max(probe, min(n_tiles, probe * target_seconds / dt)))
+    t0 = time.perf_counter()
+    oracle.decode(blob.data, ORACLE_DT[dtype_name], tiles=(0, tiles))
+    dt = time.perf_counter() - t0
+    nvec = min(tiles * I.V, I.R * I.C // 8)
+    return 8 * nvec, dt, tiles, oracle.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle's decoder on this workload's first stream, a bounded tile
+    range per step.  Rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    name, dtype_name, bpp, layers = make_workload(args)
+    V = args.tile_vectors
+    import paper_2609_34185_b200 as ep
+    blob = ep.encode(layers[0][0], bpp, tile_vectors=V)
+    I = blob.info
+    params, dt, tiles, threads = oracle_sample(blob, dtype_name, 0.5)
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oracle.decode(blob.data, ORACLE_DT[dtype_name], tiles=(0, tiles))
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    total = sum(times)
+    value = params * len(times) / total / 1e9
+    sample = f"oracle decoder, tiles 0..{tiles} of {I.n_tiles} of the first tensor ({params} params) per step"
+    line = {"impl": "reference", "metric": "decoded Gparams/s", "value": value, "unit": "Gparams/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
+            "config": {"workload": name, "target_bpp": bpp, "stored_bpp": blob.stored_bpp, "tile_vectors": I.V},
+            "cpu_baseline": {"value": value, "unit": "Gparams/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "Gparams/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- the GPU arm ---------------------------------------------------------------------------------------
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2609_34185_b200 as ep
+
+    ep.load()   # fails loudly if the CUDA library is missing: there is no fallback
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    name, dtype_name, bpp, layers = make_workload(args)
+    DT = {"bf16": ep.BF16, "fp16": ep.FP16, "fp8": ep.FP8_E4M3, "int8": ep.INT8}[dtype_name]
+    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp8": torch.float8_e4m3fn, "int8": torch.int8}[dtype_name]
+    esize = ep.DTYPE_BYTES[DT]
+
+    # every rank decodes its own replica of the workload: tiles and tensors are independent, no collective
+    blobs = encode_layers(layers, bpp, args.tile_vectors)
+    n_layers = args.layers if args.workload == "c5" else len(blobs)
+    resident = [[ep.upload(b, device=dev) for b in blobs[l % len(blobs)]] for l in range(n_layers)]
+    layer_params = [sum(b.info.R * b.info.C for b in blobs[l % len(blobs)]) for l in range(n_layers)]
+    layer_bytes_in = [sum(len(b) for b in blobs[l % len(blobs)]) for l in range(n_layers)]
+    params_per_step = sum(layer_params)
+    comp_bytes_per_step = sum(layer_bytes_in)
+    out_bytes_layer = max(layer_params) * esize
+    out_buf = torch.empty(max(layer_params), dtype=tdt, device=dev)     # one reused layer buffer
+
+    def layer_outs(l):
+        outs, at = [], 0
+        for d in resident[l]:
+            n = d.info.R * d.info.C
+            outs.append(out_buf[at:at + n].view(d.info.R, d.info.C))
+            at += n
+        return outs
+
+    outs_by_layer = [layer_outs(l) for l in range(n_layers)]
+    launches_per_step = sum((len(r) + ep.binding.MAX_BATCH - 1) // ep.binding.MAX_BATCH for r in resident)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for l in range(n_layers):
+            if len(resident[l]) == 1:
+                ep.decode(resident[l][0], DT, out=outs_by_layer[l][0], stream=stream)
+            else:
+                ep.decode_many(resident[l], DT, outs_by_layer[l], stream=stream)
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    barrier()
+    if ep.last_device_status() != 0:
+        raise RuntimeError("decoder reported an inconsistent stream during warm-up")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    evs = []
+    for _ in range(args.steps):
+        flush.fill_(0)      # L2 flush between timed iterations, outside the events
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record(stream)
+        step()
+        e.record(stream)
+        evs.append((s, e))
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    times_ms = [s.elapsed_time(e) for s, e in evs]
+    total_ms = sum(times_ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * params_per_step / (ms_per_step * 1e-3) / 1e9           # Gparams/s, whole job
+    alg_bytes_step = comp_bytes_per_step + params_per_step * esize
+    eff_gbs = alg_bytes_step / (ms_per_step * 1e-3) / 1e9                  # per GPU
+
+    # end to end through the public call with host buffers: pinned blob -> device, decode, result -> pinned host
+    e2e = None
+    if not args.no_e2e:
+        l0 = 0
+        pinned_in = [torch.from_numpy(b.data).pin_memory() for b in blobs[l0]]
+        dev_in = [torch.empty(len(b), dtype=torch.uint8, device=dev) for b in blobs[l0]]
+        pinned_out = torch.empty(layer_params[l0], dtype=tdt).pin_memory()
+        h2d = sum(len(b) for b in blobs[l0])
+        d2h = layer_params[l0] * esize
+        e2e_steps = max(3, min(args.steps, 10))
+
+        def e2e_step():
+            ds = []
+            for p, d, b in zip(pinned_in, dev_in, blobs[l0]):
+                d.copy_(p, non_blocking=True)
+                ds.append(ep.DeviceBlob(d, b.info))
+            if len(ds) == 1:
+                ep.decode(ds[0], DT, out=outs_by_layer[l0][0], stream=stream)
+            else:
+                ep.decode_many(ds, DT, outs_by_layer[l0], stream=stream)
+            pinned_out.copy_(out_buf[:layer_params[l0]], non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e.record(stream)
+        barrier()
+        ms = s.elapsed_time(e) / e2e_steps
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * layer_params[l0] / (ms * 1e-3) / 1e9, "unit": "Gparams/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms,
+               "what": "one layer: pinned host blob -> device, decode, decoded tensor -> pinned host"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    # dominant (only) kernel: the fused decode; algorithmic bytes per launch = compressed bytes + weight bytes
+    launch_bytes = alg_bytes_step / launches_per_step
+    launch_ms = ms_per_step / launches_per_step
+    achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, bpp, dtype_name)), "peak_source": peak_src,
+                "kernel": "ep_decode_smem_kernel", "bytes_per_launch": launch_bytes, "ms_per_launch": launch_ms}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        b0 = blobs[0][0]
+        p, dt, tiles, threads = oracle_sample(b0, dtype_name, 2.0)
+        cpu = {"value": p / dt / 1e9, "unit": "Gparams/s", "cores": threads, "kind": "oracle",
+               "sample": f"oracle decoder on tiles 0..{tiles} of {b0.info.n_tiles} of the first tensor ({p} params, {dt:.2f} s)"}
+
+    b0 = blobs[0][0]
+    stored = 8.0 * comp_bytes_per_step / params_per_step
+    line = {"metric": "decoded Gparams/s", "value": value, "unit": "Gparams/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
+            "config": {"workload": name, "target_bpp": bpp, "stored_bpp": stored, "tile_vectors": b0.info.V,
+                       "tiles_first_tensor": b0.info.n_tiles, "b": b0.info.b, "out_dtype": dtype_name,
+                       "params_per_step": params_per_step, "l2": "flushed between timed steps (512 MB write)",
+                       "min_ms": min(times_ms), "median_ms": statistics.median(times_ms)},
+            "effective_GBps": eff_gbs, "pct_of_measured_hbm": 100.0 * eff_gbs / peak, "pct_of_8TBps": 100.0 * eff_gbs / 8000.0,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -17,7 +17,8 @@ NUM_TABLES = 17
 MAX_BATCH = 16
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libentropack_b200.so")
+# ENTROPACK_LIB selects another build of the same library (e.g. one compiled with different flags)
+_LIB_PATH = os.environ.get("ENTROPACK_LIB") or os.path.join(_HERE, "libentropack_b200.so")
 
 
 class EntroPackError(RuntimeError):

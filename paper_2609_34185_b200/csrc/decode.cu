@@ -12,6 +12,11 @@
 // (entry & 0xFF800) | 0x45800000 is the fp32 number 4096 + code, so one subtraction of
 // 4096 - zlo - c/2 yields the lattice coordinate p exactly, and one fp32 multiply by the row scale
 // gives the product of Eq. 19 with the same operands and rounding as the definition.
+//
+// Payload words reach the lanes through a per-warp ring in shared memory, filled 512 bytes at a
+// time by cp.async (16 bytes per lane, source clamped to the end of the payload) a few chunks ahead
+// of the read cursor; the first 640 bytes of the ring are mirrored behind its end so that the nine
+// steps of a group never have to wrap an address.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -21,12 +26,19 @@
 
 namespace {
 
-constexpr int kThreads = 1024;
+#ifndef EP_THREADS
+#define EP_THREADS 1024
+#endif
+constexpr int kThreads = EP_THREADS;
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kLutEntries = 2048;                 // 2^11 slots per table
 constexpr uint32_t kLutStride = kLutEntries * 4;       // bytes per table in shared memory
 constexpr uint32_t kCosetTableOff = 16 * kLutStride;   // coset table sits after the 16 coordinate tables
 constexpr uint32_t kLutBytes = 17 * kLutStride;        // 139264
+constexpr uint32_t kRingBytes = 2048;                  // four 512-byte chunks per warp
+constexpr uint32_t kRingMirror = 640;                  // >= 9 steps * 32 words * 2 bytes + one lane span
+constexpr uint32_t kRingStride = kRingBytes + kRingMirror;
+constexpr uint32_t kSmemBytes = kLutBytes + kWarps * kRingStride;   // 225280
 constexpr uint32_t kCodeMask = 0x000FF800u;
 constexpr uint32_t kExp4096 = 0x45800000u;             // fp32 bit pattern of 4096.0
 
@@ -45,6 +57,9 @@ struct JobParams {
     uint32_t V, n_tiles, b;
     int32_t zlo;                  // even, <= -2
     uint32_t cta_begin, cta_count;
+    uint32_t n_full;              // tiles holding exactly V vectors (all but a ragged last one)
+    uint32_t iters;               // ceil(n_full / (cta_count * warps)): every warp runs this many rounds
+    uint32_t last_cta;            // CTA (relative to cta_begin) whose warp 0 decodes a ragged last tile
     int16_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint16_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
@@ -64,21 +79,31 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ uint32_t ldg_u16(const uint16_t *p) {
-    uint16_t v;
-    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
-    return v;
+__device__ __forceinline__ void cp_async16(uint32_t dst, uint64_t src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// two fp32 lanes per instruction (sm_100 packed fp32)
-__device__ __forceinline__ void sub2(float &a0, float &a1, float k) {
-    asm("{ .reg .b64 ta, tb; mov.b64 ta, {%0, %1}; mov.b64 tb, {%2, %2}; sub.rn.f32x2 ta, ta, tb; mov.b64 {%0, %1}, ta; }"
-        : "+f"(a0), "+f"(a1) : "f"(k));
+// two fp32 lanes per instruction (sm_100 packed fp32), operands kept as 64-bit register pairs
+__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
 }
-__device__ __forceinline__ void mul2(float &a0, float &a1, float k) {
-    asm("{ .reg .b64 ta, tb; mov.b64 ta, {%0, %1}; mov.b64 tb, {%2, %2}; mul.rn.f32x2 ta, ta, tb; mov.b64 {%0, %1}, ta; }"
-        : "+f"(a0), "+f"(a1) : "f"(k));
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack64(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 
 // snap_tau of Eq. 19 for two neighbouring weights (lo = lower address)
@@ -108,10 +133,9 @@ __device__ __forceinline__ uint32_t cvt_s8(float v) {
 // first slot, every lane writes the first four slots of its own symbol, and symbols with more than
 // four slots are then filled by the whole warp.
 __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t lut_addr, uint32_t warp, uint32_t lane) {
-    if (warp >= EP_NUM_TABLES) return;
-    const uint32_t t = warp;
+  for (uint32_t t = warp; t < EP_NUM_TABLES; t += kWarps) {
     const uint32_t K = J.tK[t];
-    if (K == 0) return;
+    if (K == 0) continue;
     const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_freq) + J.foff[t];
     const int32_t tmin = J.tmin[t];
     const uint32_t base = lut_addr + (t == 0 ? kCosetTableOff : (t - 1) * kLutStride);
@@ -144,29 +168,65 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
         }
         run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
+  }
 }
 
 // ---- one rANS symbol (Eq. 18) followed by renormalisation --------------------------------------
-// x: this lane's state; ptr: the tile's word cursor (warp-uniform, absolute word index in the payload).
-// Lanes that need a word take them in lane order: lane l reads word ptr + popc(ballot & lanes below l).
-template <bool TAIL, bool CAREFUL>
-__device__ __forceinline__ uint32_t rans_step(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &ptr,
-                                              const uint16_t *pay, uint32_t lt, bool act, uint32_t last_word) {
+// x: this lane's state; wa: shared-memory byte address of the tile's word cursor (same in all lanes).
+// Lanes that need a word take them in lane order: lane l reads the word popc(ballot & lanes below l)
+// places after the cursor (every lane reads, only the needy merge); the cursor then advances by
+// popc(ballot) words.  Returns the table entry.
+template <uint32_t TABLE_OFF>
+__device__ __forceinline__ uint32_t rans_step(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &wa,
+                                              uint32_t lt) {
+    uint32_t e;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b32 u, f, q, bias, bal, t, w;\n\t"
+        "and.b32 u, %1, %3;\n\t"
+        "shl.b32 u, u, 2;\n\t"
+        "add.u32 u, u, %5;\n\t"
+        "ld.shared.u32 %0, [u + %7];\n\t"
+        "shr.u32 f, %0, 20;\n\t"
+        "and.b32 bias, %0, 0x7FF;\n\t"
+        "shr.u32 q, %1, %4;\n\t"
+        "mad.lo.u32 %1, f, q, bias;\n\t"
+        "setp.lt.u32 p, %1, 32768;\n\t"
+        "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"
+        "and.b32 t, bal, %6;\n\t"
+        "popc.b32 t, t;\n\t"
+        "shl.b32 t, t, 1;\n\t"
+        "add.u32 t, t, %2;\n\t"
+        "ld.shared.u16 w, [t];\n\t"
+        "@p mad.lo.u32 %1, %1, 65536, w;\n\t"
+        "popc.b32 t, bal;\n\t"
+        "shl.b32 t, t, 1;\n\t"
+        "add.u32 %2, %2, t;\n\t"
+        "}"
+        : "=&r"(e), "+r"(x), "+r"(wa)
+        : "r"(mask), "r"(b), "r"(table_addr), "r"(lt), "n"(TABLE_OFF)
+        : "memory");
+    return e;
+}
+
+// the same for the last, partly filled group of a tile: lanes without a vector leave their state alone
+__device__ __forceinline__ uint32_t rans_step_tail(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &wa,
+                                                   uint32_t lt, bool act) {
     uint32_t e = 0;
     bool need = false;
-    if (!TAIL || act) {
-        const uint32_t u = x & mask;
-        e = lds32(table_addr + (u << 2));
+    if (act) {
+        e = lds32(table_addr + ((x & mask) << 2));
         x = (e >> 20) * (x >> b) + (e & 0x7FFu);
         need = x < ep::kStateLow;
     }
     const uint32_t bal = __ballot_sync(0xFFFFFFFFu, need);
     if (need) {
-        uint32_t idx = ptr + __popc(bal & lt);
-        if (CAREFUL) idx = min(idx, last_word);
-        x = (x << 16) | ldg_u16(pay + idx);
+        uint16_t w;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(w) : "r"(wa + 2u * __popc(bal & lt)));
+        x = (x << 16) | w;
     }
-    ptr += __popc(bal);
+    wa += 2u * __popc(bal);
     return e;
 }
 
@@ -209,18 +269,33 @@ struct Out<EP_INT8> {
     }
 };
 
+template <int DT>
+struct BlockBytes { static constexpr uint32_t value = Out<DT>::kBlockBytes; };
+template <>
+struct BlockBytes<EP_FIELDS_I32> { static constexpr uint32_t value = 36; };
+
 // ---- one group of 32 vectors: nine symbols per lane, then Eq. 5 / Eq. 19 and the store ------------
-template <int DT, bool TAIL, bool CAREFUL>
-__device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &ptr, const uint16_t *pay, uint32_t lut_addr, uint32_t mask,
-                                             uint32_t b, uint32_t lt, bool act, uint32_t last_word, float k0, float sigma,
-                                             int32_t zlo, void *dst) {
+template <int DT, bool TAIL>
+__device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &wa, uint32_t lut_addr, uint32_t mask, uint32_t b, uint32_t lt,
+                                             bool act, uint32_t k0_bits, float sigma, int32_t zlo, void *dst) {
     uint32_t e[9];
-    e[0] = rans_step<TAIL, CAREFUL>(x, lut_addr + kCosetTableOff, mask, b, ptr, pay, lt, act, last_word);
+    e[0] = TAIL ? rans_step_tail(x, lut_addr + kCosetTableOff, mask, b, wa, lt, act)
+                : rans_step<kCosetTableOff>(x, lut_addr, mask, b, wa, lt);
     const uint32_t coff = e[0] & kCodeMask;          // 0 or 65536: byte offset of this coset's tables
     const uint32_t tab = lut_addr + coff;
+    if (TAIL) {
 #pragma unroll
-    for (int k = 1; k <= 8; ++k)
-        e[k] = rans_step<TAIL, CAREFUL>(x, tab + uint32_t(k - 1) * kLutStride, mask, b, ptr, pay, lt, act, last_word);
+        for (int k = 1; k <= 8; ++k) e[k] = rans_step_tail(x, tab + uint32_t(k - 1) * kLutStride, mask, b, wa, lt, act);
+    } else {
+        e[1] = rans_step<0 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[2] = rans_step<1 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[3] = rans_step<2 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[4] = rans_step<3 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[5] = rans_step<4 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[6] = rans_step<5 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[7] = rans_step<6 * kLutStride>(x, tab, mask, b, wa, lt);
+        e[8] = rans_step<7 * kLutStride>(x, tab, mask, b, wa, lt);
+    }
     if (TAIL && !act) return;
     // parity of z1 + ... + z7 = xor of the codes' lowest bits (zlo is even); it is the lowest bit of z8
     const uint32_t par = (e[1] ^ e[2] ^ e[3] ^ e[4] ^ e[5] ^ e[6] ^ e[7]) & 0x800u;
@@ -230,59 +305,120 @@ __device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &ptr, const u
 #pragma unroll
         for (int k = 1; k <= 7; ++k) f[k] = int32_t((e[k] & kCodeMask) >> 11) + zlo;
         f[8] = (int32_t((e[8] & kCodeMask) >> 11) + zlo) >> 1;
-        return;
     } else {
-        // 4096 + code as fp32; subtracting kc = 4096 - zlo - c/2 gives p = z + c/2 exactly
-        const float kc = __uint_as_float(__float_as_uint(k0) - (coff >> 6));   // one ulp here is 2^-11: c/2 = 1024 ulps
+        // (entry & mask) | 0x45800000 is 4096 + code as fp32; subtracting kc = 4096 - zlo - c/2 gives
+        // p = z + c/2 exactly (one ulp here is 2^-11, so c/2 is 1024 ulps of the bit pattern)
+        const uint32_t kc = k0_bits - (coff >> 6);
+        const uint64_t kk = pack64(kc, kc);
+        const uint64_t ss = pack64(__float_as_uint(sigma), __float_as_uint(sigma));
+        uint32_t xb[8];
+#pragma unroll
+        for (int k = 1; k <= 7; ++k) xb[k - 1] = (e[k] & kCodeMask) | kExp4096;
+        xb[7] = (e[8] & kCodeMask) | par | kExp4096;
         float w[8];
+#ifdef EP_SCALAR_FP32
 #pragma unroll
-        for (int k = 1; k <= 7; ++k) w[k - 1] = __uint_as_float((e[k] & kCodeMask) | kExp4096);
-        w[7] = __uint_as_float((e[8] & kCodeMask) | par | kExp4096);
+        for (int i = 0; i < 8; ++i) w[i] = __fmul_rn(__fsub_rn(__uint_as_float(xb[i]), __uint_as_float(kc)), sigma);
+        (void)kk; (void)ss;
+#else
 #pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            sub2(w[i], w[i + 1], kc);
-            mul2(w[i], w[i + 1], sigma);
-        }
+        for (int i = 0; i < 8; i += 2) unpack64(mul2(sub2(pack64(xb[i], xb[i + 1]), kk), ss), w[i], w[i + 1]);
+#endif
         Out<DT>::store(dst, w);
     }
 }
 
-template <int DT>
-struct BlockBytes { static constexpr uint32_t value = Out<DT>::kBlockBytes; };
-template <>
-struct BlockBytes<EP_FIELDS_I32> { static constexpr uint32_t value = 36; };
+// ---- payload ring ------------------------------------------------------------------------------------
+// chunk c of a tile = global bytes [a0 + 512c, a0 + 512c + 512), a0 = tile's first word rounded down to
+// 16 bytes; it lives in ring slot c & 3.  `room` = bytes from a0 to the end of the payload: nothing
+// beyond it is read (cp.async zero-fills the rest).
+__device__ __forceinline__ void ring_issue(uint32_t ring, uint64_t a0, uint32_t room, uint32_t c, uint32_t lane) {
+    uint32_t o = 512u * c + 16u * lane;
+    uint32_t n = 16;
+    if (o + 16u > room) {
+        n = o < room ? room - o : 0u;
+        if (n == 0) o = 0;                       // nothing is read, but keep the address a valid one
+    }
+    const uint32_t slot = c & 3u;
+    const uint32_t dst = ring + 512u * slot + 16u * lane;
+    cp_async16(dst, a0 + o, n);
+    if (slot == 0 || (slot == 1 && lane < 8)) cp_async16(dst + kRingBytes, a0 + o, n);   // mirror of the first 640 bytes
+    cp_async_commit();
+}
 
-template <int DT, bool CAREFUL>
-__device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t lane) {
+// The cursor entered a new 512-byte chunk: request chunks up to three ahead of it and wait for all but
+// the newest.  `threshold` = start of the chunk after the cursor's at the previous service; chunks up
+// to (threshold >> 9) + 2 have been requested.  A group touches at most 576 + 62 bytes from its start,
+// i.e. chunks cur .. cur+2, which are complete after this call.
+__device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_t room, uint32_t pos, uint32_t &threshold,
+                                             uint32_t lane) {
+    const uint32_t cur = pos >> 9;
+    for (uint32_t c = (threshold >> 9) + 3u; c < cur + 4u; ++c) ring_issue(ring, a0, room, c, lane);
+    cp_async_wait<1>();
+    __syncwarp();
+    threshold = 512u * (cur + 1u);
+}
+
+// WIDE: rows hold at least 32 vectors, so a group advances the row index by at most one.
+// FULL: the tile holds exactly V vectors, so every loop bound is a kernel parameter.  The compiler then
+// sees warp-uniform control flow throughout the hot loop and emits no divergence handling around the
+// warp votes; a ragged last tile takes the same code with data-dependent bounds.
+template <int DT, bool WIDE, bool FULL>
+__device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
     uint32_t x = rec[lane];
-    uint32_t ptr = rec[32];
+    const uint32_t off = rec[32];
     const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
     const uint32_t v0 = tile * J.V;
-    const uint32_t nv = min(J.V, J.n_vec - v0);
+    const uint32_t nv = FULL ? J.V : min(J.V, J.n_vec - v0);
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
-    const uint16_t *pay = reinterpret_cast<const uint16_t *>(J.stream + J.off_payload);
-    const uint32_t last_word = J.total_words ? J.total_words - 1 : 0;
-    const float k0 = float(4096 - J.zlo);
+    const uint32_t per_row = J.per_row;
+    const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
+    const uint64_t first = pay + 2ull * off;
+    const uint64_t a0 = first & ~15ull;
+    const uint32_t lead = uint32_t(first - a0);
+    const uint32_t room = uint32_t(pay + 2ull * J.total_words - a0);     // the payload is shorter than 4 GB
+    uint32_t pos = lead;          // byte position of the cursor relative to a0
+    uint32_t threshold;           // next chunk boundary the cursor has not yet crossed
+    for (uint32_t c = 0; c < 4; ++c) ring_issue(ring, a0, room, c, lane);
+    cp_async_wait<1>();
+    __syncwarp();
+    threshold = 512u;
+    const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
     uint32_t v = v0 + lane;
-    uint32_t row = v / J.per_row, col = v - row * J.per_row;
+    uint32_t row = v / per_row, col = v - row * per_row;
     uint8_t *dst = static_cast<uint8_t *>(J.out) + size_t(v) * BlockBytes<DT>::value;
     const uint32_t full = nv >> 5;
     for (uint32_t g = 0; g < full; ++g) {
-        if (lane < 4) prefetch_l1(pay + min(ptr + 256u + 64u * lane, last_word));   // next lines of this tile's words
+        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
+        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
+        uint32_t wa = wa0;
         const float sigma = (DT == EP_FIELDS_I32) ? 0.f : __ldg(J.scales + row);
-        decode_group<DT, false, CAREFUL>(x, ptr, pay, lut_addr, mask, b, lt, true, last_word, k0, sigma, J.zlo, dst);
+        decode_group<DT, false>(x, wa, lut_addr, mask, b, lt, true, k0_bits, sigma, J.zlo, dst);
+        pos += wa - wa0;
         dst += 32u * BlockBytes<DT>::value;
         col += 32;
-        while (col >= J.per_row) { col -= J.per_row; ++row; }
+        if (WIDE) {
+            const bool wrap = col >= per_row;
+            col -= wrap ? per_row : 0u;
+            row += wrap ? 1u : 0u;
+        } else {
+            while (col >= per_row) { col -= per_row; ++row; }
+        }
     }
     if (nv & 31u) {
+        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
+        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
+        uint32_t wa = wa0;
         const bool act = lane < (nv & 31u);
         const float sigma = (DT == EP_FIELDS_I32 || !act) ? 0.f : __ldg(J.scales + row);
-        decode_group<DT, true, CAREFUL>(x, ptr, pay, lut_addr, mask, b, lt, act, last_word, k0, sigma, J.zlo, dst);
+        decode_group<DT, true>(x, wa, lut_addr, mask, b, lt, act, k0_bits, sigma, J.zlo, dst);
+        pos += wa - wa0;
     }
+    cp_async_wait<0>();          // nothing may still be landing in the ring when the next tile starts
+    __syncwarp();
     // integrity: the encoder started every state at 2^15 and the tile's words end where the next tile's begin
-    const bool bad = (x != ep::kStateLow) || (ptr != end);
+    const bool bad = (x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end);
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
 }
 
@@ -294,17 +430,27 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
     while (j + 1 < P.n_jobs && blockIdx.x >= P.job[j + 1].cta_begin) ++j;
     const JobParams &J = P.job[j];
     const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
+    const uint32_t ring = lut_addr + kLutBytes + warp * kRingStride;
     build_tables_smem(J, lut_addr, warp, lane);
     __syncthreads();
     const uint32_t cta = blockIdx.x - J.cta_begin;
-    for (uint32_t tile = cta * kWarps + warp; tile < J.n_tiles; tile += J.cta_count * kWarps) {
-        // a damaged stream could ask for up to one word per symbol: only tiles that close to the end of the
-        // payload need their word index clamped
-        const uint32_t off = J.tile_index[size_t(tile) * 33u + 32u];
-        const uint32_t nv = min(J.V, J.n_vec - tile * J.V);
-        if (uint64_t(off) + 9ull * nv >= J.total_words) decode_tile<DT, true>(J, tile, lut_addr, lane);
-        else decode_tile<DT, false>(J, tile, lut_addr, lane);
+    // Rounds over the full tiles: warp w of CTA c takes tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and
+    // the test for a CTA past the end are functions of blockIdx and kernel parameters only, so control flow stays
+    // warp-uniform in the compiler's eyes; inside the one CTA that straddles the end, warps past it redo the last full
+    // tile (the same bytes are written twice) instead of branching around the hot loop.
+    const bool wide = J.per_row >= 32u;
+    if (cta < J.cta_count) {
+        for (uint32_t i = 0; i < J.iters; ++i) {
+            const uint32_t base = (cta + i * J.cta_count) * kWarps;
+            if (base >= J.n_full) break;
+            const uint32_t tile = min(base + warp, J.n_full - 1u);
+            if (wide) decode_tile<DT, true, true>(J, tile, lut_addr, ring, lane);
+            else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
+        }
     }
+    // a ragged last tile belongs to warp 0 of one CTA chosen by the host (an extra CTA when the GPU has room for it)
+    if (J.n_full < J.n_tiles && cta == J.last_cta && warp == 0)
+        decode_tile<DT, false, false>(J, J.n_tiles - 1u, lut_addr, ring, lane);
 }
 
 // ---- host side -----------------------------------------------------------------------------------
@@ -361,11 +507,11 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kLutBytes));
+        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    ep_decode_smem_kernel<DT><<<grid, kThreads, kLutBytes, st>>>(P);
+    ep_decode_smem_kernel<DT><<<grid, kThreads, kSmemBytes, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -427,6 +573,19 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *
         J.zlo = int32_t(even_base(coord_range(I)));
         J.cta_begin = next;
         J.cta_count = uint32_t(share);
+        const bool ragged = (uint64_t(J.n_vec) % I.V) != 0;
+        J.n_full = ragged ? I.n_tiles - 1u : I.n_tiles;
+        const uint32_t round_tiles = J.cta_count * uint32_t(kWarps);
+        J.iters = (J.n_full + round_tiles - 1u) / round_tiles;
+        J.last_cta = 0;
+        uint32_t extra = 0;
+        if (ragged) {
+            // CTAs [0, used) have work in the last round; prefer an extra CTA while the launch still fits the SMs,
+            // else the first CTA that is idle (or least loaded) in the last round
+            const uint32_t used = J.n_full ? ((J.n_full - (J.iters - 1u) * round_tiles) + uint32_t(kWarps) - 1u) / uint32_t(kWarps) : 0u;
+            if (uint64_t(next) + share < uint64_t(sms) && n_jobs == 1) { J.last_cta = J.cta_count; extra = 1; }
+            else J.last_cta = used % J.cta_count;
+        }
         uint32_t acc = 0;
         for (int t = 0; t < EP_NUM_TABLES; ++t) {
             J.tmin[t] = int16_t(I.table_min[t]);
@@ -434,7 +593,7 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *
             J.foff[t] = uint16_t(acc);
             acc += I.table_K[t];
         }
-        next += uint32_t(share);
+        next += uint32_t(share) + extra;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
