@@ -38,7 +38,7 @@ NCU_TRAFFIC_BYTES = {}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c5"])
@@ -104,7 +104,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.gpu), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -114,7 +114,16 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line)
 
-    def stop(self):
+    def wait_first(self, timeout=5.0):
+        t0 = time.time()
+        while self.proc is not None and not self.lines and time.time() - t0 < timeout:
+            time.sleep(0.01)
+
+    def mark(self):
+        """Index of the next sample: samples from here on were taken during the timed region."""
+        return len(self.lines)
+
+    def stop(self, start=0, min_samples=3):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -123,7 +132,8 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        lines = self.lines[start:] if len(self.lines) - start >= min_samples else self.lines
+        for ln in lines:
             p = [t.strip() for t in ln.split(",")]
             if len(p) < 9:
                 continue
@@ -172,7 +182,8 @@ def run_reference(args):
     import paper_2609_34185_b200 as ep
     blob = ep.encode(layers[0][0], bpp, tile_vectors=V)
     I = blob.info
-    params, dt, tiles, threads = oracle_sample(blob, dtype_name, 0.5)
+    # each step decodes a leading tile range sized so that the whole run stays near a minute
+    params, dt, tiles, threads = oracle_sample(blob, dtype_name, min(0.5, 60.0 / max(1, args.steps + args.warmup)))
     times = []
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
@@ -256,17 +267,18 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        sampler.wait_first()
     for _ in range(max(args.warmup, 3)):
         flush.fill_(1)
         step()
     barrier()
     if ep.last_device_status() != 0:
         raise RuntimeError("decoder reported an inconsistent stream during warm-up")
-
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     barrier()
+    mark = sampler.mark()
     evs = []
     for _ in range(args.steps):
         flush.fill_(0)      # L2 flush between timed iterations, outside the events
@@ -276,7 +288,7 @@ def main():
         e.record(stream)
         evs.append((s, e))
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(mark) if rank == 0 else None
     times_ms = [s.elapsed_time(e) for s, e in evs]
     total_ms = sum(times_ms)
     if world > 1:

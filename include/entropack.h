@@ -79,6 +79,10 @@ typedef struct {
     int32_t b_start;               /* 0 = 11 for targets <= 7 bpp, 12 above */
     int32_t b_max;                 /* 15 */
     double retained_bits;          /* constant of Eq. 10 (bits assumed to stay in each state): 16 */
+    int32_t polish_steps;          /* corrections of s from the full-tensor estimate after Algorithm 1 (an
+                                      addition to the paper's procedure; 0 = the literal Algorithm 1): 3 */
+    double polish_retained_bits;   /* bits per state taken as retained in those corrections: 8 (states end up
+                                      spread over [2^15, 2^31), so about 8 bits each stay out of the payload) */
     int32_t threads;               /* host worker threads; 0 = all hardware threads */
 } ep_encode_opts;
 

@@ -58,6 +58,9 @@ typedef struct {
     int32_t b_start;               /* 0 = 11 for targets <= 7 bpp, else 12 */
     int32_t b_max;                 /* default 15 */
     double retained_bits;          /* constant of Eq. 10, default 16 */
+    int32_t polish_steps;          /* full-tensor corrections of s after Algorithm 1 (not in the paper), default 3 */
+    double polish_retained_bits;   /* bits per state assumed retained in those corrections: 8, the measured mean
+                                      of log2(final state / 2^15) for states spread over [2^15, 2^31) */
 } epo_opts;
 
 typedef struct {
@@ -96,6 +99,8 @@ void epo_default_opts(epo_opts *o) {
     o->bracket_lo = 1e-3; o->bracket_hi = 8.0; o->search_steps = 12;
     o->sample_vectors = 1u << 18; o->tile_vectors = 0; o->b_start = 0; o->b_max = 15;
     o->retained_bits = 16.0;
+    o->polish_steps = 3;
+    o->polish_retained_bits = 8.0;
 }
 
 void epo_free(void *p) { free(p); }
@@ -840,6 +845,44 @@ int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const 
             s32 = (float)(1.05 * (double)s32 * (double)amax / (double)(1u << b));   /* coarsen */
         }
         if (done) break;
+    }
+    /* Not in Algorithm 1: the sampled tables see fewer rare symbols than the full tensor, so on heavy-tailed
+     * inputs the stored rate lands above the sampled estimate.  Correct s from the full-tensor estimate of
+     * Eq. 10-11 (first with the one-bit-per-doubling law of Eq. 9, then with the measured slope) and
+     * requantise, at most polish_steps times. */
+    double ls_prev = 0.0, r_prev = 0.0;
+    int have_prev = 0;
+    for (int ps = 0; ps < o.polish_steps; ++ps) {
+        epo_tab t[EPO_NT];
+        tabs_count(fields, nvec, t);
+        tabs_normalise(t, b);
+        double est = estimate_bits(t, b, nvec, R, V, o.polish_retained_bits, NULL) / ((double)R * (double)C);
+        tabs_free(t);
+        if (fabs(est - target_bpp) <= 0.002 * target_bpp) break;
+        /* bits per doubling of s: 1 by Eq. 9 at first, then the secant through the last two evaluations */
+        double ls = log2((double)s32), slope = 1.0;
+        if (have_prev && ls != ls_prev) {
+            slope = -(est - r_prev) / (ls - ls_prev);
+            if (!(slope >= 0.5)) slope = 0.5;
+            if (slope > 4.0) slope = 4.0;
+        }
+        ls_prev = ls; r_prev = est; have_prev = 1;
+        float s_prev = s32;
+        s32 = (float)exp2(ls + (est - target_bpp) / slope);
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < (int64_t)R; ++r)
+            quantise_row(W + (size_t)r * C, C, mu[r], s32, fields + 9 * (size_t)r * (C / 8));
+        tabs_count(fields, nvec, t);
+        uint32_t worst = 0;
+        for (int i = 0; i < EPO_NT; ++i) { uint32_t ob = tabs_observed(t, i); if (ob > worst) worst = ob; }
+        tabs_free(t);
+        if (worst > (1u << b)) {      /* a finer scale no longer fits the tables: go back and stop */
+            s32 = s_prev;
+#pragma omp parallel for schedule(static)
+            for (int64_t r = 0; r < (int64_t)R; ++r)
+                quantise_row(W + (size_t)r * C, C, mu[r], s32, fields + 9 * (size_t)r * (C / 8));
+            break;
+        }
     }
     float *sigma = (float *)malloc(sizeof(float) * R);
     epo_refit(W, R, C, fields, s32, mu, sigma);

@@ -422,6 +422,261 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
 }
 
+// ---- the hot loop in PTX -------------------------------------------------------------------------------
+// All full groups of one full tile.  Written as one asm statement so that every branch can be marked
+// warp-uniform (bra.uni) and the rare work - refilling the payload ring, moving to the next row - sits
+// out of line.  Per group: 9 x rans step, Eq. 5 / Eq. 19 on eight weights, one vector store.
+//
+// Register roles (asm operands):
+//   x      rANS state                      wa    cursor (shared-memory byte address)
+//   wthr   cursor value that triggers the next ring service (next 512-byte chunk boundary)
+//   wbase  wa - (byte position of the cursor relative to a0)
+//   col,row  this lane's block column inside its row / row index;  sig = row scale bits
+//   doff   byte offset of this lane's block in the output;  left = groups still to do
+//   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
+//                     the payload bytes left from there (may be <= 0)
+#define EP_S_STEP(E, TAB, OFF)                                  \
+    "and.b32 u, %0, %13;\n\t"                                   \
+    "shl.b32 u, u, 2;\n\t"                                      \
+    "add.u32 u, u, " TAB ";\n\t"                                \
+    "ld.shared.u32 " E ", [u+" OFF "];\n\t"                     \
+    "shr.u32 f, " E ", 20;\n\t"                                 \
+    "and.b32 bias, " E ", 0x7FF;\n\t"                           \
+    "shr.u32 q, %0, %14;\n\t"                                   \
+    "mad.lo.u32 %0, f, q, bias;\n\t"                            \
+    "setp.lt.u32 p, %0, 32768;\n\t"                             \
+    "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"              \
+    "and.b32 t, bal, %12;\n\t"                                  \
+    "popc.b32 t, t;\n\t"                                        \
+    "shl.b32 t, t, 1;\n\t"                                      \
+    "add.u32 t, t, %1;\n\t"                                     \
+    "ld.shared.u16 w, [t];\n\t"                                 \
+    "@p mad.lo.u32 %0, %0, 65536, w;\n\t"                       \
+    "popc.b32 t, bal;\n\t"                                      \
+    "shl.b32 t, t, 1;\n\t"                                      \
+    "add.u32 %1, %1, t;\n\t"
+
+#define EP_S_PAIR(P, XA, XB, WA, WB)                            \
+    "mov.b64 " P ", {" XA ", " XB "};\n\t"                      \
+    "sub.rn.f32x2 " P ", " P ", kk;\n\t"                        \
+    "mul.rn.f32x2 " P ", " P ", ss;\n\t"                        \
+    "mov.b64 {" WA ", " WB "}, " P ";\n\t"
+
+#define EP_S_STORE_BF16                                         \
+    "cvt.rn.bf16x2.f32 o0, w1, w0;\n\t"                         \
+    "cvt.rn.bf16x2.f32 o1, w3, w2;\n\t"                         \
+    "cvt.rn.bf16x2.f32 o2, w5, w4;\n\t"                         \
+    "cvt.rn.bf16x2.f32 o3, w7, w6;\n\t"                         \
+    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"
+#define EP_S_STORE_FP16                                         \
+    "cvt.rn.satfinite.f16x2.f32 o0, w1, w0;\n\t"                \
+    "cvt.rn.satfinite.f16x2.f32 o1, w3, w2;\n\t"                \
+    "cvt.rn.satfinite.f16x2.f32 o2, w5, w4;\n\t"                \
+    "cvt.rn.satfinite.f16x2.f32 o3, w7, w6;\n\t"                \
+    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"
+#define EP_S_STORE_E4M3                                         \
+    "cvt.rn.satfinite.e4m3x2.f32 h0, w1, w0;\n\t"               \
+    "cvt.rn.satfinite.e4m3x2.f32 h1, w3, w2;\n\t"               \
+    "cvt.rn.satfinite.e4m3x2.f32 h2, w5, w4;\n\t"               \
+    "cvt.rn.satfinite.e4m3x2.f32 h3, w7, w6;\n\t"               \
+    "mov.b32 o0, {h0, h1};\n\t"                                 \
+    "mov.b32 o1, {h2, h3};\n\t"                                 \
+    "st.global.v2.b32 [ad], {o0, o1};\n\t"
+#define EP_S_STORE_INT8                                         \
+    "cvt.rni.sat.s8.f32 o0, w0;\n\t"                            \
+    "cvt.rni.sat.s8.f32 o2, w1;\n\t"                            \
+    "and.b32 o0, o0, 0xFF;\n\t"                                 \
+    "bfi.b32 o0, o2, o0, 8, 8;\n\t"                             \
+    "cvt.rni.sat.s8.f32 o2, w2;\n\t"                            \
+    "bfi.b32 o0, o2, o0, 16, 8;\n\t"                            \
+    "cvt.rni.sat.s8.f32 o2, w3;\n\t"                            \
+    "bfi.b32 o0, o2, o0, 24, 8;\n\t"                            \
+    "cvt.rni.sat.s8.f32 o1, w4;\n\t"                            \
+    "cvt.rni.sat.s8.f32 o2, w5;\n\t"                            \
+    "and.b32 o1, o1, 0xFF;\n\t"                                 \
+    "bfi.b32 o1, o2, o1, 8, 8;\n\t"                             \
+    "cvt.rni.sat.s8.f32 o2, w6;\n\t"                            \
+    "bfi.b32 o1, o2, o1, 16, 8;\n\t"                            \
+    "cvt.rni.sat.s8.f32 o2, w7;\n\t"                            \
+    "bfi.b32 o1, o2, o1, 24, 8;\n\t"                            \
+    "st.global.v2.b32 [ad], {o0, o1};\n\t"
+
+#define EP_FULL_GROUPS_ASM(STORE, GROUP_BYTES)                                                                        \
+    asm volatile(                                                                                                     \
+        "{\n\t"                                                                                                       \
+        ".reg .pred p, ps, pw, pa, pl, pq, pv, pm, pm1, plow;\n\t"                                                    \
+        ".reg .b32 u, f, q, bias, bal, t, w, coff, tab, kc, par, pos, cur, lim, n, slot, d;\n\t"                      \
+        ".reg .b32 e0, e1, e2, e3, e4, e5, e6, e7, e8, x1, x2, x3, x4, x5, x6, x7, x8, o0, o1, o2, o3;\n\t"           \
+        ".reg .b16 h0, h1, h2, h3;\n\t"                                                                               \
+        ".reg .f32 w0, w1, w2, w3, w4, w5, w6, w7;\n\t"                                                               \
+        ".reg .b64 kk, ss, p0, p1, p2, p3, ad, src;\n\t"                                                              \
+        "setp.lt.u32 plow, %22, 128;\n\t"                                                                             \
+        "EP_LOOP:\n\t"                                                                                                \
+        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
+        "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
+        "@ps bra.uni EP_SERVICE;\n\t"                                                                                 \
+        "EP_RESUME:\n\t"                                                                                              \
+        EP_S_STEP("e0", "%15", "131072")                                                                              \
+        "and.b32 coff, e0, 0xFF800;\n\t"                                                                              \
+        "add.u32 tab, %15, coff;\n\t"                                                                                 \
+        EP_S_STEP("e1", "tab", "0")                                                                                   \
+        EP_S_STEP("e2", "tab", "8192")                                                                                \
+        EP_S_STEP("e3", "tab", "16384")                                                                               \
+        EP_S_STEP("e4", "tab", "24576")                                                                               \
+        EP_S_STEP("e5", "tab", "32768")                                                                               \
+        EP_S_STEP("e6", "tab", "40960")                                                                               \
+        EP_S_STEP("e7", "tab", "49152")                                                                               \
+        EP_S_STEP("e8", "tab", "57344")                                                                               \
+        /* Eq. 5: 4096 + code as fp32, minus kc = 4096 - zlo - c/2 (one ulp = 2^-11, c/2 = 1024 ulps) */              \
+        "shr.u32 t, coff, 6;\n\t"                                                                                     \
+        "sub.u32 kc, %18, t;\n\t"                                                                                     \
+        "lop3.b32 x1, e1, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x2, e2, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x3, e3, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x4, e4, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x5, e5, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x6, e6, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x7, e7, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 par, e1, e2, e3, 0x96;\n\t"                                                                         \
+        "lop3.b32 par, par, e4, e5, 0x96;\n\t"                                                                        \
+        "lop3.b32 par, par, e6, e7, 0x96;\n\t"                                                                        \
+        "lop3.b32 par, par, 0x800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x8, e8, 0xFF800, par, 0xEA;\n\t"                                                                    \
+        "mov.b64 kk, {kc, kc};\n\t"                                                                                   \
+        "mov.b64 ss, {%6, %6};\n\t"                                                                                   \
+        EP_S_PAIR("p0", "x1", "x2", "w0", "w1")                                                                       \
+        EP_S_PAIR("p1", "x3", "x4", "w2", "w3")                                                                       \
+        EP_S_PAIR("p2", "x5", "x6", "w4", "w5")                                                                       \
+        EP_S_PAIR("p3", "x7", "x8", "w6", "w7")                                                                       \
+        "cvt.u64.u32 ad, %7;\n\t"                                                                                     \
+        "add.s64 ad, ad, %19;\n\t"                                                                                    \
+        STORE                                                                                                         \
+        "add.u32 %7, %7, " #GROUP_BYTES ";\n\t"                                                                       \
+        "add.u32 %4, %4, 32;\n\t"                                                                                     \
+        "setp.ge.u32 pw, %4, %17;\n\t"                                                                                \
+        "vote.sync.any.pred pa, pw, 0xffffffff;\n\t"                                                                  \
+        "@pa bra.uni EP_ROWCHG;\n\t"                                                                                  \
+        "EP_ROWDONE:\n\t"                                                                                             \
+        "sub.u32 %8, %8, 1;\n\t"                                                                                      \
+        "setp.ne.u32 pl, %8, 0;\n\t"                                                                                  \
+        "@pl bra.uni EP_LOOP;\n\t"                                                                                    \
+        "bra.uni EP_DONE;\n\t"                                                                                        \
+        /* ---- some lane moved to the next row: reload its scale ---- */                                             \
+        "EP_ROWCHG:\n\t"                                                                                              \
+        "@pw sub.u32 %4, %4, %17;\n\t"                                                                                \
+        "@pw add.u32 %5, %5, 1;\n\t"                                                                                  \
+        "min.u32 t, %5, %23;\n\t"                                                                                     \
+        "mul.wide.u32 ad, t, 4;\n\t"                                                                                  \
+        "add.s64 ad, ad, %20;\n\t"                                                                                    \
+        "@pw ld.global.nc.b32 %6, [ad];\n\t"                                                                          \
+        "bra.uni EP_ROWDONE;\n\t"                                                                                     \
+        /* ---- the cursor entered a new 512-byte chunk: request chunks up to cur+3, wait for all but the newest */   \
+        "EP_SERVICE:\n\t"                                                                                             \
+        "sub.u32 pos, %1, %3;\n\t"                                                                                    \
+        "shr.u32 cur, pos, 9;\n\t"                                                                                    \
+        "add.u32 lim, cur, 4;\n\t"                                                                                    \
+        "EP_SVC_LOOP:\n\t"                                                                                            \
+        "setp.ge.u32 pq, %11, lim;\n\t"                                                                               \
+        "@pq bra.uni EP_SVC_DONE;\n\t"                                                                                \
+        "min.s32 n, %10, 16;\n\t"                                                                                     \
+        "max.s32 n, n, 0;\n\t"                                                                                        \
+        "setp.gt.s32 pv, %10, 0;\n\t"                                                                                 \
+        "selp.b64 src, %9, %21, pv;\n\t"                                                                              \
+        "and.b32 slot, %11, 3;\n\t"                                                                                   \
+        "shl.b32 d, slot, 9;\n\t"                                                                                     \
+        "add.u32 d, d, %16;\n\t"                                                                                      \
+        "add.u32 d, d, %22;\n\t"                                                                                      \
+        "cp.async.cg.shared.global [d], [src], 16, n;\n\t"                                                            \
+        "setp.eq.u32 pm, slot, 0;\n\t"                                                                                \
+        "setp.eq.u32 pm1, slot, 1;\n\t"                                                                               \
+        "and.pred pm1, pm1, plow;\n\t"                                                                                \
+        "or.pred pm, pm, pm1;\n\t"                                                                                    \
+        "@pm cp.async.cg.shared.global [d+2048], [src], 16, n;\n\t"                                                   \
+        "cp.async.commit_group;\n\t"                                                                                  \
+        "add.s64 %9, %9, 512;\n\t"                                                                                    \
+        "sub.s32 %10, %10, 512;\n\t"                                                                                  \
+        "add.u32 %11, %11, 1;\n\t"                                                                                    \
+        "bra.uni EP_SVC_LOOP;\n\t"                                                                                    \
+        "EP_SVC_DONE:\n\t"                                                                                            \
+        "cp.async.wait_group 1;\n\t"                                                                                  \
+        "bar.warp.sync 0xffffffff;\n\t"                                                                               \
+        "and.b32 t, pos, 2047;\n\t"                                                                                   \
+        "add.u32 %1, %16, t;\n\t"                                                                                     \
+        "sub.u32 %3, %1, pos;\n\t"                                                                                    \
+        "shl.b32 t, cur, 9;\n\t"                                                                                      \
+        "add.u32 t, t, 512;\n\t"                                                                                      \
+        "add.u32 %2, %3, t;\n\t"                                                                                      \
+        "bra.uni EP_RESUME;\n\t"                                                                                      \
+        "EP_DONE:\n\t"                                                                                                \
+        "}"                                                                                                           \
+        /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
+        : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(col), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
+          "+&r"(left), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                          \
+        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),            \
+          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max)                                                             \
+        : "memory")
+
+// One full tile (exactly V vectors) of a tensor whose rows hold at least 32 blocks: the full groups in
+// PTX, a last partial group (V not a multiple of 32) through decode_group.
+template <int DT>
+__device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring,
+                                                 uint32_t lane) {
+    const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
+    uint32_t x = rec[lane];
+    const uint32_t off = rec[32];
+    const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
+    const uint32_t v0 = tile * J.V;
+    const uint32_t nv = J.V;
+    const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
+    const uint32_t per_row = J.per_row;
+    const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
+    const uint64_t first = pay + 2ull * off;
+    const uint64_t a0 = first & ~15ull;
+    const uint32_t lead = uint32_t(first - a0);
+    const uint32_t room = uint32_t(pay + 2ull * J.total_words - a0);     // the payload is shorter than 2 GB
+    const uint32_t lane16 = 16u * lane;
+    for (uint32_t c = 0; c < 4; ++c) ring_issue(ring, a0, room, c, lane);
+    cp_async_wait<1>();
+    __syncwarp();
+    uint32_t wa = ring + lead;                    // cursor
+    uint32_t wbase = ring;                        // wa - position
+    uint32_t wthr = ring + 512u;                  // next chunk boundary
+    uint64_t srcp = a0 + 2048u + lane16;          // this lane's part of chunk 4
+    uint32_t rem = room - (2048u + lane16);       // signed in the asm: may be negative
+    uint32_t nextc = 4;
+    const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
+    const uint32_t v = v0 + lane;
+    uint32_t row = v / per_row, col = v - row * per_row;
+    const float *scales = J.scales;
+    uint32_t sig = __float_as_uint(__ldg(scales + row));
+    uint32_t doff = v * Out<DT>::kBlockBytes;
+    const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
+    uint32_t left = nv >> 5;
+    const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
+    if (left) {
+        if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
+        else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
+        else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
+        else EP_FULL_GROUPS_ASM(EP_S_STORE_INT8, 256);
+    }
+    uint32_t pos = wa - wbase;
+    if (nv & 31u) {
+        uint32_t threshold = wthr - wbase;
+        // chunks up to (threshold >> 9) + 2 are requested: the same bookkeeping as ring_service expects
+        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
+        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
+        uint32_t wt = wa0;
+        const bool act = lane < (nv & 31u);
+        decode_group<DT, true>(x, wt, lut_addr, mask, b, lt, act, k0_bits, __uint_as_float(sig), J.zlo,
+                               static_cast<uint8_t *>(J.out) + doff);
+        pos += wt - wa0;
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+    const bool bad = (x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end);
+    if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __grid_constant__ BatchParams P) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -444,8 +699,13 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
             const uint32_t base = (cta + i * J.cta_count) * kWarps;
             if (base >= J.n_full) break;
             const uint32_t tile = min(base + warp, J.n_full - 1u);
-            if (wide) decode_tile<DT, true, true>(J, tile, lut_addr, ring, lane);
-            else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
+            if constexpr (DT != EP_FIELDS_I32) {
+                if (wide) decode_tile_fast<DT>(J, tile, lut_addr, ring, lane);
+                else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
+            } else {
+                if (wide) decode_tile<DT, true, true>(J, tile, lut_addr, ring, lane);
+                else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
+            }
         }
     }
     // a ragged last tile belongs to warp 0 of one CTA chosen by the host (an extra CTA when the GPU has room for it)

@@ -430,6 +430,8 @@ extern "C" void ep_encode_opts_default(ep_encode_opts *o) {
     o->b_start = 0;
     o->b_max = 15;
     o->retained_bits = 16.0;
+    o->polish_steps = 3;
+    o->polish_retained_bits = 8.0;
     o->threads = 0;
 }
 
@@ -441,7 +443,7 @@ extern "C" int ep_encode(const float *W, uint32_t R, uint32_t C, double target_b
     if (nvec >= (1ull << 32)) return EP_ERR_BAD_ARG;
     ep_encode_opts o;
     if (opts_in) o = *opts_in; else ep_encode_opts_default(&o);
-    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.b_max > 15 || o.b_max < 9 ||
+    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.polish_steps < 0 || o.b_max > 15 || o.b_max < 9 ||
         (o.b_start != 0 && (o.b_start < 9 || o.b_start > o.b_max)))
         return EP_ERR_BAD_ARG;
     try {
@@ -487,6 +489,40 @@ extern "C" int ep_encode(const float *W, uint32_t R, uint32_t C, double target_b
                 s = float(1.05 * double(s) * double(amax) / double(1u << b));
             }
             if (fits) break;
+        }
+        // Beyond Algorithm 1: steer s with the full-tensor estimate (Eq. 10-11), first by the one-bit-per-doubling
+        // law (Eq. 9), then by the measured slope.  The sampled tables miss rare symbols of the full tensor, which costs rate on heavy tails.
+        struct { double log_s, rate; bool valid; } last{0.0, 0.0, false};
+        for (int step = 0; step < o.polish_steps; ++step) {
+            double est;
+            {
+                Model m;
+                m.count(fields.data(), nvec, threads);
+                m.normalise(b);
+                est = estimate_bits(m, b, nvec, R, V, o.polish_retained_bits, nullptr) / (double(R) * double(C));
+            }
+            if (std::fabs(est - target_bpp) <= 0.002 * target_bpp) break;
+            // rate lost per doubling of s: 1 bit by Eq. 9 for the first move, afterwards the secant slope
+            const double log_s = std::log2(double(s));
+            double per_doubling = 1.0;
+            if (last.valid && log_s != last.log_s) {
+                per_doubling = -(est - last.rate) / (log_s - last.log_s);
+                if (!(per_doubling >= 0.5)) per_doubling = 0.5;
+                if (per_doubling > 4.0) per_doubling = 4.0;
+            }
+            last = {log_s, est, true};
+            const float before = s;
+            s = float(std::exp2(log_s + (est - target_bpp) / per_doubling));
+            quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
+            Model m;
+            m.count(fields.data(), nvec, threads);
+            uint32_t worst = 0;
+            for (const auto &tb : m.t) worst = std::max(worst, tb.observed());
+            if (worst > (1u << b)) {   // the finer scale overflows the tables: undo and stop
+                s = before;
+                quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
+                break;
+            }
         }
         std::vector<float> sigma(R);
         refit(W, R, C, fields.data(), s, mu.data(), sigma.data(), threads);
