@@ -868,7 +868,11 @@ int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const 
         }
         ls_prev = ls; r_prev = est; have_prev = 1;
         float s_prev = s32;
-        s32 = (float)exp2(ls + (est - target_bpp) / slope);
+        double s_new = exp2(ls + (est - target_bpp) / slope);
+        if (!(s_new >= o.bracket_lo)) s_new = o.bracket_lo;       /* stay inside the search bracket */
+        if (s_new > o.bracket_hi) s_new = o.bracket_hi;
+        s32 = (float)s_new;
+        if (s32 == s_prev) break;
 #pragma omp parallel for schedule(static)
         for (int64_t r = 0; r < (int64_t)R; ++r)
             quantise_row(W + (size_t)r * C, C, mu[r], s32, fields + 9 * (size_t)r * (C / 8));

@@ -435,17 +435,29 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 //   doff   byte offset of this lane's block in the output;  left = groups still to do
 //   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
 //                     the payload bytes left from there (may be <= 0)
-#define EP_S_STEP(E, TAB, OFF)                                  \
-    "and.b32 u, %0, %13;\n\t"                                   \
-    "shl.b32 u, u, 2;\n\t"                                      \
-    "add.u32 u, u, " TAB ";\n\t"                                \
-    "ld.shared.u32 " E ", [u+" OFF "];\n\t"                     \
+#ifdef EP_X_MULHI
+#define EP_S_FQ(E)                                              \
+    "mul.hi.u32 f, " E ", %24;\n\t"                             \
+    "mul.hi.u32 q, %0, %25;\n\t"
+#else
+#define EP_S_FQ(E)                                              \
     "shr.u32 f, " E ", 20;\n\t"                                 \
-    "and.b32 bias, " E ", 0x7FF;\n\t"                           \
-    "shr.u32 q, %0, %14;\n\t"                                   \
-    "mad.lo.u32 %0, f, q, bias;\n\t"                            \
-    "setp.lt.u32 p, %0, 32768;\n\t"                             \
-    "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"              \
+    "shr.u32 q, %0, %14;\n\t"
+#endif
+#ifdef EP_X_INCL
+/* %12 holds the mask of lanes <= this one: the inclusive count of lane 31 is the step's total */
+#define EP_S_FETCH                                              \
+    "and.b32 t, bal, %12;\n\t"                                  \
+    "popc.b32 t, t;\n\t"                                        \
+    "shfl.sync.idx.b32 u, t, 31, 31, 0xffffffff;\n\t"           \
+    "shl.b32 t, t, 1;\n\t"                                      \
+    "add.u32 t, t, %1;\n\t"                                     \
+    "ld.shared.u16 w, [t+-2];\n\t"                              \
+    "@p mad.lo.u32 %0, %0, 65536, w;\n\t"                       \
+    "shl.b32 u, u, 1;\n\t"                                      \
+    "add.u32 %1, %1, u;\n\t"
+#else
+#define EP_S_FETCH                                              \
     "and.b32 t, bal, %12;\n\t"                                  \
     "popc.b32 t, t;\n\t"                                        \
     "shl.b32 t, t, 1;\n\t"                                      \
@@ -455,6 +467,18 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
     "popc.b32 t, bal;\n\t"                                      \
     "shl.b32 t, t, 1;\n\t"                                      \
     "add.u32 %1, %1, t;\n\t"
+#endif
+#define EP_S_STEP(E, TAB, OFF)                                  \
+    "and.b32 u, %0, %13;\n\t"                                   \
+    "shl.b32 u, u, 2;\n\t"                                      \
+    "add.u32 u, u, " TAB ";\n\t"                                \
+    "ld.shared.u32 " E ", [u+" OFF "];\n\t"                     \
+    EP_S_FQ(E)                                                  \
+    "and.b32 bias, " E ", 0x7FF;\n\t"                           \
+    "mad.lo.u32 %0, f, q, bias;\n\t"                            \
+    "setp.lt.u32 p, %0, 32768;\n\t"                             \
+    "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"              \
+    EP_S_FETCH
 
 #define EP_S_PAIR(P, XA, XB, WA, WB)                            \
     "mov.b64 " P ", {" XA ", " XB "};\n\t"                      \
@@ -612,8 +636,8 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
         : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(col), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
           "+&r"(left), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                          \
-        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),            \
-          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max)                                                             \
+        : "r"(lt_asm), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),        \
+          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max), "r"(mul_f), "r"(mul_q)                                     \
         : "memory")
 
 // One full tile (exactly V vectors) of a tensor whose rows hold at least 32 blocks: the full groups in
@@ -653,6 +677,12 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
     uint32_t left = nv >> 5;
     const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
+#ifdef EP_X_INCL
+    const uint32_t lt_asm = lt | (1u << lane);
+#else
+    const uint32_t lt_asm = lt;
+#endif
+    const uint32_t mul_f = 4096u, mul_q = 1u << (32u - b);   // multiply-high forms of >> 20 and >> b
     if (left) {
         if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
         else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
@@ -711,6 +741,147 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
     // a ragged last tile belongs to warp 0 of one CTA chosen by the host (an extra CTA when the GPU has room for it)
     if (J.n_full < J.n_tiles && cta == J.last_cta && warp == 0)
         decode_tile<DT, false, false>(J, J.n_tiles - 1u, lut_addr, ring, lane);
+}
+
+// ======================================================================================================
+// Large-table path: b >= 12 or a coordinate range above 512.  The seventeen tables (2^b slots of 8 bytes:
+// {f | (u - F) << 16, value}) are built into caller-provided scratch by one launch and read through L1/L2
+// by the decode launch that follows on the same stream.  Same tile / lane / word order as above; payload
+// words are read straight from global memory with the index clamped to the payload.
+// ======================================================================================================
+
+struct GJobParams {
+    const uint8_t *stream;
+    const uint32_t *tile_index;
+    const float *scales;
+    void *out;
+    uint2 *lut;                   // scratch: 17 << b entries
+    uint32_t off_tables;          // byte offset of the table section (directory, then frequencies)
+    uint32_t off_payload;
+    uint32_t total_words;
+    uint32_t n_vec;
+    uint32_t per_row;
+    uint32_t V, n_tiles, b;
+    uint32_t cta_begin, cta_count;
+};
+
+struct GBatchParams {
+    GJobParams job[EP_MAX_BATCH];
+    int32_t n_jobs;
+};
+
+constexpr int kGThreads = 256;
+constexpr int kGWarps = kGThreads / 32;
+
+// one CTA per (table, job): exclusive prefix sums of the frequencies in shared memory (as u16; the last
+// entry 2^b <= 32768 still fits), then every slot finds its symbol by binary search
+__global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_constant__ GBatchParams P) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    __shared__ uint32_t part[1024];
+    const GJobParams &J = P.job[blockIdx.y];
+    const uint32_t t = blockIdx.x, tid = threadIdx.x;
+    const uint8_t *dir = J.stream + J.off_tables;
+    const int32_t tmin = reinterpret_cast<const int32_t *>(dir)[t];
+    const uint32_t *Ks = reinterpret_cast<const uint32_t *>(dir) + EP_NUM_TABLES;
+    const uint32_t K = Ks[t];
+    if (K == 0) return;
+    uint32_t before = 0;
+    for (uint32_t i = 0; i < t; ++i) before += Ks[i];
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(dir + 8 * EP_NUM_TABLES) + before;
+    uint16_t *F = reinterpret_cast<uint16_t *>(smem);              // K + 1 entries
+    const uint32_t per = (K + blockDim.x - 1) / blockDim.x;
+    const uint32_t j0 = min(tid * per, K), j1 = min(j0 + per, K);
+    uint32_t sum = 0;
+    for (uint32_t j = j0; j < j1; ++j) sum += fq[j];
+    part[tid] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (uint32_t i = 0; i < blockDim.x; ++i) { const uint32_t v = part[i]; part[i] = run; run += v; }
+        F[K] = uint16_t(run);                                        // = 2^b for a valid stream
+    }
+    __syncthreads();
+    uint32_t run = part[tid];
+    for (uint32_t j = j0; j < j1; ++j) { F[j] = uint16_t(run); run += fq[j]; }
+    __syncthreads();
+    const uint32_t M = 1u << J.b;
+    uint2 *lut = J.lut + (size_t(t) << J.b);
+    for (uint32_t u = tid; u < M; u += blockDim.x) {
+        uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u; F[K] = 2^b > u
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
+        }
+        const uint32_t f = uint32_t(F[lo + 1]) - uint32_t(F[lo]);
+        lut[u] = make_uint2(f | ((u - uint32_t(F[lo])) << 16), uint32_t(tmin + int32_t(lo)));
+    }
+}
+
+__device__ __forceinline__ int32_t grans_step(uint32_t &x, const uint2 *table, uint32_t mask, uint32_t b, uint32_t &ptr,
+                                              const uint16_t *pay, uint32_t lt, bool act, uint32_t last_word) {
+    int32_t value = 0;
+    bool need = false;
+    if (act) {
+        const uint2 e = __ldg(table + (x & mask));
+        x = (e.x & 0xFFFFu) * (x >> b) + (e.x >> 16);
+        value = int32_t(e.y);
+        need = x < ep::kStateLow;
+    }
+    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, need);
+    if (need) x = (x << 16) | __ldg(pay + min(ptr + __popc(bal & lt), last_word));
+    ptr += __popc(bal);
+    return value;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_constant__ GBatchParams P) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    int j = 0;
+    while (j + 1 < P.n_jobs && blockIdx.x >= P.job[j + 1].cta_begin) ++j;
+    const GJobParams &J = P.job[j];
+    const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
+    const uint16_t *pay = reinterpret_cast<const uint16_t *>(J.stream + J.off_payload);
+    const uint32_t last_word = J.total_words ? J.total_words - 1u : 0u;
+    const uint32_t cta = blockIdx.x - J.cta_begin;
+    for (uint32_t tile = cta * kGWarps + warp; tile < J.n_tiles; tile += J.cta_count * kGWarps) {
+        const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
+        uint32_t x = rec[lane];
+        uint32_t ptr = rec[32];
+        const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
+        const uint32_t v0 = tile * J.V;
+        const uint32_t nv = min(J.V, J.n_vec - v0);
+        for (uint32_t g = 0; g * 32u < nv; ++g) {
+            const uint32_t i = g * 32u + lane;
+            const bool act = i < nv;
+            int32_t fld[9];
+            fld[0] = grans_step(x, J.lut, mask, b, ptr, pay, lt, act, last_word);
+            const uint2 *tabs = J.lut + (size_t(1 + 8 * (fld[0] & 1)) << b);
+#pragma unroll
+            for (int k = 1; k <= 8; ++k)
+                fld[k] = grans_step(x, tabs + (size_t(k - 1) << b), mask, b, ptr, pay, lt, act, last_word);
+            if (!act) continue;
+            const uint32_t v = v0 + i;
+            if constexpr (DT == EP_FIELDS_I32) {
+                int32_t *o = static_cast<int32_t *>(J.out) + size_t(v) * 9u;
+#pragma unroll
+                for (int k = 0; k < 9; ++k) o[k] = fld[k];
+            } else {
+                // Eq. 5 on doubled coordinates q = 2p (integers), then p = q/2 exactly and Eq. 19
+                const float sigma = __ldg(J.scales + v / J.per_row);
+                int32_t s7 = 0;
+                float w[8];
+#pragma unroll
+                for (int k = 1; k <= 7; ++k) {
+                    s7 += fld[k];
+                    w[k - 1] = __fmul_rn(sigma, float(2 * fld[k] + fld[0]) * 0.5f);
+                }
+                w[7] = __fmul_rn(sigma, float(2 * (2 * fld[8] + (s7 & 1)) + fld[0]) * 0.5f);
+                Out<DT>::store(static_cast<uint8_t *>(J.out) + size_t(v) * Out<DT>::kBlockBytes, w);
+            }
+        }
+        const bool bad = (x != ep::kStateLow) || (ptr != end);
+        if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
+    }
 }
 
 // ---- host side -----------------------------------------------------------------------------------
@@ -783,17 +954,84 @@ extern "C" size_t ep_decode_scratch_bytes(const ep_info *info) {
     return size_t(EP_NUM_TABLES) * (size_t(1) << info->b) * 8u;
 }
 
-extern "C" int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream) {
-    if (!jobs || n_jobs <= 0 || n_jobs > EP_MAX_BATCH) return EP_ERR_BAD_ARG;
-    const int sms = num_sms();
-    if (sms <= 0) return EP_ERR_CUDA;
-    BatchParams P;
+namespace {
+
+template <int DT>
+cudaError_t launch_glut(const GBatchParams &P, uint32_t grid, cudaStream_t st) {
+    ep_decode_glut_kernel<DT><<<grid, kGThreads, 0, st>>>(P);
+    return cudaGetLastError();
+}
+
+// jobs whose tables do not fit shared memory: build the tables into scratch, then decode from them
+int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt, int sms, cudaStream_t st) {
+    GBatchParams P;
     std::memset(&P, 0, sizeof(P));
     P.n_jobs = n_jobs;
-    const int32_t dt = jobs[0].out_dtype;
-    uint64_t tiles_total = 0;
+    uint32_t next = 0, max_K = 1;
     for (int i = 0; i < n_jobs; ++i) {
-        const ep_decode_job &jb = jobs[i];
+        const ep_decode_job &jb = *jobs[i];
+        const ep_info &I = *jb.info;
+        const size_t need = size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 8u;
+        if (!jb.d_scratch || jb.scratch_bytes < need || (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255)) return EP_ERR_SCRATCH;
+        for (int t = 0; t < EP_NUM_TABLES; ++t) {
+            if (I.table_K[t] > 65535u) return EP_ERR_UNSUPPORTED;
+            if (I.table_K[t] > max_K) max_K = I.table_K[t];
+        }
+        GJobParams &J = P.job[i];
+        J.stream = static_cast<const uint8_t *>(jb.d_stream);
+        J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
+        J.scales = jb.d_row_scales;
+        J.out = jb.d_out;
+        J.lut = static_cast<uint2 *>(jb.d_scratch);
+        J.off_tables = I.off_tables;
+        J.off_payload = I.off_payload;
+        J.total_words = uint32_t(I.total_words);
+        J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
+        J.per_row = I.C / 8;
+        J.V = I.V;
+        J.n_tiles = I.n_tiles;
+        J.b = I.b;
+        const uint64_t want = (uint64_t(I.n_tiles) + kGWarps - 1) / kGWarps;
+        const uint64_t cap = uint64_t(sms) * 8u;
+        J.cta_begin = next;
+        J.cta_count = uint32_t(want < cap ? want : cap);
+        next += J.cta_count;
+    }
+    const size_t smem = 2u * (size_t(max_K) + 1u);
+    if (smem > 48u * 1024u) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
+        if (cudaFuncSetAttribute(ep_build_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+            return EP_ERR_CUDA;
+    }
+    ep_build_tables_kernel<<<dim3(EP_NUM_TABLES, n_jobs), 1024, smem, st>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return EP_ERR_CUDA;
+    cudaError_t e;
+    switch (dt) {
+    case EP_BF16: e = launch_glut<EP_BF16>(P, next, st); break;
+    case EP_FP16: e = launch_glut<EP_FP16>(P, next, st); break;
+    case EP_FP8_E4M3: e = launch_glut<EP_FP8_E4M3>(P, next, st); break;
+    case EP_INT8: e = launch_glut<EP_INT8>(P, next, st); break;
+    case EP_FIELDS_I32: e = launch_glut<EP_FIELDS_I32>(P, next, st); break;
+    default: return EP_ERR_BAD_ARG;
+    }
+    return e == cudaSuccess ? EP_OK : EP_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void *stream) {
+    if (!jobs_in || n_in <= 0 || n_in > EP_MAX_BATCH) return EP_ERR_BAD_ARG;
+    const int sms = num_sms();
+    if (sms <= 0) return EP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int32_t dt = jobs_in[0].out_dtype;
+    if (dt != EP_BF16 && dt != EP_FP16 && dt != EP_FP8_E4M3 && dt != EP_INT8 && dt != EP_FIELDS_I32) return EP_ERR_BAD_ARG;
+    const ep_decode_job *fast[EP_MAX_BATCH], *large[EP_MAX_BATCH];
+    int n_jobs = 0, n_large = 0;
+    uint64_t tiles_total = 0;
+    for (int i = 0; i < n_in; ++i) {
+        const ep_decode_job &jb = jobs_in[i];
         if (!jb.info || !jb.d_stream || !jb.d_tile_index || !jb.d_out) return EP_ERR_BAD_ARG;
         if (jb.out_dtype != dt) return EP_ERR_BAD_ARG;   // one output type per launch
         if (dt != EP_FIELDS_I32 && !jb.d_row_scales) return EP_ERR_BAD_ARG;
@@ -803,15 +1041,25 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *
             (reinterpret_cast<uintptr_t>(jb.d_out) & 15))
             return EP_ERR_BAD_ARG;
         if (I.table_K[0] == 0 || I.table_min[0] < 0 || int64_t(I.table_min[0]) + I.table_K[0] > 2) return EP_ERR_BAD_STREAM;
-        if (!fits_smem_tables(I)) return EP_ERR_UNSUPPORTED;
-        tiles_total += I.n_tiles;
+        // 32-bit byte offsets into the output and a signed 32-bit payload remainder in the kernels
+        if (uint64_t(I.R) * I.C * 4u >= (1ull << 32) || I.total_words >= (1ull << 30)) return EP_ERR_UNSUPPORTED;
+        if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; tiles_total += I.n_tiles; }
+        else large[n_large++] = &jb;
     }
+    if (n_large) {
+        const int rc = decode_large_tables(large, n_large, dt, sms, st);
+        if (rc) return rc;
+    }
+    if (n_jobs == 0) return EP_OK;
+    BatchParams P;
+    std::memset(&P, 0, sizeof(P));
+    P.n_jobs = n_jobs;
     // persistent CTAs: a single tensor gets one CTA per SM (or fewer if it has under 32 tiles per SM);
     // a batch shares twice the SM count in proportion to the tensors' tile counts
     const uint64_t budget = n_jobs == 1 ? uint64_t(sms) : 2ull * sms;
     uint32_t next = 0;
     for (int i = 0; i < n_jobs; ++i) {
-        const ep_decode_job &jb = jobs[i];
+        const ep_decode_job &jb = *fast[i];
         const ep_info &I = *jb.info;
         JobParams &J = P.job[i];
         const uint64_t want = (uint64_t(I.n_tiles) + kWarps - 1) / kWarps;
@@ -855,7 +1103,6 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *
         }
         next += uint32_t(share) + extra;
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     switch (dt) {
     case EP_BF16: e = launch_smem<EP_BF16>(P, next, st); break;

@@ -512,7 +512,11 @@ extern "C" int ep_encode(const float *W, uint32_t R, uint32_t C, double target_b
             }
             last = {log_s, est, true};
             const float before = s;
-            s = float(std::exp2(log_s + (est - target_bpp) / per_doubling));
+            double moved = std::exp2(log_s + (est - target_bpp) / per_doubling);
+            if (!(moved >= o.bracket_lo)) moved = o.bracket_lo;   // never leave the search bracket
+            if (moved > o.bracket_hi) moved = o.bracket_hi;
+            s = float(moved);
+            if (s == before) break;
             quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
             Model m;
             m.count(fields.data(), nvec, threads);

@@ -134,6 +134,56 @@ def test_decode_argument_checks():
         ep.decode_tensor(d.info, 0, d.d_tile_index, d.d_row_scales, ep.BF16, out.data_ptr())
 
 
+# ---- streams whose lookup tables do not fit shared memory (b >= 12 or coordinate range > 512) -----
+
+def test_large_table_path_high_precision_and_high_rate():
+    W = synth.laplace_rows(96, 1024, 77)
+    for kw, bpp in ((dict(b_start=12), 4.0), (dict(), 8.0), (dict(b_start=15, tile_vectors=100), 5.0),
+                    (dict(b_start=13, tile_vectors=33), 3.0)):
+        blob = ep.encode(W, bpp, **kw)
+        assert blob.info.b >= 12 and ep.decode_scratch_bytes(blob.info) == 17 * 8 << blob.info.b
+        _check_all_types(blob.data)
+        if "tile_vectors" not in kw:          # tiny tiles are metadata-bound: no rate claim there
+            assert abs(blob.stored_bpp - bpp) < 0.02 * bpp
+    # oracle stream, paper's 8 bpp defaults (b = 12, 4096-symbol tiles)
+    ora, rep = oracle.encode(synth.gaussian_rows(64, 2048, 5), 8.0)
+    assert rep["b"] == 12 and rep["V"] == 455
+    _check_all_types(ora)
+
+
+def test_large_table_path_wide_coordinate_range():
+    # b = 11 but coordinates spread over more than 512 values: a few huge outliers
+    rng = np.random.default_rng(3)
+    n = 6 * 64
+    fields = np.zeros((n, 9), np.int32)
+    fields[:, 0] = rng.integers(0, 2, n)
+    fields[:, 1:] = np.rint(rng.standard_normal((n, 8)) * 4).astype(np.int32)
+    fields[5, 3] = 700
+    fields[77, 8] = -400
+    fields[100, 1] = -3000
+    blob = ep.pack_fields(fields, 6, 512, 11, 50, np.linspace(0.01, 0.02, 6).astype(np.float32))
+    assert ep.decode_scratch_bytes(blob.info) > 0
+    _check_all_types(blob.data)
+
+
+def test_large_table_path_needs_scratch_and_mixes_in_a_batch():
+    W = synth.gaussian_rows(64, 512, 8)
+    big = ep.encode(W, 4.0, b_start=12)
+    small = ep.encode(W, 4.0)
+    d_big, d_small = ep.upload(big), ep.upload(small)
+    out = torch.empty((64, 512), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ep.EntroPackError) as ei:
+        ep.decode_tensor(d_big.info, d_big.d_stream, d_big.d_tile_index, d_big.d_row_scales, ep.BF16, out.data_ptr())
+    assert ei.value.status == -7
+    outs = [torch.empty((64, 512), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    ep.decode_many([d_small, d_big, d_small], ep.BF16, outs)
+    torch.cuda.synchronize()
+    for b, o in zip((small, big, small), outs):
+        ref, _ = oracle.decode(b.data, oracle.BF16)
+        assert np.array_equal(_bits(o), ref)
+    assert ep.last_device_status() == 0
+
+
 # ---- full-size configurations, in the launch configuration the bench times -----------------------
 
 def _full_compare(W, bpp, dt, V=0):
@@ -152,10 +202,11 @@ def test_config2_full_size():
     _full_compare(synth.config2(), 3.0, ep.BF16)
 
 
-def test_config4_full_size_two_rates():
+def test_config4_full_size_three_rates():
     W = synth.config4()
     _full_compare(W, 4.0, ep.FP16)
     _full_compare(W, 2.0, ep.FP16)
+    _full_compare(W, 6.0, ep.FP16)
 
 
 def test_config3_one_wide_tensor_fp8_and_int8_containers():
