@@ -56,7 +56,8 @@ typedef enum {
     EP_ERR_CUDA = -4,        /* a CUDA runtime call failed */
     EP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out */
     EP_ERR_NOMEM = -6,       /* host allocation failed */
-    EP_ERR_SCRATCH = -7      /* scratch buffer missing, misaligned or too small */
+    EP_ERR_SCRATCH = -7,     /* scratch buffer missing, misaligned or too small */
+    EP_ERR_STATIC_LIMIT = -8 /* ep_decode_tensor_static: the stream's tables exceed the built-in area */
 } ep_status;
 
 /* Output element types of the decoder: snap_tau of Eq. 19. */
@@ -175,6 +176,28 @@ int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_ti
 /* The same for up to EP_MAX_BATCH tensors in one kernel launch (independent tiles of all tensors
  * share the grid).  Jobs needing scratch get their lookup tables built by one extra launch first. */
 int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
+
+/* Largest probability precision b served by ep_decode_tensor_static: its built-in table area holds
+ * 17 tables of 2^13 eight-byte entries = 1 114 112 bytes of device memory per GPU that loads the library. */
+#define EP_STATIC_MAX_B 13
+
+/* (No counterpart in the paper: an integration aid of this library.)
+ * Same decode as ep_decode_tensor, for callers that cannot hand over a scratch buffer because they
+ * cannot allocate device memory at the point of the call: code running inside a host framework that owns
+ * the allocator and passes in nothing but input and output buffers, or a serving loop in which a
+ * cudaMalloc would stall the whole device.  Streams whose lookup tables do not fit shared memory
+ * normally need ep_decode_scratch_bytes() of caller memory; here the tables are built in a fixed area
+ * compiled into the library instead.  The call itself allocates and frees nothing.
+ *   - Limit: b <= EP_STATIC_MAX_B.  A stream with larger b is refused with EP_ERR_STATIC_LIMIT (use
+ *     ep_decode_tensor with your own scratch for those).  Streams that need no scratch are decoded
+ *     exactly as by ep_decode_tensor.
+ *   - The first call on each device looks up the device address of the built-in area (the device must be
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one area and it keeps whatever the previous call left there; each
+ *     call rewrites every table it reads, so nothing has to be cleared, but two calls whose kernels
+ *     overlap on the GPU (different streams, no ordering between them) race on it.  Serialise them. */
+int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                            const float *d_row_scales, int32_t out_dtype, void *d_out, void *stream);
 
 /* Device-side integrity word.  The kernel ORs in a flag when a tile does not end with every state
  * at 2^15 and its word pointer at the next tile's offset (a damaged stream).  This call

@@ -91,6 +91,8 @@ def load():
     L.ep_decode_scratch_bytes.argtypes = [C.POINTER(Info)]
     L.ep_decode_tensor.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ep_decode_tensor_static.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                          C.c_void_p]
     L.ep_decode_batch.argtypes = [C.POINTER(DecodeJob), C.c_int32, C.c_void_p]
     L.ep_last_device_status.argtypes = [C.c_void_p]
     L.ep_strerror.restype = C.c_char_p
@@ -198,6 +200,14 @@ def decode_tensor(info: Info, d_stream: int, d_tile_index: int, d_row_scales: in
     """ep_decode_tensor with raw device addresses (ints)."""
     _check(load().ep_decode_tensor(C.byref(info), d_stream, d_tile_index, d_row_scales, out_dtype, d_out,
                                    d_scratch or None, scratch_bytes, stream or None), "ep_decode_tensor")
+
+
+def decode_tensor_static(info: Info, d_stream: int, d_tile_index: int, d_row_scales: int, out_dtype: int, d_out: int,
+                         stream: int = 0) -> None:
+    """ep_decode_tensor_static: the same decode for callers that cannot allocate a scratch buffer; large lookup
+    tables go to a fixed area inside the library (b <= 13).  Calls sharing a device must not overlap."""
+    _check(load().ep_decode_tensor_static(C.byref(info), d_stream, d_tile_index, d_row_scales, out_dtype, d_out,
+                                          stream or None), "ep_decode_tensor_static")
 
 
 def decode_batch(jobs: list[DecodeJob], stream: int = 0) -> None:

@@ -1138,3 +1138,46 @@ extern "C" int ep_last_device_status(void *stream) {
     if (v && cudaMemcpyToSymbol(g_ep_status, &zero, sizeof(zero)) != cudaSuccess) return EP_ERR_CUDA;
     return v ? EP_ERR_BAD_STREAM : EP_OK;
 }
+
+// ---- decode without a caller-provided scratch buffer ----------------------------------------------------
+// For callers that cannot allocate device memory when they need to decode (they were given input and
+// output buffers by a framework that owns the allocator, or an allocation would stall the device in the
+// middle of serving).  The large-table path then builds its tables in this fixed area instead of in
+// caller scratch.  One area per device, shared by every call: calls that overlap on the GPU race on it.
+namespace {
+
+constexpr size_t kStaticTableBytes = size_t(EP_NUM_TABLES) * (size_t(1) << EP_STATIC_MAX_B) * 8u;   // 1 114 112
+static __device__ __align__(256) unsigned char g_ep_static_tables[kStaticTableBytes];
+
+// In host code `g_ep_static_tables` is only a handle for the runtime, not an address a kernel could use:
+// the device address is asked for once per device, with that device current.
+void *g_static_tables_addr[64] = {};
+
+int static_tables_address(void **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return EP_ERR_UNSUPPORTED;
+    if (!g_static_tables_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_ep_static_tables) != cudaSuccess || !p) return EP_ERR_CUDA;
+        g_static_tables_addr[dev] = p;
+    }
+    *out = g_static_tables_addr[dev];
+    return EP_OK;
+}
+
+}  // namespace
+
+extern "C" int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                                       const float *d_row_scales, int32_t out_dtype, void *d_out, void *stream) {
+    if (!info) return EP_ERR_BAD_ARG;
+    void *tables = nullptr;
+    size_t bytes = 0;
+    if (ep_decode_scratch_bytes(info) != 0) {
+        if (info->b > EP_STATIC_MAX_B) return EP_ERR_STATIC_LIMIT;   // tables of 2^b slots would not fit the built-in area
+        const int rc = static_tables_address(&tables);
+        if (rc) return rc;
+        bytes = kStaticTableBytes;
+    }
+    return ep_decode_tensor(info, d_stream, d_tile_index, d_row_scales, out_dtype, d_out, tables, bytes, stream);
+}

@@ -107,6 +107,7 @@ extern "C" const char *ep_strerror(int status) {
     case EP_ERR_TIMEOUT: return "device-side wait timed out";
     case EP_ERR_NOMEM: return "out of host memory";
     case EP_ERR_SCRATCH: return "scratch buffer missing, misaligned or too small";
+    case EP_ERR_STATIC_LIMIT: return "stream needs lookup tables larger than the built-in area (b above EP_STATIC_MAX_B)";
     default: return "unknown status";
     }
 }
