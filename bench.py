@@ -43,7 +43,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--bpp", type=float, default=None, help="target bits/param (default: the workload's)")
-    ap.add_argument("--tile-vectors", type=int, default=0, help="V; 0 = the paper's default for the target rate")
+    ap.add_argument("--tile-vectors", type=int, default=-1,
+                    help="V; 0 = the paper's default for the target rate; -1 (default) = ep_suggest_tile_vectors: "
+                         "the largest V up to the paper's default that fills whole rounds of the GPU's tile slots")
     ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp8", "int8"])
     ap.add_argument("--layers", type=int, default=48, help="c5: resident layers")
     ap.add_argument("--distinct-layers", type=int, default=2, help="c5: distinct layers actually encoded")
@@ -84,9 +86,14 @@ def make_workload(args):
     raise ValueError(w)
 
 
-def encode_layers(layers, bpp, V):
+def pick_tile_vectors(V, shape, bpp, slots):
     import paper_2609_34185_b200 as ep
-    return [[ep.encode(W, bpp, tile_vectors=V) for W in mats] for mats in layers]
+    return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots) if V < 0 else V
+
+
+def encode_layers(layers, bpp, V, slots):
+    import paper_2609_34185_b200 as ep
+    return [[ep.encode(W, bpp, tile_vectors=pick_tile_vectors(V, W.shape, bpp, slots)) for W in mats] for mats in layers]
 
 
 # ---- clocks ------------------------------------------------------------------------------------------
@@ -188,7 +195,7 @@ def run_reference(args):
     name, dtype_name, bpp, layers = make_workload(args)
     V = args.tile_vectors
     import paper_2609_34185_b200 as ep
-    blob = ep.encode(layers[0][0], bpp, tile_vectors=V)
+    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 32))
     I = blob.info
     # each step decodes a leading tile range (repeated if short) sized so that the whole run stays near a minute
     params, tiles, reps, threads = oracle_sample(blob, dtype_name, min(0.5, 60.0 / max(1, args.steps + args.warmup)))
@@ -238,7 +245,10 @@ def main():
     esize = ep.DTYPE_BYTES[DT]
 
     # every rank decodes its own replica of the workload: tiles and tensors are independent, no collective
-    blobs = encode_layers(layers, bpp, args.tile_vectors)
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    # a single tensor gets one 32-warp CTA per SM
+    slots = 32 * n_sms if sum(len(m) for m in layers) == len(layers) else 0   # batches keep the paper's tile size
+    blobs = encode_layers(layers, bpp, args.tile_vectors, slots)
     n_layers = args.layers if args.workload == "c5" else len(blobs)
     resident = [[ep.upload(b, device=dev) for b in blobs[l % len(blobs)]] for l in range(n_layers)]
     layer_params = [sum(b.info.R * b.info.C for b in blobs[l % len(blobs)]) for l in range(n_layers)]

@@ -208,6 +208,15 @@ int ep_last_device_status(void *stream);
 /* ---- misc --------------------------------------------------------------------------------- */
 const char *ep_strerror(int status);
 uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile-size defaults */
+
+/* Tile size for a decoder with `decode_slots` concurrent tile slots (32 per SM for this library: 4736 on
+ * a 148-SM B200): the largest V not above the paper's default for the target rate for which the tensor's
+ * R*C/8 blocks split into a whole number of rounds of decode_slots tiles (the last round nearly full),
+ * rounded up to a multiple of 32 vectors when that stays within the default.
+ * Larger tiles amortise the 132 bytes of per-tile metadata, but a tensor with fewer tiles than slots
+ * leaves SMs idle (App. "Tile layout and storage": tile size trades storage against parallelism).
+ * Never below a quarter of the default (small tensors); returns the default when decode_slots is 0. */
+uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint32_t decode_slots);
 int ep_version(void);
 
 #ifdef __cplusplus

@@ -99,6 +99,8 @@ def load():
     L.ep_strerror.argtypes = [C.c_int]
     L.ep_default_tile_vectors.restype = C.c_uint32
     L.ep_default_tile_vectors.argtypes = [C.c_double]
+    L.ep_suggest_tile_vectors.restype = C.c_uint32
+    L.ep_suggest_tile_vectors.argtypes = [C.c_uint32, C.c_uint32, C.c_double, C.c_uint32]
     L.ep_encode_opts_default.argtypes = [C.POINTER(EncodeOpts)]
     L.ep_encode_opts_default.restype = None
     _lib = L
@@ -119,6 +121,11 @@ def _check(rc: int, what: str):
 
 def default_tile_vectors(target_bpp: float) -> int:
     return load().ep_default_tile_vectors(float(target_bpp))
+
+
+def suggest_tile_vectors(R: int, Cc: int, target_bpp: float, decode_slots: int = 148 * 32) -> int:
+    """ep_suggest_tile_vectors: tile size that fills whole rounds of `decode_slots` concurrent tiles."""
+    return load().ep_suggest_tile_vectors(R, Cc, float(target_bpp), decode_slots)
 
 
 class Blob:

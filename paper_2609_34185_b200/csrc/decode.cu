@@ -57,9 +57,7 @@ struct JobParams {
     uint32_t V, n_tiles, b;
     int32_t zlo;                  // even, <= -2
     uint32_t cta_begin, cta_count;
-    uint32_t n_full;              // tiles holding exactly V vectors (all but a ragged last one)
-    uint32_t iters;               // ceil(n_full / (cta_count * warps)): every warp runs this many rounds
-    uint32_t last_cta;            // CTA (relative to cta_begin) whose warp 0 decodes a ragged last tile
+    uint32_t iters;               // ceil(n_tiles / (cta_count * warps)): every warp runs this many rounds
     int16_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint16_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
@@ -359,10 +357,8 @@ __device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_
     threshold = 512u * (cur + 1u);
 }
 
-// WIDE: rows hold at least 32 vectors, so a group advances the row index by at most one.
-// FULL: the tile holds exactly V vectors, so every loop bound is a kernel parameter.  The compiler then
-// sees warp-uniform control flow throughout the hot loop and emits no divergence handling around the
-// warp votes; a ragged last tile takes the same code with data-dependent bounds.
+// Plain C++ version of the tile loop, used for the field-dump mode and for tensors with fewer than 32
+// blocks per row (WIDE = false: a group may then cross several rows).
 template <int DT, bool WIDE, bool FULL>
 __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
@@ -535,6 +531,9 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         ".reg .f32 w0, w1, w2, w3, w4, w5, w6, w7;\n\t"                                                               \
         ".reg .b64 kk, ss, p0, p1, p2, p3, ad, src;\n\t"                                                              \
         "setp.lt.u32 plow, %22, 128;\n\t"                                                                             \
+        "setp.eq.u32 pl, %8, 0;\n\t"                                                                                  \
+        "vote.sync.all.pred pl, pl, 0xffffffff;\n\t"                                                                  \
+        "@pl bra.uni EP_DONE;\n\t"                                                                                    \
         "EP_LOOP:\n\t"                                                                                                \
         "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
         "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
@@ -583,6 +582,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "EP_ROWDONE:\n\t"                                                                                             \
         "sub.u32 %8, %8, 1;\n\t"                                                                                      \
         "setp.ne.u32 pl, %8, 0;\n\t"                                                                                  \
+        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */        \
         "@pl bra.uni EP_LOOP;\n\t"                                                                                    \
         "bra.uni EP_DONE;\n\t"                                                                                        \
         /* ---- some lane moved to the next row: reload its scale ---- */                                             \
@@ -640,17 +640,19 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
           "l"(scales), "l"(a0), "r"(lane16), "r"(row_max), "r"(mul_f), "r"(mul_q)                                     \
         : "memory")
 
-// One full tile (exactly V vectors) of a tensor whose rows hold at least 32 blocks: the full groups in
-// PTX, a last partial group (V not a multiple of 32) through decode_group.
+// One tile of a tensor whose rows hold at least 32 blocks: the full groups in PTX, a last partial group
+// through decode_group.  `valid` is false for a warp whose slot lies past the last tile (`tile` is then
+// the last tile, only so that addresses stay inside the stream): it does no group at all.  The number of
+// groups is data here, not control flow the compiler reasons about: every branch on it is a bra.uni.
 template <int DT>
-__device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring,
-                                                 uint32_t lane) {
+__device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t tile, bool valid, uint32_t lut_addr,
+                                                 uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
     uint32_t x = rec[lane];
     const uint32_t off = rec[32];
     const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
     const uint32_t v0 = tile * J.V;
-    const uint32_t nv = J.V;
+    const uint32_t nv = valid ? min(J.V, J.n_vec - v0) : 0u;
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
     const uint32_t per_row = J.per_row;
     const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
@@ -675,7 +677,9 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     uint32_t sig = __float_as_uint(__ldg(scales + row));
     uint32_t doff = v * Out<DT>::kBlockBytes;
     const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
-    uint32_t left = nv >> 5;
+    // The group count is the same in all lanes but comes from loaded data, which the compiler treats as possibly
+    // different per lane; the loop therefore branches on warp votes of it (see the asm), never on the value itself.
+    uint32_t left = nv >> 5;                           // may be 0: the asm then falls straight through
     const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
 #ifdef EP_X_INCL
     const uint32_t lt_asm = lt | (1u << lane);
@@ -683,12 +687,10 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     const uint32_t lt_asm = lt;
 #endif
     const uint32_t mul_f = 4096u, mul_q = 1u << (32u - b);   // multiply-high forms of >> 20 and >> b
-    if (left) {
-        if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
-        else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
-        else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
-        else EP_FULL_GROUPS_ASM(EP_S_STORE_INT8, 256);
-    }
+    if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
+    else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
+    else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
+    else EP_FULL_GROUPS_ASM(EP_S_STORE_INT8, 256);
     uint32_t pos = wa - wbase;
     if (nv & 31u) {
         uint32_t threshold = wthr - wbase;
@@ -703,7 +705,7 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     }
     cp_async_wait<0>();
     __syncwarp();
-    const bool bad = (x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end);
+    const bool bad = valid && ((x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end));
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
 }
 
@@ -719,28 +721,26 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
     build_tables_smem(J, lut_addr, warp, lane);
     __syncthreads();
     const uint32_t cta = blockIdx.x - J.cta_begin;
-    // Rounds over the full tiles: warp w of CTA c takes tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and
-    // the test for a CTA past the end are functions of blockIdx and kernel parameters only, so control flow stays
-    // warp-uniform in the compiler's eyes; inside the one CTA that straddles the end, warps past it redo the last full
-    // tile (the same bytes are written twice) instead of branching around the hot loop.
+    // Rounds over the tiles: warp w of CTA c takes tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and the
+    // test for a CTA past the end depend on blockIdx and kernel parameters only, so the compiler sees warp-uniform
+    // control flow and puts no divergence guards around the warp votes of the hot loop; inside the one CTA that
+    // straddles the end, a warp past the last tile goes through the same code with zero groups to do.
     const bool wide = J.per_row >= 32u;
-    if (cta < J.cta_count) {
-        for (uint32_t i = 0; i < J.iters; ++i) {
-            const uint32_t base = (cta + i * J.cta_count) * kWarps;
-            if (base >= J.n_full) break;
-            const uint32_t tile = min(base + warp, J.n_full - 1u);
-            if constexpr (DT != EP_FIELDS_I32) {
-                if (wide) decode_tile_fast<DT>(J, tile, lut_addr, ring, lane);
-                else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
-            } else {
-                if (wide) decode_tile<DT, true, true>(J, tile, lut_addr, ring, lane);
-                else decode_tile<DT, false, true>(J, tile, lut_addr, ring, lane);
+    for (uint32_t i = 0; i < J.iters; ++i) {
+        const uint32_t base = (cta + i * J.cta_count) * kWarps;
+        if (base >= J.n_tiles) break;
+        const uint32_t tile = base + warp;
+        if constexpr (DT != EP_FIELDS_I32) {
+            if (wide && J.V < (1u << 20)) {
+                decode_tile_fast<DT>(J, min(tile, J.n_tiles - 1u), tile < J.n_tiles, lut_addr, ring, lane);
+                continue;
             }
         }
+        if (tile < J.n_tiles) {
+            if (wide) decode_tile<DT, true, false>(J, tile, lut_addr, ring, lane);
+            else decode_tile<DT, false, false>(J, tile, lut_addr, ring, lane);
+        }
     }
-    // a ragged last tile belongs to warp 0 of one CTA chosen by the host (an extra CTA when the GPU has room for it)
-    if (J.n_full < J.n_tiles && cta == J.last_cta && warp == 0)
-        decode_tile<DT, false, false>(J, J.n_tiles - 1u, lut_addr, ring, lane);
 }
 
 // ======================================================================================================
@@ -1081,19 +1081,8 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.zlo = int32_t(even_base(coord_range(I)));
         J.cta_begin = next;
         J.cta_count = uint32_t(share);
-        const bool ragged = (uint64_t(J.n_vec) % I.V) != 0;
-        J.n_full = ragged ? I.n_tiles - 1u : I.n_tiles;
         const uint32_t round_tiles = J.cta_count * uint32_t(kWarps);
-        J.iters = (J.n_full + round_tiles - 1u) / round_tiles;
-        J.last_cta = 0;
-        uint32_t extra = 0;
-        if (ragged) {
-            // CTAs [0, used) have work in the last round; prefer an extra CTA while the launch still fits the SMs,
-            // else the first CTA that is idle (or least loaded) in the last round
-            const uint32_t used = J.n_full ? ((J.n_full - (J.iters - 1u) * round_tiles) + uint32_t(kWarps) - 1u) / uint32_t(kWarps) : 0u;
-            if (uint64_t(next) + share < uint64_t(sms) && n_jobs == 1) { J.last_cta = J.cta_count; extra = 1; }
-            else J.last_cta = used % J.cta_count;
-        }
+        J.iters = (J.n_tiles + round_tiles - 1u) / round_tiles;
         uint32_t acc = 0;
         for (int t = 0; t < EP_NUM_TABLES; ++t) {
             J.tmin[t] = int16_t(I.table_min[t]);
@@ -1101,7 +1090,7 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
             J.foff[t] = uint16_t(acc);
             acc += I.table_K[t];
         }
-        next += uint32_t(share) + extra;
+        next += uint32_t(share);
     }
     cudaError_t e;
     switch (dt) {

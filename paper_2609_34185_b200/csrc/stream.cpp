@@ -119,4 +119,22 @@ extern "C" uint32_t ep_default_tile_vectors(double target_bpp) {
     return V < 32u ? 32u : V;
 }
 
+extern "C" uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint32_t decode_slots) {
+    const uint32_t vmax = ep_default_tile_vectors(target_bpp);
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    if (decode_slots == 0 || nvec == 0) return vmax;
+    // a small tensor cannot fill the decoder anyway: never let metadata grow beyond 4x the default's share
+    const uint64_t floor_v = vmax / 4 > 32 ? vmax / 4 : 32;
+    // fewest rounds whose tiles are not larger than the default; tile sizes are multiples of 32 vectors (whole
+    // groups of 32 rANS states, no partly filled last group) whenever that still fits
+    for (uint64_t rounds = 1;; ++rounds) {
+        const uint64_t tiles = rounds * decode_slots;
+        uint64_t V = (nvec + tiles - 1) / tiles;
+        if (V > vmax) continue;
+        const uint64_t V32 = (V + 31) & ~uint64_t(31);
+        if (V32 <= vmax) V = V32;
+        return uint32_t(V < floor_v ? floor_v : V);
+    }
+}
+
 extern "C" int ep_version(void) { return 1; }
