@@ -87,8 +87,15 @@ def make_workload(args):
 
 
 def pick_tile_vectors(V, shape, bpp, slots):
+    """V < 0: single tensors get ep_suggest_tile_vectors for the GPU's tile slots; tensors of a batch (slots == 0)
+    share the grid, there the paper's default is kept but capped at its 4 bpp value (1820 vectors): the 3640-vector
+    default of the lowest rates leaves too few tiles per tensor to balance a batch."""
     import paper_2609_34185_b200 as ep
-    return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots) if V < 0 else V
+    if V >= 0:
+        return V
+    if slots:
+        return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots)
+    return min(ep.default_tile_vectors(bpp), 1820)
 
 
 def encode_layers(layers, bpp, V, slots):
@@ -247,7 +254,8 @@ def main():
     # every rank decodes its own replica of the workload: tiles and tensors are independent, no collective
     n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
     # a single tensor gets one 32-warp CTA per SM
-    slots = 32 * n_sms if sum(len(m) for m in layers) == len(layers) else 0   # batches keep the paper's tile size
+    single = sum(len(m) for m in layers) == len(layers)
+    slots = 32 * n_sms if single else 0
     blobs = encode_layers(layers, bpp, args.tile_vectors, slots)
     n_layers = args.layers if args.workload == "c5" else len(blobs)
     resident = [[ep.upload(b, device=dev) for b in blobs[l % len(blobs)]] for l in range(n_layers)]

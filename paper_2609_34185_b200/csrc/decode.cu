@@ -359,14 +359,14 @@ __device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_
 
 // Plain C++ version of the tile loop, used for the field-dump mode and for tensors with fewer than 32
 // blocks per row (WIDE = false: a group may then cross several rows).
-template <int DT, bool WIDE, bool FULL>
+template <int DT, bool WIDE>
 __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
     uint32_t x = rec[lane];
     const uint32_t off = rec[32];
     const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
     const uint32_t v0 = tile * J.V;
-    const uint32_t nv = FULL ? J.V : min(J.V, J.n_vec - v0);
+    const uint32_t nv = min(J.V, J.n_vec - v0);
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
     const uint32_t per_row = J.per_row;
     const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
@@ -419,7 +419,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 }
 
 // ---- the hot loop in PTX -------------------------------------------------------------------------------
-// All full groups of one full tile.  Written as one asm statement so that every branch can be marked
+// All full groups of one tile.  Written as one asm statement so that every branch can be marked
 // warp-uniform (bra.uni) and the rare work - refilling the payload ring, moving to the next row - sits
 // out of line.  Per group: 9 x rans step, Eq. 5 / Eq. 19 on eight weights, one vector store.
 //
@@ -431,28 +431,9 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 //   doff   byte offset of this lane's block in the output;  left = groups still to do
 //   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
 //                     the payload bytes left from there (may be <= 0)
-#ifdef EP_X_MULHI
-#define EP_S_FQ(E)                                              \
-    "mul.hi.u32 f, " E ", %24;\n\t"                             \
-    "mul.hi.u32 q, %0, %25;\n\t"
-#else
 #define EP_S_FQ(E)                                              \
     "shr.u32 f, " E ", 20;\n\t"                                 \
     "shr.u32 q, %0, %14;\n\t"
-#endif
-#ifdef EP_X_INCL
-/* %12 holds the mask of lanes <= this one: the inclusive count of lane 31 is the step's total */
-#define EP_S_FETCH                                              \
-    "and.b32 t, bal, %12;\n\t"                                  \
-    "popc.b32 t, t;\n\t"                                        \
-    "shfl.sync.idx.b32 u, t, 31, 31, 0xffffffff;\n\t"           \
-    "shl.b32 t, t, 1;\n\t"                                      \
-    "add.u32 t, t, %1;\n\t"                                     \
-    "ld.shared.u16 w, [t+-2];\n\t"                              \
-    "@p mad.lo.u32 %0, %0, 65536, w;\n\t"                       \
-    "shl.b32 u, u, 1;\n\t"                                      \
-    "add.u32 %1, %1, u;\n\t"
-#else
 #define EP_S_FETCH                                              \
     "and.b32 t, bal, %12;\n\t"                                  \
     "popc.b32 t, t;\n\t"                                        \
@@ -463,7 +444,6 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
     "popc.b32 t, bal;\n\t"                                      \
     "shl.b32 t, t, 1;\n\t"                                      \
     "add.u32 %1, %1, t;\n\t"
-#endif
 #define EP_S_STEP(E, TAB, OFF)                                  \
     "and.b32 u, %0, %13;\n\t"                                   \
     "shl.b32 u, u, 2;\n\t"                                      \
@@ -636,8 +616,8 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
         : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(col), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
           "+&r"(left), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                          \
-        : "r"(lt_asm), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),        \
-          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max), "r"(mul_f), "r"(mul_q)                                     \
+        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),        \
+          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max)                                                             \
         : "memory")
 
 // One tile of a tensor whose rows hold at least 32 blocks: the full groups in PTX, a last partial group
@@ -681,12 +661,6 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     // different per lane; the loop therefore branches on warp votes of it (see the asm), never on the value itself.
     uint32_t left = nv >> 5;                           // may be 0: the asm then falls straight through
     const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
-#ifdef EP_X_INCL
-    const uint32_t lt_asm = lt | (1u << lane);
-#else
-    const uint32_t lt_asm = lt;
-#endif
-    const uint32_t mul_f = 4096u, mul_q = 1u << (32u - b);   // multiply-high forms of >> 20 and >> b
     if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
     else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
     else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
@@ -737,8 +711,8 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
             }
         }
         if (tile < J.n_tiles) {
-            if (wide) decode_tile<DT, true, false>(J, tile, lut_addr, ring, lane);
-            else decode_tile<DT, false, false>(J, tile, lut_addr, ring, lane);
+            if (wide) decode_tile<DT, true>(J, tile, lut_addr, ring, lane);
+            else decode_tile<DT, false>(J, tile, lut_addr, ring, lane);
         }
     }
 }
