@@ -66,6 +66,10 @@ typedef enum {
     EP_FP16 = 1,        /* round to nearest even, saturating to +-65504 */
     EP_FP8_E4M3 = 2,    /* E4M3FN, round to nearest even incl. subnormals, saturating to +-448 */
     EP_INT8 = 3,        /* round to nearest even integer, saturating to [-128, 127] */
+    EP_FP32 = 4,        /* the fp32 product itself */
+    EP_FP8_E5M2 = 5,    /* E5M2, round to nearest even incl. subnormals, saturating to +-57344 */
+    EP_UINT8 = 6,       /* round to nearest even integer, saturating to [0, 255] (for weights that were
+                           shifted into the unsigned range before compression) */
     EP_FIELDS_I32 = 16  /* verification mode: the nine decoded fields (c, z1..z7, m) of Eq. 4 as
                            int32[R*C/8][9]; row scales are not read */
 } ep_dtype;

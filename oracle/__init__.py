@@ -16,9 +16,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "entropack_oracle.c")
 _LIB = os.path.join(_HERE, "libentropack_oracle.so")
 
-BF16, FP16, E4M3, INT8, FP32 = 0, 1, 2, 3, 4
-DTYPE_SIZE = {BF16: 2, FP16: 2, E4M3: 1, INT8: 1, FP32: 4}
-_NP_OUT = {BF16: np.uint16, FP16: np.uint16, E4M3: np.uint8, INT8: np.int8, FP32: np.float32}
+BF16, FP16, E4M3, INT8, FP32, E5M2, UINT8 = 0, 1, 2, 3, 4, 5, 6
+DTYPE_SIZE = {BF16: 2, FP16: 2, E4M3: 1, INT8: 1, FP32: 4, E5M2: 1, UINT8: 1}
+_NP_OUT = {BF16: np.uint16, FP16: np.uint16, E4M3: np.uint8, INT8: np.int8, FP32: np.float32, E5M2: np.uint8,
+           UINT8: np.uint8}
 
 
 def build(force: bool = False) -> str:

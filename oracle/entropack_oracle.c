@@ -48,7 +48,7 @@
 #define EPO_MAGIC 0x314B5045u /* "EPK1" little-endian */
 #define EPO_ETA 1e-12
 
-enum { EPO_BF16 = 0, EPO_FP16 = 1, EPO_E4M3 = 2, EPO_INT8 = 3, EPO_FP32 = 4 };
+enum { EPO_BF16 = 0, EPO_FP16 = 1, EPO_E4M3 = 2, EPO_INT8 = 3, EPO_FP32 = 4, EPO_E5M2 = 5, EPO_UINT8 = 6 };
 
 typedef struct {
     double bracket_lo, bracket_hi; /* scale bracket, default [1e-3, 8] */
@@ -535,6 +535,28 @@ static uint8_t snap_e4m3(float v) {   /* FP8 E4M3FN: RNE incl. subnormals (step 
     return (uint8_t)(sign | ((ex + 7) << 3) | man);
 }
 
+static uint8_t snap_e5m2(float v) {   /* FP8 E5M2: RNE incl. subnormals (step 2^-16), saturating to +-57344 */
+    if (isnan(v)) return 0x7F;
+    double r = round_to_format((double)v, 2, -14);
+    uint8_t sign = signbit(v) ? 0x80 : 0;
+    double a = fabs(r);
+    if (a > 57344.0) return (uint8_t)(sign | 0x7B);
+    if (a == 0.0) return sign;
+    int e; double m = frexp(a, &e);
+    int ex = e - 1;
+    if (ex < -14) return (uint8_t)(sign | (uint8_t)(a / ldexp(1.0, -16)));
+    uint8_t man = (uint8_t)((m * 2.0 - 1.0) * 4.0);
+    return (uint8_t)(sign | ((ex + 15) << 2) | man);
+}
+
+static uint8_t snap_uint8(float v) {  /* round to nearest even integer, saturating to [0, 255] */
+    if (isnan(v)) return 0;
+    double r = rint((double)v);
+    if (r > 255.0) r = 255.0;
+    if (r < 0.0) r = 0.0;
+    return (uint8_t)r;
+}
+
 static int8_t snap_int8(float v) {
     if (isnan(v)) return 0;
     double r = rint((double)v);
@@ -551,6 +573,8 @@ void epo_snap(const float *v, size_t n, int dtype, void *out) {
         case EPO_FP16: ((uint16_t *)out)[i] = snap_fp16(v[i]); break;
         case EPO_E4M3: ((uint8_t *)out)[i] = snap_e4m3(v[i]); break;
         case EPO_INT8: ((int8_t *)out)[i] = snap_int8(v[i]); break;
+        case EPO_E5M2: ((uint8_t *)out)[i] = snap_e5m2(v[i]); break;
+        case EPO_UINT8: ((uint8_t *)out)[i] = snap_uint8(v[i]); break;
         default: ((float *)out)[i] = v[i]; break;
         }
     }

@@ -11,8 +11,8 @@ import os
 
 import numpy as np
 
-BF16, FP16, FP8_E4M3, INT8, FIELDS_I32 = 0, 1, 2, 3, 16
-DTYPE_BYTES = {BF16: 2, FP16: 2, FP8_E4M3: 1, INT8: 1}
+BF16, FP16, FP8_E4M3, INT8, FP32, FP8_E5M2, UINT8, FIELDS_I32 = 0, 1, 2, 3, 4, 5, 6, 16
+DTYPE_BYTES = {BF16: 2, FP16: 2, FP8_E4M3: 1, INT8: 1, FP32: 4, FP8_E5M2: 1, UINT8: 1}
 NUM_TABLES = 17
 MAX_BATCH = 16
 
@@ -235,7 +235,8 @@ def _torch():
 
 def _out_torch_dtype(dt: int):
     torch = _torch()
-    return {BF16: torch.bfloat16, FP16: torch.float16, FP8_E4M3: torch.float8_e4m3fn, INT8: torch.int8}[dt]
+    return {BF16: torch.bfloat16, FP16: torch.float16, FP8_E4M3: torch.float8_e4m3fn, INT8: torch.int8,
+            FP32: torch.float32, FP8_E5M2: torch.float8_e5m2, UINT8: torch.uint8}[dt]
 
 
 class DeviceBlob:

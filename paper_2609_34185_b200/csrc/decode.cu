@@ -120,6 +120,16 @@ __device__ __forceinline__ uint32_t pack_e4m3(float lo, float hi) {
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
     return r;
 }
+__device__ __forceinline__ uint32_t pack_e5m2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t cvt_u8(float v) {
+    uint32_t r;
+    asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r & 0xFFu;
+}
 __device__ __forceinline__ uint32_t cvt_s8(float v) {
     int32_t r;
     asm("cvt.rni.sat.s8.f32 %0, %1;" : "=r"(r) : "f"(v));
@@ -263,6 +273,33 @@ struct Out<EP_INT8> {
     static __device__ __forceinline__ void store(void *dst, const float (&w)[8]) {
         uint2 q = make_uint2(cvt_s8(w[0]) | (cvt_s8(w[1]) << 8) | (cvt_s8(w[2]) << 16) | (cvt_s8(w[3]) << 24),
                              cvt_s8(w[4]) | (cvt_s8(w[5]) << 8) | (cvt_s8(w[6]) << 16) | (cvt_s8(w[7]) << 24));
+        *reinterpret_cast<uint2 *>(dst) = q;
+    }
+};
+
+template <>
+struct Out<EP_FP32> {
+    static constexpr uint32_t kBlockBytes = 32;
+    static __device__ __forceinline__ void store(void *dst, const float (&w)[8]) {
+        reinterpret_cast<float4 *>(dst)[0] = make_float4(w[0], w[1], w[2], w[3]);
+        reinterpret_cast<float4 *>(dst)[1] = make_float4(w[4], w[5], w[6], w[7]);
+    }
+};
+template <>
+struct Out<EP_FP8_E5M2> {
+    static constexpr uint32_t kBlockBytes = 8;
+    static __device__ __forceinline__ void store(void *dst, const float (&w)[8]) {
+        uint2 q = make_uint2(pack_e5m2(w[0], w[1]) | (pack_e5m2(w[2], w[3]) << 16),
+                             pack_e5m2(w[4], w[5]) | (pack_e5m2(w[6], w[7]) << 16));
+        *reinterpret_cast<uint2 *>(dst) = q;
+    }
+};
+template <>
+struct Out<EP_UINT8> {
+    static constexpr uint32_t kBlockBytes = 8;
+    static __device__ __forceinline__ void store(void *dst, const float (&w)[8]) {
+        uint2 q = make_uint2(cvt_u8(w[0]) | (cvt_u8(w[1]) << 8) | (cvt_u8(w[2]) << 16) | (cvt_u8(w[3]) << 24),
+                             cvt_u8(w[4]) | (cvt_u8(w[5]) << 8) | (cvt_u8(w[6]) << 16) | (cvt_u8(w[7]) << 24));
         *reinterpret_cast<uint2 *>(dst) = q;
     }
 };
@@ -482,6 +519,41 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
     "mov.b32 o0, {h0, h1};\n\t"                                 \
     "mov.b32 o1, {h2, h3};\n\t"                                 \
     "st.global.v2.b32 [ad], {o0, o1};\n\t"
+#define EP_S_STORE_FP32                                         \
+    "mov.b32 o0, w0;\n\t"                                       \
+    "mov.b32 o1, w1;\n\t"                                       \
+    "mov.b32 o2, w2;\n\t"                                       \
+    "mov.b32 o3, w3;\n\t"                                       \
+    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"              \
+    "mov.b32 o0, w4;\n\t"                                       \
+    "mov.b32 o1, w5;\n\t"                                       \
+    "mov.b32 o2, w6;\n\t"                                       \
+    "mov.b32 o3, w7;\n\t"                                       \
+    "st.global.v4.b32 [ad+16], {o0, o1, o2, o3};\n\t"
+#define EP_S_STORE_E5M2                                         \
+    "cvt.rn.satfinite.e5m2x2.f32 h0, w1, w0;\n\t"               \
+    "cvt.rn.satfinite.e5m2x2.f32 h1, w3, w2;\n\t"               \
+    "cvt.rn.satfinite.e5m2x2.f32 h2, w5, w4;\n\t"               \
+    "cvt.rn.satfinite.e5m2x2.f32 h3, w7, w6;\n\t"               \
+    "mov.b32 o0, {h0, h1};\n\t"                                 \
+    "mov.b32 o1, {h2, h3};\n\t"                                 \
+    "st.global.v2.b32 [ad], {o0, o1};\n\t"
+#define EP_S_STORE_UINT8                                        \
+    "cvt.rni.sat.u8.f32 o0, w0;\n\t"                            \
+    "cvt.rni.sat.u8.f32 o2, w1;\n\t"                            \
+    "bfi.b32 o0, o2, o0, 8, 8;\n\t"                             \
+    "cvt.rni.sat.u8.f32 o2, w2;\n\t"                            \
+    "bfi.b32 o0, o2, o0, 16, 8;\n\t"                            \
+    "cvt.rni.sat.u8.f32 o2, w3;\n\t"                            \
+    "bfi.b32 o0, o2, o0, 24, 8;\n\t"                            \
+    "cvt.rni.sat.u8.f32 o1, w4;\n\t"                            \
+    "cvt.rni.sat.u8.f32 o2, w5;\n\t"                            \
+    "bfi.b32 o1, o2, o1, 8, 8;\n\t"                             \
+    "cvt.rni.sat.u8.f32 o2, w6;\n\t"                            \
+    "bfi.b32 o1, o2, o1, 16, 8;\n\t"                            \
+    "cvt.rni.sat.u8.f32 o2, w7;\n\t"                            \
+    "bfi.b32 o1, o2, o1, 24, 8;\n\t"                            \
+    "st.global.v2.b32 [ad], {o0, o1};\n\t"
 #define EP_S_STORE_INT8                                         \
     "cvt.rni.sat.s8.f32 o0, w0;\n\t"                            \
     "cvt.rni.sat.s8.f32 o2, w1;\n\t"                            \
@@ -664,6 +736,9 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
     else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
     else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
+    else if constexpr (DT == EP_FP32) EP_FULL_GROUPS_ASM(EP_S_STORE_FP32, 1024);
+    else if constexpr (DT == EP_FP8_E5M2) EP_FULL_GROUPS_ASM(EP_S_STORE_E5M2, 256);
+    else if constexpr (DT == EP_UINT8) EP_FULL_GROUPS_ASM(EP_S_STORE_UINT8, 256);
     else EP_FULL_GROUPS_ASM(EP_S_STORE_INT8, 256);
     uint32_t pos = wa - wbase;
     if (nv & 31u) {
@@ -986,6 +1061,9 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
     case EP_FP16: e = launch_glut<EP_FP16>(P, next, st); break;
     case EP_FP8_E4M3: e = launch_glut<EP_FP8_E4M3>(P, next, st); break;
     case EP_INT8: e = launch_glut<EP_INT8>(P, next, st); break;
+    case EP_FP32: e = launch_glut<EP_FP32>(P, next, st); break;
+    case EP_FP8_E5M2: e = launch_glut<EP_FP8_E5M2>(P, next, st); break;
+    case EP_UINT8: e = launch_glut<EP_UINT8>(P, next, st); break;
     case EP_FIELDS_I32: e = launch_glut<EP_FIELDS_I32>(P, next, st); break;
     default: return EP_ERR_BAD_ARG;
     }
@@ -1000,7 +1078,9 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     if (sms <= 0) return EP_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int32_t dt = jobs_in[0].out_dtype;
-    if (dt != EP_BF16 && dt != EP_FP16 && dt != EP_FP8_E4M3 && dt != EP_INT8 && dt != EP_FIELDS_I32) return EP_ERR_BAD_ARG;
+    if (dt != EP_BF16 && dt != EP_FP16 && dt != EP_FP8_E4M3 && dt != EP_INT8 && dt != EP_FP32 && dt != EP_FP8_E5M2 &&
+        dt != EP_UINT8 && dt != EP_FIELDS_I32)
+        return EP_ERR_BAD_ARG;
     const ep_decode_job *fast[EP_MAX_BATCH], *large[EP_MAX_BATCH];
     int n_jobs = 0, n_large = 0;
     uint64_t tiles_total = 0;
@@ -1072,6 +1152,9 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     case EP_FP16: e = launch_smem<EP_FP16>(P, next, st); break;
     case EP_FP8_E4M3: e = launch_smem<EP_FP8_E4M3>(P, next, st); break;
     case EP_INT8: e = launch_smem<EP_INT8>(P, next, st); break;
+    case EP_FP32: e = launch_smem<EP_FP32>(P, next, st); break;
+    case EP_FP8_E5M2: e = launch_smem<EP_FP8_E5M2>(P, next, st); break;
+    case EP_UINT8: e = launch_smem<EP_UINT8>(P, next, st); break;
     case EP_FIELDS_I32: e = launch_smem<EP_FIELDS_I32>(P, next, st); break;
     default: return EP_ERR_BAD_ARG;
     }

@@ -11,14 +11,17 @@ from paper_2609_34185_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-ORACLE_DT = {ep.BF16: oracle.BF16, ep.FP16: oracle.FP16, ep.FP8_E4M3: oracle.E4M3, ep.INT8: oracle.INT8}
+ORACLE_DT = {ep.BF16: oracle.BF16, ep.FP16: oracle.FP16, ep.FP8_E4M3: oracle.E4M3, ep.INT8: oracle.INT8,
+             ep.FP32: oracle.FP32, ep.FP8_E5M2: oracle.E5M2, ep.UINT8: oracle.UINT8}
 
 
 def _bits(t: torch.Tensor) -> np.ndarray:
     if t.dtype in (torch.bfloat16, torch.float16):
         return t.view(torch.int16).cpu().numpy().view(np.uint16)
-    if t.dtype == torch.float8_e4m3fn:
+    if t.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
         return t.view(torch.uint8).cpu().numpy()
+    if t.dtype == torch.float32:
+        return t.view(torch.int32).cpu().numpy().view(np.uint32)
     return t.cpu().numpy()
 
 
@@ -30,6 +33,8 @@ def _check_all_types(blob_bytes, scales=None):
         got = ep.decode(d, dt, row_scales=sc_dev)
         ref, ref_fields = oracle.decode(blob_bytes, odt, scales=scales, want_fields=True)
         torch.cuda.synchronize()
+        if dt == ep.FP32:
+            ref = ref.view(np.uint32)
         assert np.array_equal(_bits(got), ref), f"dtype {dt}"
     f = ep.decode(d, ep.FIELDS_I32)
     assert np.array_equal(f.cpu().numpy(), ref_fields)

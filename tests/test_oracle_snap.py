@@ -67,6 +67,21 @@ def test_e4m3_every_rounding_boundary():
     assert list(oracle.snap(t, oracle.E4M3)) == [0x7E, 0x7E, 0x7E, 0x7E, 0xFE, 0xFE]
 
 
+def test_e5m2_matches_library_cast_in_range_and_saturates():
+    v = _vals()
+    v = np.concatenate([v, np.array([1.5e-5, 7.6e-6, 2.3e-5, 3e-5, 6.1e-5, 57344.0, 50000.0], np.float32)])
+    v = v[np.abs(v) <= 57344.0]
+    ref = torch.from_numpy(v).to(torch.float8_e5m2).view(torch.uint8).numpy()
+    assert np.array_equal(oracle.snap(v, oracle.E5M2), ref)
+    t = np.array([61439.0, 61440.0, 1e9, np.inf, -1e9], np.float32)     # beyond the last rounding boundary: saturate
+    assert list(oracle.snap(t, oracle.E5M2)) == [0x7B, 0x7B, 0x7B, 0x7B, 0xFB]
+
+
+def test_uint8_round_half_even_and_saturation():
+    t = np.array([0.5, 1.5, 2.5, -0.5, -3.0, 254.5, 255.5, 300.0, 127.49, 128.5], np.float32)
+    assert list(oracle.snap(t, oracle.UINT8)) == [0, 2, 2, 0, 0, 254, 255, 255, 127, 128]
+
+
 def test_int8_round_half_even_and_saturation():
     t = np.array([0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 126.5, 127.5, 300.0, -128.5, -129.5, -1e9, 3.49, -3.51],
                  np.float32)
