@@ -22,17 +22,9 @@
 #include <thread>
 #include <vector>
 
-#include "stream.hpp"
-
-struct ep_blob {
-    std::vector<uint8_t> bytes;
-    ep_encode_report report{};
-};
+#include "encoder_core.hpp"
 
 namespace ep {
-namespace {
-
-constexpr double kEta = 1e-12;
 
 // ---- small thread helper: static contiguous partition of [0, n) -------------------------------
 void parallel_for(uint64_t n, int threads, const std::function<void(uint64_t, uint64_t, int)> &body) {
@@ -52,6 +44,312 @@ int resolve_threads(int requested) {
     const unsigned hw = std::thread::hardware_concurrency();
     return hw ? int(hw) : 1;
 }
+
+// ---- Sec. 3.3: the seventeen categorical tables -------------------------------------------------
+uint32_t Table::observed() const {
+    uint32_t o = 0;
+    for (uint64_t c : n) o += c != 0;
+    return o;
+}
+
+// counts from field tuples; threads reduce private (min, max) first, then private histograms
+void Model::count(const int32_t *fld, uint64_t nvec, int threads) {
+    struct Range { int64_t lo[EP_NUM_TABLES], hi[EP_NUM_TABLES]; bool any[EP_NUM_TABLES]; };
+    const int T = std::max(1, threads);
+    std::vector<Range> rg(T);
+    for (auto &r : rg) for (int i = 0; i < EP_NUM_TABLES; ++i) { r.any[i] = false; r.lo[i] = r.hi[i] = 0; }
+    parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
+        Range &r = rg[id];
+        for (uint64_t v = a; v < b; ++v) {
+            const int32_t *q = fld + 9 * v;
+            for (int k = 0; k < 9; ++k) {
+                const int ti = table_id(q[0], k);
+                if (!r.any[ti]) { r.any[ti] = true; r.lo[ti] = r.hi[ti] = q[k]; }
+                else { r.lo[ti] = std::min<int64_t>(r.lo[ti], q[k]); r.hi[ti] = std::max<int64_t>(r.hi[ti], q[k]); }
+            }
+        }
+    });
+    for (int i = 0; i < EP_NUM_TABLES; ++i) {
+        bool any = false;
+        int64_t lo = 0, hi = 0;
+        for (auto &r : rg) if (r.any[i]) {
+            if (!any) { lo = r.lo[i]; hi = r.hi[i]; any = true; }
+            else { lo = std::min(lo, r.lo[i]); hi = std::max(hi, r.hi[i]); }
+        }
+        t[i] = Table();
+        if (any) { t[i].lo = int32_t(lo); t[i].n.assign(size_t(hi - lo + 1), 0); }
+    }
+    std::vector<std::vector<uint64_t>> priv(size_t(T) * EP_NUM_TABLES);
+    parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
+        std::vector<uint64_t> *h = &priv[size_t(id) * EP_NUM_TABLES];
+        for (int i = 0; i < EP_NUM_TABLES; ++i) h[i].assign(t[i].n.size(), 0);
+        for (uint64_t v = a; v < b; ++v) {
+            const int32_t *q = fld + 9 * v;
+            for (int k = 0; k < 9; ++k) {
+                const int ti = table_id(q[0], k);
+                h[ti][size_t(q[k] - t[ti].lo)]++;
+            }
+        }
+    });
+    for (int id = 0; id < T; ++id)
+        for (int i = 0; i < EP_NUM_TABLES; ++i) {
+            const auto &h = priv[size_t(id) * EP_NUM_TABLES + i];
+            for (size_t j = 0; j < h.size(); ++j) { t[i].n[j] += h[j]; t[i].total += h[j]; }
+        }
+}
+
+void Model::from_histograms(const uint32_t *hist, uint32_t bins, int32_t origin) {
+    for (int i = 0; i < EP_NUM_TABLES; ++i) {
+        const uint32_t *h = hist + size_t(i) * bins;
+        uint32_t first = bins, last = 0;
+        for (uint32_t j = 0; j < bins; ++j)
+            if (h[j]) { if (first == bins) first = j; last = j; }
+        t[i] = Table();
+        if (first == bins) continue;
+        t[i].lo = origin + int32_t(first);
+        t[i].n.assign(h + first, h + last + 1);
+        for (uint64_t c : t[i].n) t[i].total += c;
+    }
+}
+
+// integer frequencies summing to 2^b, every observed symbol >= 1
+void Model::normalise(int b) {
+    const uint64_t M = 1ull << b;
+    for (auto &tb : t) {
+        const uint32_t K = tb.K();
+        tb.f.assign(K, 0);
+        tb.F.assign(K + 1, 0);
+        if (!K || !tb.total) continue;
+        uint64_t sum = 0;
+        for (uint32_t j = 0; j < K; ++j) {
+            if (!tb.n[j]) continue;
+            const uint64_t q = tb.n[j] * M / tb.total;
+            tb.f[j] = uint32_t(std::max<uint64_t>(q, 1));
+            sum += tb.f[j];
+        }
+        auto largest = [&] { return uint32_t(std::max_element(tb.f.begin(), tb.f.end()) - tb.f.begin()); };
+        if (sum < M) tb.f[largest()] += uint32_t(M - sum);
+        while (sum > M) {
+            const uint32_t j = largest();
+            const uint64_t take = std::min<uint64_t>(sum - M, uint64_t(tb.f[j]) - 1);
+            tb.f[j] -= uint32_t(take);
+            sum -= take;
+        }
+        for (uint32_t j = 0; j < K; ++j) tb.F[j + 1] = tb.F[j] + tb.f[j];
+    }
+}
+
+// Eq. 8
+double Model::cross_entropy_bits(int b) const {
+    double acc = 0.0;
+    for (const auto &tb : t)
+        for (uint32_t j = 0; j < tb.K(); ++j)
+            if (tb.n[j]) acc += double(tb.n[j]) * (double(b) - std::log2(double(tb.f[j])));
+    return acc;
+}
+
+uint64_t Model::section_bytes() const {
+    uint32_t K[EP_NUM_TABLES];
+    for (int i = 0; i < EP_NUM_TABLES; ++i) K[i] = t[i].K();
+    return table_section_bytes(K);
+}
+
+uint32_t Model::worst_observed() const {
+    uint32_t w = 0;
+    for (const auto &tb : t) w = std::max(w, tb.observed());
+    return w;
+}
+
+uint32_t Model::worst_coordinate_observed() const {
+    uint32_t w = 0;
+    for (int i = 1; i < EP_NUM_TABLES; ++i) w = std::max(w, t[i].observed());
+    return w;
+}
+
+// Eq. 10-11: estimated stored bits of nvec vectors in `rows` rows under model m
+double estimate_bits(const Model &m, int b, uint64_t nvec, uint64_t rows, uint32_t V, double retained, double *cce_out) {
+    const double cce = m.cross_entropy_bits(b);
+    const uint64_t n_tile = (nvec + V - 1) / V;
+    const double left = std::max(0.0, cce - retained * double(kStates) * double(n_tile));
+    const double payload = 16.0 * std::ceil(left / 16.0);
+    const double restart = double(n_tile) * (32.0 * kStates + 32.0) + 32.0;
+    const double tables = 8.0 * double(m.section_bytes());
+    const double scales = 32.0 * double(rows);
+    const double other = 8.0 * kHeaderBytes;
+    if (cce_out) *cce_out = cce;
+    return payload + restart + tables + scales + other;
+}
+
+// ---- App. "Scale-search settings": the fixed row sample -----------------------------------------
+static inline uint64_t splitmix64(uint64_t &state) {
+    uint64_t z = (state += 0x9E3779B97F4A7C15ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+std::vector<uint32_t> sample_rows(uint32_t R, uint32_t C, uint32_t budget_vectors) {
+    const uint32_t per_row = C / 8;
+    uint32_t n = std::max<uint32_t>(1, budget_vectors / per_row);
+    n = std::min(n, R);
+    std::vector<uint32_t> idx(R);
+    for (uint32_t i = 0; i < R; ++i) idx[i] = i;
+    uint64_t st = (uint64_t(R) << 32) + uint64_t(C);
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint32_t j = i + uint32_t(splitmix64(st) % uint64_t(R - i));
+        std::swap(idx[i], idx[j]);
+    }
+    idx.resize(n);
+    std::sort(idx.begin(), idx.end());
+    return idx;
+}
+
+// header + tables + scales + tile index + payload
+int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
+                  const uint32_t *states, const uint16_t *const *tile_words, const uint32_t *tile_len, ep_blob *out) {
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    const uint32_t n_tiles = uint32_t((nvec + V - 1) / V);
+    uint64_t total_words = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) total_words += tile_len[t];
+    // coordinate range of z_1..z_8 (z_8 = 2m + parity spans [2 m_lo, 2 m_hi + 1])
+    bool any = false;
+    int64_t cmin = 0, cmax = 0;
+    for (int c = 0; c < 2; ++c)
+        for (int k = 1; k <= 8; ++k) {
+            const Table &tb = m.t[table_id(c, k)];
+            if (!tb.K()) continue;
+            int64_t lo = tb.lo, hi = int64_t(tb.lo) + tb.K() - 1;
+            if (k == 8) { lo *= 2; hi = 2 * hi + 1; }
+            if (!any) { cmin = lo; cmax = hi; any = true; }
+            else { cmin = std::min(cmin, lo); cmax = std::max(cmax, hi); }
+        }
+    cmin = std::max<int64_t>(cmin, -32768);
+    cmax = std::min<int64_t>(cmax, 32767);
+    const uint64_t tb_bytes = m.section_bytes();
+    const uint64_t off_tables = kHeaderBytes, off_scales = off_tables + tb_bytes, off_tiles = off_scales + 4ull * R;
+    const uint64_t off_payload = off_tiles + uint64_t(kTileRecordBytes) * n_tiles + 4, total = off_payload + 2 * total_words;
+    if (total >= (1ull << 32)) return EP_ERR_UNSUPPORTED;   // section offsets are 32-bit
+    std::vector<uint8_t> &B = out->bytes;
+    B.assign(size_t(total), 0);
+    uint8_t *p = B.data();
+    store_le<uint32_t>(p, kMagic);
+    store_le<uint16_t>(p + 4, 1);
+    p[6] = uint8_t(b);
+    p[7] = uint8_t(kStates);
+    store_le<uint32_t>(p + 8, R);
+    store_le<uint32_t>(p + 12, C);
+    store_le<uint32_t>(p + 16, V);
+    store_le<uint32_t>(p + 20, n_tiles);
+    store_le<float>(p + 24, s_info);
+    store_le<int16_t>(p + 28, int16_t(cmin));
+    store_le<int16_t>(p + 30, int16_t(cmax));
+    store_le<uint32_t>(p + 32, uint32_t(off_tables));
+    store_le<uint32_t>(p + 36, uint32_t(off_scales));
+    store_le<uint32_t>(p + 40, uint32_t(off_tiles));
+    store_le<uint32_t>(p + 44, uint32_t(off_payload));
+    store_le<uint64_t>(p + 48, total);
+    store_le<uint32_t>(p + 56, uint32_t(total_words));
+    uint8_t *dir = p + off_tables;
+    uint8_t *fq = dir + 8 * EP_NUM_TABLES;
+    for (int i = 0; i < EP_NUM_TABLES; ++i) {
+        store_le<int32_t>(dir + 4 * i, m.t[i].lo);
+        store_le<uint32_t>(dir + 4 * EP_NUM_TABLES + 4 * i, m.t[i].K());
+        for (uint32_t j = 0; j < m.t[i].K(); ++j, fq += 2) store_le<uint16_t>(fq, uint16_t(m.t[i].f[j]));
+    }
+    std::memcpy(p + off_scales, sigma, 4ull * R);
+    uint64_t at = 0;
+    for (uint32_t t = 0; t < n_tiles; ++t) {
+        uint8_t *rec = p + off_tiles + uint64_t(kTileRecordBytes) * t;
+        std::memcpy(rec, states + size_t(t) * kStates, 4 * kStates);
+        store_le<uint32_t>(rec + 4 * kStates, uint32_t(at));
+        if (tile_len[t]) std::memcpy(p + off_payload + 2 * at, tile_words[t], 2ull * tile_len[t]);
+        at += tile_len[t];
+    }
+    store_le<uint32_t>(p + off_tiles + uint64_t(kTileRecordBytes) * n_tiles, uint32_t(at));
+    return EP_OK;
+}
+
+// ---- Algorithm 1 + rate correction + packing, over a back end ---------------------------------------
+int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts &o, ep_blob **out) {
+    const uint64_t nvec = uint64_t(R) * (C / 8);
+    const uint32_t V = o.tile_vectors ? o.tile_vectors : ep_default_tile_vectors(target_bpp);
+    int b = o.b_start ? o.b_start : (target_bpp <= 7.0 ? 11 : 12);
+    b = std::min(b, o.b_max);
+    const std::vector<uint32_t> rows = sample_rows(R, C, o.sample_vectors);
+    const uint64_t svec = uint64_t(rows.size()) * (C / 8);
+    int rc = be.prepare(rows);
+    if (rc) return rc;
+    float s = 0.0f;
+    double last_rate = 0.0;
+    Model full;
+    for (;; ++b) {
+        double lo = o.bracket_lo, hi = o.bracket_hi;
+        for (int it = 0; it < o.search_steps; ++it) {
+            const double mid = std::sqrt(lo * hi);
+            Model m;
+            if ((rc = be.count_sample(float(mid), m))) return rc;
+            m.normalise(b);
+            const double bits = estimate_bits(m, b, svec, rows.size(), V, o.retained_bits, nullptr);
+            last_rate = bits / (8.0 * double(svec));
+            if (last_rate > target_bpp) lo = mid; else hi = mid;
+        }
+        s = float(std::sqrt(lo * hi));
+        bool fits = false;
+        for (;;) {
+            if ((rc = be.count_full(s, full))) return rc;
+            if (full.worst_observed() <= (1u << b)) { fits = true; break; }
+            if (b < o.b_max) break;
+            s = float(1.05 * double(s) * double(full.worst_coordinate_observed()) / double(1u << b));
+        }
+        if (fits) break;
+    }
+    // Beyond Algorithm 1: steer s with the full-tensor estimate (Eq. 10-11), first by the one-bit-per-doubling
+    // law (Eq. 9), then by the measured slope.  The sampled tables miss rare symbols of the full tensor, which
+    // costs rate on heavy tails.
+    struct { double log_s, rate; bool valid; } last{0.0, 0.0, false};
+    for (int step = 0; step < o.polish_steps; ++step) {
+        Model m = full;
+        m.normalise(b);
+        const double est = estimate_bits(m, b, nvec, R, V, o.polish_retained_bits, nullptr) / (double(R) * double(C));
+        if (std::fabs(est - target_bpp) <= 0.002 * target_bpp) break;
+        // rate lost per doubling of s: 1 bit by Eq. 9 for the first move, afterwards the secant slope
+        const double log_s = std::log2(double(s));
+        double per_doubling = 1.0;
+        if (last.valid && log_s != last.log_s) {
+            per_doubling = -(est - last.rate) / (log_s - last.log_s);
+            if (!(per_doubling >= 0.5)) per_doubling = 0.5;
+            if (per_doubling > 4.0) per_doubling = 4.0;
+        }
+        last = {log_s, est, true};
+        const float before = s;
+        double moved = std::exp2(log_s + (est - target_bpp) / per_doubling);
+        if (!(moved >= o.bracket_lo)) moved = o.bracket_lo;   // never leave the search bracket
+        if (moved > o.bracket_hi) moved = o.bracket_hi;
+        s = float(moved);
+        if (s == before) break;
+        if ((rc = be.count_full(s, full))) return rc;
+        if (full.worst_observed() > (1u << b)) {   // the finer scale overflows the tables: undo and stop
+            s = before;
+            if ((rc = be.count_full(s, full))) return rc;
+            break;
+        }
+    }
+    full.normalise(b);
+    ep_blob *blob = new ep_blob();
+    rc = be.finish(s, b, V, full, blob);
+    if (rc) { delete blob; return rc; }
+    blob->report.s = double(s);
+    blob->report.b = b;
+    blob->report.bytes = blob->bytes.size();
+    blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
+    blob->report.est_bpp_sample = last_rate;
+    blob->report.cce_bits = full.cross_entropy_bits(b);
+    blob->report.sample_rows = uint32_t(rows.size());
+    *out = blob;
+    return EP_OK;
+}
+
+namespace {
 
 // ---- Sec. 3.2 ----------------------------------------------------------------------------------
 float row_rms(const float *x, uint32_t C) {
@@ -135,151 +433,6 @@ void quantise_rows(const float *W, uint32_t C, const float *mu, const uint32_t *
     });
 }
 
-// ---- Sec. 3.3: the seventeen categorical tables -------------------------------------------------
-struct Table {
-    int32_t lo = 0;
-    std::vector<uint64_t> n;   // counts over [lo, lo + K)
-    std::vector<uint32_t> f;   // b-bit frequencies
-    std::vector<uint32_t> F;   // exclusive prefix sums, K + 1 entries
-    uint64_t total = 0;
-    uint32_t K() const { return uint32_t(n.size()); }
-    uint32_t observed() const {
-        uint32_t o = 0;
-        for (uint64_t c : n) o += c != 0;
-        return o;
-    }
-};
-
-struct Model {
-    Table t[EP_NUM_TABLES];
-
-    // counts from field tuples; threads reduce private (min, max) first, then private histograms
-    void count(const int32_t *fld, uint64_t nvec, int threads) {
-        struct Range { int64_t lo[EP_NUM_TABLES], hi[EP_NUM_TABLES]; bool any[EP_NUM_TABLES]; };
-        const int T = std::max(1, threads);
-        std::vector<Range> rg(T);
-        for (auto &r : rg) for (int i = 0; i < EP_NUM_TABLES; ++i) { r.any[i] = false; r.lo[i] = r.hi[i] = 0; }
-        parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
-            Range &r = rg[id];
-            for (uint64_t v = a; v < b; ++v) {
-                const int32_t *q = fld + 9 * v;
-                for (int k = 0; k < 9; ++k) {
-                    const int ti = table_id(q[0], k);
-                    if (!r.any[ti]) { r.any[ti] = true; r.lo[ti] = r.hi[ti] = q[k]; }
-                    else { r.lo[ti] = std::min<int64_t>(r.lo[ti], q[k]); r.hi[ti] = std::max<int64_t>(r.hi[ti], q[k]); }
-                }
-            }
-        });
-        for (int i = 0; i < EP_NUM_TABLES; ++i) {
-            bool any = false;
-            int64_t lo = 0, hi = 0;
-            for (auto &r : rg) if (r.any[i]) {
-                if (!any) { lo = r.lo[i]; hi = r.hi[i]; any = true; }
-                else { lo = std::min(lo, r.lo[i]); hi = std::max(hi, r.hi[i]); }
-            }
-            t[i] = Table();
-            if (any) { t[i].lo = int32_t(lo); t[i].n.assign(size_t(hi - lo + 1), 0); }
-        }
-        std::vector<std::vector<uint64_t>> priv(size_t(T) * EP_NUM_TABLES);
-        parallel_for(nvec, T, [&](uint64_t a, uint64_t b, int id) {
-            std::vector<uint64_t> *h = &priv[size_t(id) * EP_NUM_TABLES];
-            for (int i = 0; i < EP_NUM_TABLES; ++i) h[i].assign(t[i].n.size(), 0);
-            for (uint64_t v = a; v < b; ++v) {
-                const int32_t *q = fld + 9 * v;
-                for (int k = 0; k < 9; ++k) {
-                    const int ti = table_id(q[0], k);
-                    h[ti][size_t(q[k] - t[ti].lo)]++;
-                }
-            }
-        });
-        for (int id = 0; id < T; ++id)
-            for (int i = 0; i < EP_NUM_TABLES; ++i) {
-                const auto &h = priv[size_t(id) * EP_NUM_TABLES + i];
-                for (size_t j = 0; j < h.size(); ++j) { t[i].n[j] += h[j]; t[i].total += h[j]; }
-            }
-    }
-
-    // integer frequencies summing to 2^b, every observed symbol >= 1
-    void normalise(int b) {
-        const uint64_t M = 1ull << b;
-        for (auto &tb : t) {
-            const uint32_t K = tb.K();
-            tb.f.assign(K, 0);
-            tb.F.assign(K + 1, 0);
-            if (!K || !tb.total) continue;
-            uint64_t sum = 0;
-            for (uint32_t j = 0; j < K; ++j) {
-                if (!tb.n[j]) continue;
-                const uint64_t q = tb.n[j] * M / tb.total;
-                tb.f[j] = uint32_t(std::max<uint64_t>(q, 1));
-                sum += tb.f[j];
-            }
-            auto largest = [&] { return uint32_t(std::max_element(tb.f.begin(), tb.f.end()) - tb.f.begin()); };
-            if (sum < M) tb.f[largest()] += uint32_t(M - sum);
-            while (sum > M) {
-                const uint32_t j = largest();
-                const uint64_t take = std::min<uint64_t>(sum - M, uint64_t(tb.f[j]) - 1);
-                tb.f[j] -= uint32_t(take);
-                sum -= take;
-            }
-            for (uint32_t j = 0; j < K; ++j) tb.F[j + 1] = tb.F[j] + tb.f[j];
-        }
-    }
-
-    // Eq. 8
-    double cross_entropy_bits(int b) const {
-        double acc = 0.0;
-        for (const auto &tb : t)
-            for (uint32_t j = 0; j < tb.K(); ++j)
-                if (tb.n[j]) acc += double(tb.n[j]) * (double(b) - std::log2(double(tb.f[j])));
-        return acc;
-    }
-
-    uint64_t section_bytes() const {
-        uint32_t K[EP_NUM_TABLES];
-        for (int i = 0; i < EP_NUM_TABLES; ++i) K[i] = t[i].K();
-        return table_section_bytes(K);
-    }
-};
-
-// Eq. 10-11: estimated stored bits of nvec vectors in `rows` rows under model m
-double estimate_bits(const Model &m, int b, uint64_t nvec, uint64_t rows, uint32_t V, double retained, double *cce_out) {
-    const double cce = m.cross_entropy_bits(b);
-    const uint64_t n_tile = (nvec + V - 1) / V;
-    const double left = std::max(0.0, cce - retained * double(kStates) * double(n_tile));
-    const double payload = 16.0 * std::ceil(left / 16.0);
-    const double restart = double(n_tile) * (32.0 * kStates + 32.0) + 32.0;
-    const double tables = 8.0 * double(m.section_bytes());
-    const double scales = 32.0 * double(rows);
-    const double other = 8.0 * kHeaderBytes;
-    if (cce_out) *cce_out = cce;
-    return payload + restart + tables + scales + other;
-}
-
-// ---- App. "Scale-search settings": the fixed row sample -----------------------------------------
-inline uint64_t splitmix64(uint64_t &state) {
-    uint64_t z = (state += 0x9E3779B97F4A7C15ull);
-    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-    return z ^ (z >> 31);
-}
-
-std::vector<uint32_t> sample_rows(uint32_t R, uint32_t C, uint32_t budget_vectors) {
-    const uint32_t per_row = C / 8;
-    uint32_t n = std::max<uint32_t>(1, budget_vectors / per_row);
-    n = std::min(n, R);
-    std::vector<uint32_t> idx(R);
-    for (uint32_t i = 0; i < R; ++i) idx[i] = i;
-    uint64_t st = (uint64_t(R) << 32) + uint64_t(C);
-    for (uint32_t i = 0; i < n; ++i) {
-        const uint32_t j = i + uint32_t(splitmix64(st) % uint64_t(R - i));
-        std::swap(idx[i], idx[j]);
-    }
-    idx.resize(n);
-    std::sort(idx.begin(), idx.end());
-    return idx;
-}
-
 // ---- Sec. 3.6 / App. "Tiled rANS implementation": one tile -------------------------------------
 // The decoder visits (group of 32 vectors, field 0..8, lane 0..31); the encoder walks that order
 // backwards, emits a word before the update whenever xi >= f * 2^(31-b), and finally reverses the
@@ -307,15 +460,10 @@ void encode_tile(const int32_t *fld, uint32_t nv, const Model &m, int b, uint32_
     std::copy(xi, xi + kStates, states);
 }
 
-// final tables -> tiles -> stored representation
-int pack(const int32_t *fields, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
-         int threads, ep_blob *out, double *cce_out) {
+// tile coding of given fields under a normalised model, then assembly
+int pack_fields_host(const int32_t *fields, uint32_t R, uint32_t C, int b, uint32_t V, const Model &m, const float *sigma,
+                     float s_info, int threads, ep_blob *out) {
     const uint64_t nvec = uint64_t(R) * (C / 8);
-    Model m;
-    m.count(fields, nvec, threads);
-    for (const auto &tb : m.t) if (tb.observed() > (1u << b)) return EP_ERR_UNSUPPORTED;
-    m.normalise(b);
-    if (cce_out) *cce_out = m.cross_entropy_bits(b);
     const uint32_t n_tiles = uint32_t((nvec + V - 1) / V);
     std::vector<std::vector<uint16_t>> words(n_tiles);
     std::vector<uint32_t> states(size_t(n_tiles) * kStates);
@@ -326,64 +474,10 @@ int pack(const int32_t *fields, uint32_t R, uint32_t C, int b, uint32_t V, const
             encode_tile(fields + 9 * v0, nv, m, b, &states[t * kStates], words[t]);
         }
     });
-    uint64_t total_words = 0;
-    for (const auto &w : words) total_words += w.size();
-    // coordinate range of z_1..z_8 (z_8 = 2m + parity spans [2 m_lo, 2 m_hi + 1])
-    bool any = false;
-    int64_t cmin = 0, cmax = 0;
-    for (int c = 0; c < 2; ++c)
-        for (int k = 1; k <= 8; ++k) {
-            const Table &tb = m.t[table_id(c, k)];
-            if (!tb.K()) continue;
-            int64_t lo = tb.lo, hi = int64_t(tb.lo) + tb.K() - 1;
-            if (k == 8) { lo *= 2; hi = 2 * hi + 1; }
-            if (!any) { cmin = lo; cmax = hi; any = true; }
-            else { cmin = std::min(cmin, lo); cmax = std::max(cmax, hi); }
-        }
-    cmin = std::max<int64_t>(cmin, -32768);
-    cmax = std::min<int64_t>(cmax, 32767);
-    const uint64_t tb_bytes = m.section_bytes();
-    const uint64_t off_tables = kHeaderBytes, off_scales = off_tables + tb_bytes, off_tiles = off_scales + 4ull * R;
-    const uint64_t off_payload = off_tiles + uint64_t(kTileRecordBytes) * n_tiles + 4, total = off_payload + 2 * total_words;
-    if (total >= (1ull << 32)) return EP_ERR_UNSUPPORTED;   // section offsets are 32-bit
-    std::vector<uint8_t> &B = out->bytes;
-    B.assign(size_t(total), 0);
-    uint8_t *p = B.data();
-    store_le<uint32_t>(p, kMagic);
-    store_le<uint16_t>(p + 4, 1);
-    p[6] = uint8_t(b);
-    p[7] = uint8_t(kStates);
-    store_le<uint32_t>(p + 8, R);
-    store_le<uint32_t>(p + 12, C);
-    store_le<uint32_t>(p + 16, V);
-    store_le<uint32_t>(p + 20, n_tiles);
-    store_le<float>(p + 24, s_info);
-    store_le<int16_t>(p + 28, int16_t(cmin));
-    store_le<int16_t>(p + 30, int16_t(cmax));
-    store_le<uint32_t>(p + 32, uint32_t(off_tables));
-    store_le<uint32_t>(p + 36, uint32_t(off_scales));
-    store_le<uint32_t>(p + 40, uint32_t(off_tiles));
-    store_le<uint32_t>(p + 44, uint32_t(off_payload));
-    store_le<uint64_t>(p + 48, total);
-    store_le<uint32_t>(p + 56, uint32_t(total_words));
-    uint8_t *dir = p + off_tables;
-    uint8_t *fq = dir + 8 * EP_NUM_TABLES;
-    for (int i = 0; i < EP_NUM_TABLES; ++i) {
-        store_le<int32_t>(dir + 4 * i, m.t[i].lo);
-        store_le<uint32_t>(dir + 4 * EP_NUM_TABLES + 4 * i, m.t[i].K());
-        for (uint32_t j = 0; j < m.t[i].K(); ++j, fq += 2) store_le<uint16_t>(fq, uint16_t(m.t[i].f[j]));
-    }
-    std::memcpy(p + off_scales, sigma, 4ull * R);
-    uint64_t at = 0;
-    for (uint32_t t = 0; t < n_tiles; ++t) {
-        uint8_t *rec = p + off_tiles + uint64_t(kTileRecordBytes) * t;
-        std::memcpy(rec, &states[size_t(t) * kStates], 4 * kStates);
-        store_le<uint32_t>(rec + 4 * kStates, uint32_t(at));
-        if (!words[t].empty()) std::memcpy(p + off_payload + 2 * at, words[t].data(), 2 * words[t].size());
-        at += words[t].size();
-    }
-    store_le<uint32_t>(p + off_tiles + uint64_t(kTileRecordBytes) * n_tiles, uint32_t(at));
-    return EP_OK;
+    std::vector<const uint16_t *> ptr(n_tiles);
+    std::vector<uint32_t> len(n_tiles);
+    for (uint32_t t = 0; t < n_tiles; ++t) { ptr[t] = words[t].data(); len[t] = uint32_t(words[t].size()); }
+    return assemble_blob(m, R, C, b, V, sigma, s_info, states.data(), ptr.data(), len.data(), out);
 }
 
 // Eq. 13
@@ -415,6 +509,47 @@ void refit(const float *W, uint32_t R, uint32_t C, const int32_t *fields, float 
     });
 }
 
+
+// ---- the host back end: everything on CPU threads ------------------------------------------------------
+class HostBackend final : public EncodeBackend {
+public:
+    HostBackend(const float *W, uint32_t R, uint32_t C, int threads) : W_(W), R_(R), C_(C), threads_(threads) {}
+
+    int prepare(const std::vector<uint32_t> &sample) override {
+        rows_ = sample;
+        mu_.resize(R_);
+        parallel_for(R_, threads_, [&](uint64_t lo, uint64_t hi, int) {
+            for (uint64_t r = lo; r < hi; ++r) mu_[r] = row_rms(W_ + r * C_, C_);
+        });
+        sfields_.resize(size_t(rows_.size()) * (C_ / 8) * 9);
+        fields_.resize(size_t(R_) * (C_ / 8) * 9);
+        return EP_OK;
+    }
+    int count_sample(float s, Model &m) override {
+        quantise_rows(W_, C_, mu_.data(), rows_.data(), rows_.size(), s, sfields_.data(), threads_);
+        m.count(sfields_.data(), uint64_t(rows_.size()) * (C_ / 8), threads_);
+        return EP_OK;
+    }
+    int count_full(float s, Model &m) override {
+        quantise_rows(W_, C_, mu_.data(), nullptr, R_, s, fields_.data(), threads_);
+        m.count(fields_.data(), uint64_t(R_) * (C_ / 8), threads_);
+        return EP_OK;
+    }
+    int finish(float s, int b, uint32_t V, const Model &m, ep_blob *out) override {
+        std::vector<float> sigma(R_);
+        refit(W_, R_, C_, fields_.data(), s, mu_.data(), sigma.data(), threads_);
+        return pack_fields_host(fields_.data(), R_, C_, b, V, m, sigma.data(), s, threads_, out);
+    }
+
+private:
+    const float *W_;
+    uint32_t R_, C_;
+    int threads_;
+    std::vector<uint32_t> rows_;
+    std::vector<float> mu_;
+    std::vector<int32_t> sfields_, fields_;
+};
+
 }  // namespace
 }  // namespace ep
 
@@ -435,114 +570,28 @@ extern "C" void ep_encode_opts_default(ep_encode_opts *o) {
     o->threads = 0;
 }
 
+namespace ep {
+int check_encode_args(uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts &o) {
+    if (R == 0 || C == 0 || C % 8 != 0 || !(target_bpp > 0.0)) return EP_ERR_BAD_ARG;
+    if (uint64_t(R) * (C / 8) >= (1ull << 32)) return EP_ERR_BAD_ARG;
+    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.polish_steps < 0 || o.b_max > 15 ||
+        o.b_max < 9 || (o.b_start != 0 && (o.b_start < 9 || o.b_start > o.b_max)))
+        return EP_ERR_BAD_ARG;
+    return EP_OK;
+}
+}  // namespace ep
+
 extern "C" int ep_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts_in,
                          ep_blob **out) {
     using namespace ep;
-    if (!W || !out || R == 0 || C == 0 || C % 8 != 0 || !(target_bpp > 0.0)) return EP_ERR_BAD_ARG;
-    const uint64_t nvec = uint64_t(R) * (C / 8);
-    if (nvec >= (1ull << 32)) return EP_ERR_BAD_ARG;
+    if (!W || !out) return EP_ERR_BAD_ARG;
     ep_encode_opts o;
     if (opts_in) o = *opts_in; else ep_encode_opts_default(&o);
-    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.polish_steps < 0 || o.b_max > 15 || o.b_max < 9 ||
-        (o.b_start != 0 && (o.b_start < 9 || o.b_start > o.b_max)))
-        return EP_ERR_BAD_ARG;
+    const int bad = check_encode_args(R, C, target_bpp, o);
+    if (bad) return bad;
     try {
-        const int threads = resolve_threads(o.threads);
-        const uint32_t V = o.tile_vectors ? o.tile_vectors : ep_default_tile_vectors(target_bpp);
-        int b = o.b_start ? o.b_start : (target_bpp <= 7.0 ? 11 : 12);
-        b = std::min(b, o.b_max);
-        std::vector<float> mu(R);
-        parallel_for(R, threads, [&](uint64_t lo, uint64_t hi, int) {
-            for (uint64_t r = lo; r < hi; ++r) mu[r] = row_rms(W + r * C, C);
-        });
-        const std::vector<uint32_t> rows = sample_rows(R, C, o.sample_vectors);
-        const uint64_t svec = uint64_t(rows.size()) * (C / 8);
-        std::vector<int32_t> sfields(size_t(svec) * 9), fields(size_t(nvec) * 9);
-        float s = 0.0f;
-        double last_rate = 0.0;
-        for (;; ++b) {
-            double lo = o.bracket_lo, hi = o.bracket_hi;
-            for (int it = 0; it < o.search_steps; ++it) {
-                const double mid = std::sqrt(lo * hi);
-                quantise_rows(W, C, mu.data(), rows.data(), rows.size(), float(mid), sfields.data(), threads);
-                Model m;
-                m.count(sfields.data(), svec, threads);
-                m.normalise(b);
-                const double bits = estimate_bits(m, b, svec, rows.size(), V, o.retained_bits, nullptr);
-                last_rate = bits / (8.0 * double(svec));
-                if (last_rate > target_bpp) lo = mid; else hi = mid;
-            }
-            s = float(std::sqrt(lo * hi));
-            bool fits = false;
-            for (;;) {
-                quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
-                Model m;
-                m.count(fields.data(), nvec, threads);
-                uint32_t worst = 0, amax = 0;
-                for (int i = 0; i < EP_NUM_TABLES; ++i) {
-                    const uint32_t ob = m.t[i].observed();
-                    worst = std::max(worst, ob);
-                    if (i > 0) amax = std::max(amax, ob);
-                }
-                if (worst <= (1u << b)) { fits = true; break; }
-                if (b < o.b_max) break;
-                s = float(1.05 * double(s) * double(amax) / double(1u << b));
-            }
-            if (fits) break;
-        }
-        // Beyond Algorithm 1: steer s with the full-tensor estimate (Eq. 10-11), first by the one-bit-per-doubling
-        // law (Eq. 9), then by the measured slope.  The sampled tables miss rare symbols of the full tensor, which costs rate on heavy tails.
-        struct { double log_s, rate; bool valid; } last{0.0, 0.0, false};
-        for (int step = 0; step < o.polish_steps; ++step) {
-            double est;
-            {
-                Model m;
-                m.count(fields.data(), nvec, threads);
-                m.normalise(b);
-                est = estimate_bits(m, b, nvec, R, V, o.polish_retained_bits, nullptr) / (double(R) * double(C));
-            }
-            if (std::fabs(est - target_bpp) <= 0.002 * target_bpp) break;
-            // rate lost per doubling of s: 1 bit by Eq. 9 for the first move, afterwards the secant slope
-            const double log_s = std::log2(double(s));
-            double per_doubling = 1.0;
-            if (last.valid && log_s != last.log_s) {
-                per_doubling = -(est - last.rate) / (log_s - last.log_s);
-                if (!(per_doubling >= 0.5)) per_doubling = 0.5;
-                if (per_doubling > 4.0) per_doubling = 4.0;
-            }
-            last = {log_s, est, true};
-            const float before = s;
-            double moved = std::exp2(log_s + (est - target_bpp) / per_doubling);
-            if (!(moved >= o.bracket_lo)) moved = o.bracket_lo;   // never leave the search bracket
-            if (moved > o.bracket_hi) moved = o.bracket_hi;
-            s = float(moved);
-            if (s == before) break;
-            quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
-            Model m;
-            m.count(fields.data(), nvec, threads);
-            uint32_t worst = 0;
-            for (const auto &tb : m.t) worst = std::max(worst, tb.observed());
-            if (worst > (1u << b)) {   // the finer scale overflows the tables: undo and stop
-                s = before;
-                quantise_rows(W, C, mu.data(), nullptr, R, s, fields.data(), threads);
-                break;
-            }
-        }
-        std::vector<float> sigma(R);
-        refit(W, R, C, fields.data(), s, mu.data(), sigma.data(), threads);
-        ep_blob *blob = new ep_blob();
-        double cce = 0.0;
-        const int rc = pack(fields.data(), R, C, b, V, sigma.data(), s, threads, blob, &cce);
-        if (rc) { delete blob; return rc; }
-        blob->report.s = double(s);
-        blob->report.b = b;
-        blob->report.bytes = blob->bytes.size();
-        blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
-        blob->report.est_bpp_sample = last_rate;
-        blob->report.cce_bits = cce;
-        blob->report.sample_rows = uint32_t(rows.size());
-        *out = blob;
-        return EP_OK;
+        HostBackend be(W, R, C, resolve_threads(o.threads));
+        return run_encode(be, R, C, target_bpp, o, out);
     } catch (const std::bad_alloc &) {
         return EP_ERR_NOMEM;
     } catch (...) {
@@ -559,15 +608,19 @@ extern "C" int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int
     for (uint64_t v = 0; v < nvec; ++v)
         if (fields[9 * v] != 0 && fields[9 * v] != 1) return EP_ERR_BAD_ARG;
     try {
+        const int T = resolve_threads(threads);
+        Model m;
+        m.count(fields, nvec, T);
+        if (m.worst_observed() > (1u << b)) return EP_ERR_UNSUPPORTED;
+        m.normalise(b);
         ep_blob *blob = new ep_blob();
-        double cce = 0.0;
-        const int rc = pack(fields, R, C, b, V, row_scales, s_info, resolve_threads(threads), blob, &cce);
+        const int rc = pack_fields_host(fields, R, C, b, V, m, row_scales, s_info, T, blob);
         if (rc) { delete blob; return rc; }
         blob->report.s = double(s_info);
         blob->report.b = b;
         blob->report.bytes = blob->bytes.size();
         blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
-        blob->report.cce_bits = cce;
+        blob->report.cce_bits = m.cross_entropy_bits(b);
         *out = blob;
         return EP_OK;
     } catch (const std::bad_alloc &) {
