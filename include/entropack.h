@@ -151,6 +151,17 @@ int ep_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const e
 int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int32_t b, uint32_t V,
                    const float *row_scales, float s_info, int32_t threads, ep_blob **out);
 
+/* The same encoder with the heavy steps on the GPU (row RMS, E8 quantisation and field histograms, Eq. 13,
+ * tile coding); the search itself and the table arithmetic stay on the host, so the result is byte for
+ * byte the blob ep_encode produces for the same W and options.  d_W is a device copy of W (16-byte
+ * aligned), d_workspace a 256-byte aligned device buffer of ep_encode_device_workspace_bytes() bytes
+ * (about 54 bytes per 8-weight block).  The call enqueues on `stream` and synchronises it several times;
+ * it returns the finished host blob.  EP_ERR_UNSUPPORTED (use ep_encode instead) if a lattice coordinate
+ * exceeds +-4095 or the tables hold more than 40960 symbols in total. */
+size_t ep_encode_device_workspace_bytes(uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts);
+int ep_encode_device(const float *d_W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts,
+                     void *d_workspace, size_t workspace_bytes, void *stream, ep_blob **out);
+
 const void *ep_blob_data(const ep_blob *blob);   /* host pointer valid until ep_blob_free */
 size_t ep_blob_bytes(const ep_blob *blob);       /* B_stored of Eq. 1 */
 int ep_blob_report(const ep_blob *blob, ep_encode_report *out);

@@ -78,6 +78,10 @@ def load():
     L.ep_encode.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_double, C.POINTER(EncodeOpts), C.POINTER(C.c_void_p)]
     L.ep_pack_fields.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_int32, C.c_uint32, C.c_void_p, C.c_float,
                                  C.c_int32, C.POINTER(C.c_void_p)]
+    L.ep_encode_device_workspace_bytes.restype = C.c_size_t
+    L.ep_encode_device_workspace_bytes.argtypes = [C.c_uint32, C.c_uint32, C.c_double, C.POINTER(EncodeOpts)]
+    L.ep_encode_device.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_double, C.POINTER(EncodeOpts), C.c_void_p,
+                                   C.c_size_t, C.c_void_p, C.POINTER(C.c_void_p)]
     L.ep_blob_data.restype = C.c_void_p
     L.ep_blob_data.argtypes = [C.c_void_p]
     L.ep_blob_bytes.restype = C.c_size_t
@@ -170,6 +174,22 @@ def encode(W: np.ndarray, target_bpp: float, **opts) -> Blob:
     o = encode_opts(**opts)
     h = C.c_void_p()
     _check(load().ep_encode(W.ctypes.data, W.shape[0], W.shape[1], float(target_bpp), C.byref(o), C.byref(h)), "ep_encode")
+    return _take(h)
+
+
+def encode_device(W_dev, target_bpp: float, workspace=None, stream=None, **opts) -> Blob:
+    """ep_encode_device: the encoder with its heavy steps on the GPU.  W_dev is a CUDA float32 tensor [R, C];
+    the result is the same host blob ep_encode gives for the same matrix and options."""
+    torch = _torch()
+    assert W_dev.is_cuda and W_dev.dtype == torch.float32 and W_dev.dim() == 2 and W_dev.is_contiguous()
+    R, Cc = W_dev.shape
+    o = encode_opts(**opts)
+    need = load().ep_encode_device_workspace_bytes(R, Cc, float(target_bpp), C.byref(o))
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=W_dev.device)
+    h = C.c_void_p()
+    _check(load().ep_encode_device(W_dev.data_ptr(), R, Cc, float(target_bpp), C.byref(o), workspace.data_ptr(),
+                                   workspace.numel(), _stream_handle(stream), C.byref(h)), "ep_encode_device")
     return _take(h)
 
 
