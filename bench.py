@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp8", "int8"])
     ap.add_argument("--layers", type=int, default=48, help="c5: resident layers")
     ap.add_argument("--distinct-layers", type=int, default=2, help="c5: distinct layers actually encoded")
+    ap.add_argument("--sweep", action="store_true",
+                    help="c4 only: after the main line's measurement also time every target rate 2.0, 2.5 .. 6.0 "
+                         "(throughput and stored vs target bpp per rate, in the JSON key 'sweep')")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -278,12 +281,15 @@ def main():
     launches_per_step = sum((len(r) + ep.binding.MAX_BATCH - 1) // ep.binding.MAX_BATCH for r in resident)
     stream = torch.cuda.current_stream()
 
+    def decode_layer(l):
+        if len(resident[l]) == 1:
+            ep.decode(resident[l][0], DT, out=outs_by_layer[l][0], stream=stream)
+        else:
+            ep.decode_many(resident[l], DT, outs_by_layer[l], stream=stream)
+
     def step():
         for l in range(n_layers):
-            if len(resident[l]) == 1:
-                ep.decode(resident[l][0], DT, out=outs_by_layer[l][0], stream=stream)
-            else:
-                ep.decode_many(resident[l], DT, outs_by_layer[l], stream=stream)
+            decode_layer(l)
 
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
 
@@ -376,6 +382,51 @@ def main():
                "d2h_bytes_per_step": d2h, "ms_per_step": ms,
                "what": "one layer: pinned host blob -> device, decode, decoded tensor -> pinned host"}
 
+    # per-layer device times of one more pass (config 5 asks for total and per-layer decode time)
+    per_layer_ms = None
+    if n_layers > 1:
+        pev = [torch.cuda.Event(enable_timing=True) for _ in range(n_layers + 1)]
+        pev[0].record(stream)
+        for l in range(n_layers):
+            decode_layer(l)
+            pev[l + 1].record(stream)
+        barrier()
+        per_layer_ms = [pev[l].elapsed_time(pev[l + 1]) for l in range(n_layers)]
+
+    # relative L2 error of the decoded first tensor against its source (Eq. 1; reporting only, torch fp64 on the GPU)
+    d0, W0 = resident[0][0], torch.from_numpy(layers[0][0]).to(dev)
+    got0 = ep.decode(d0, DT, out=outs_by_layer[0][0], stream=stream)
+    torch.cuda.synchronize()
+    g64, w64 = got0.to(torch.float64), W0.to(torch.float64)
+    rel_l2_first = float(torch.sqrt(((g64 - w64) ** 2).sum() / (w64 ** 2).sum()).item())
+    del g64, w64, W0
+
+    sweep = None
+    if args.sweep and args.workload == "c4" and rank == 0:
+        sweep = []
+        W = layers[0][0]
+        for r in (2.0, 2.5, 3.0, 3.5, 4.0, 4.5, 5.0, 5.5, 6.0):
+            V = pick_tile_vectors(args.tile_vectors, W.shape, r, slots)
+            bl = ep.encode(W, r, tile_vectors=V)
+            dd = ep.upload(bl, device=dev)
+            for _ in range(3):
+                ep.decode(dd, DT, out=outs_by_layer[0][0], stream=stream)
+            ts = []
+            for _ in range(15):                      # the paper's protocol: minimum of fifteen after three warm-ups
+                flush.fill_(0)
+                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                ep.decode(dd, DT, out=outs_by_layer[0][0], stream=stream)
+                b_.record(stream)
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b_))
+            med = statistics.median(ts)
+            nbytes = len(bl) + W.size * esize
+            sweep.append({"target_bpp": r, "stored_bpp": bl.stored_bpp, "tile_vectors": bl.info.V, "min_ms": min(ts),
+                          "median_ms": med, "Gparams_per_s": W.size / (med * 1e-3) / 1e9,
+                          "effective_GBps": nbytes / (med * 1e-3) / 1e9})
+            del dd
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -419,9 +470,10 @@ def main():
                        "tiles_first_tensor": b0.info.n_tiles, "b": b0.info.b, "out_dtype": dtype_name,
                        "params_per_step": params_per_step, "l2": "flushed between timed steps (512 MB write)",
                        "min_ms": min(times_ms), "median_ms": statistics.median(times_ms),
-                       "warm_ms_per_step_no_flush": warm_ms},
+                       "warm_ms_per_step_no_flush": warm_ms, "rel_l2_first_tensor": rel_l2_first},
             "effective_GBps": eff_gbs, "pct_of_measured_hbm": 100.0 * eff_gbs / peak, "pct_of_8TBps": 100.0 * eff_gbs / 8000.0,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+            "per_layer_ms": per_layer_ms, "sweep": sweep,
             "clocks": clocks}
     print(json.dumps(line), flush=True)
     if world > 1:
