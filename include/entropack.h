@@ -89,6 +89,10 @@ typedef struct {
     double polish_retained_bits;   /* bits per state taken as retained in those corrections: 8 (states end up
                                       spread over [2^15, 2^31), so about 8 bits each stay out of the payload) */
     int32_t threads;               /* host worker threads; 0 = all hardware threads */
+    int32_t rdo_candidates;        /* K of the per-row rate-distortion refinement (Sec. 3.5, Alg. 2): candidate
+                                      scales rho_k * s per row, rho in [0.70, 1.45]; 1 = off (the paper's default).
+                                      Host encoder only */
+    int32_t rdo_sweeps;            /* T allocation / model-update sweeps: 1 */
 } ep_encode_opts;
 
 /* What the encoder decided; filled by ep_blob_report(). */

@@ -35,7 +35,7 @@ class Opts(C.Structure):
     _fields_ = [("bracket_lo", C.c_double), ("bracket_hi", C.c_double), ("search_steps", C.c_int32),
                 ("sample_vectors", C.c_uint32), ("tile_vectors", C.c_uint32), ("b_start", C.c_int32),
                 ("b_max", C.c_int32), ("retained_bits", C.c_double), ("polish_steps", C.c_int32),
-                ("polish_retained_bits", C.c_double)]
+                ("polish_retained_bits", C.c_double), ("rdo_candidates", C.c_int32), ("rdo_sweeps", C.c_int32)]
 
 
 class Report(C.Structure):
@@ -116,6 +116,13 @@ def point2_from_fields(f: np.ndarray) -> np.ndarray:
     q = np.zeros(8, np.int32)
     lib().epo_point2_from_fields(_p(f), _p(q))
     return q
+
+
+def rdo_ratios(K: int) -> np.ndarray:
+    """The K nested candidate ratios of the per-row refinement."""
+    out = np.zeros(max(K, 1), np.float64)
+    lib().epo_rdo_ratios(C.c_int(K), _p(out))
+    return out[:K]
 
 
 def quantise(W: np.ndarray, s: float):

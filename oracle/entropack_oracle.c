@@ -14,6 +14,7 @@
  *   stored-size estimate             Eq. 10, Eq. 11
  *   sampled geometric scale search   Eq. 12, Algorithm 1, App. "Scale-search settings"
  *   row-scale refit                  Eq. 13
+ *   per-row RDO refinement (optional) Sec. 3.5, Eq. 14-16, Algorithm 2
  *   tiled 32-state rANS encode       Eq. 17, App. "Tiled rANS implementation"
  *   rANS decode + reconstruction     Eq. 18, Eq. 5, Eq. 19
  *   relative L2 error, stored rate   Eq. 1
@@ -28,7 +29,9 @@
  * Parity unpinned by the paper (fixed only by this build's stated readings):
  * the coset tie rule, the integer frequency-normalisation rule, the row
  * sampler, default tile size between the listed targets, the byte layout of
- * tables and header.
+ * tables and header, the full-tensor rate correction after Algorithm 1, and
+ * the open details of Algorithm 2 (candidate ratios, smoothing range, the
+ * initial rate penalty).
  *
  * Parallelism: OpenMP over rows (quantisation) and over tiles (coding) only;
  * the arithmetic of one row / one tile is untouched by it.
@@ -61,6 +64,8 @@ typedef struct {
     int32_t polish_steps;          /* full-tensor corrections of s after Algorithm 1 (not in the paper), default 3 */
     double polish_retained_bits;   /* bits per state assumed retained in those corrections: 8, the measured mean
                                       of log2(final state / 2^15) for states spread over [2^15, 2^31) */
+    int32_t rdo_candidates;        /* K of the per-row refinement (Sec. 3.5, Alg. 2); 1 = off (the paper's default) */
+    int32_t rdo_sweeps;            /* T, default 1 */
 } epo_opts;
 
 typedef struct {
@@ -101,6 +106,8 @@ void epo_default_opts(epo_opts *o) {
     o->retained_bits = 16.0;
     o->polish_steps = 3;
     o->polish_retained_bits = 8.0;
+    o->rdo_candidates = 1;
+    o->rdo_sweeps = 1;
 }
 
 void epo_free(void *p) { free(p); }
@@ -812,6 +819,191 @@ void epo_refit(const float *W, uint32_t R, uint32_t C, const int32_t *fields, fl
     }
 }
 
+/* ------------------------- Sec. 3.5 / Alg. 2: per-row rate-distortion refinement */
+
+/* K nested candidate ratios in [0.70, 1.45]: 1 first, then the log-midpoint of the widest remaining
+ * interval (the first one on ties; the two bounds themselves are never candidates - reading). */
+void epo_rdo_ratios(int K, double *rho) {
+    double pts[80];
+    int n = 3;
+    pts[0] = log(0.70); pts[1] = 0.0; pts[2] = log(1.45);
+    rho[0] = 1.0;
+    for (int i = 1; i < K && i < 64; ++i) {
+        int best = 0;
+        double w = -1.0;
+        for (int j = 0; j + 1 < n; ++j) { double d = pts[j + 1] - pts[j]; if (d > w) { w = d; best = j; } }
+        double mid = 0.5 * (pts[best] + pts[best + 1]);
+        for (int j = n; j > best + 1; --j) pts[j] = pts[j - 1];
+        pts[best + 1] = mid;
+        ++n;
+        rho[i] = exp(mid);
+    }
+}
+
+/* kappa_lambda(r) = argmin_k D + lambda R (first k on ties); returns L(lambda) = sum_r R[r][kappa] */
+static double rdo_choose(const double *D, const double *Rr, uint32_t R, int K, double lambda, int *choice) {
+    double L = 0.0;
+    for (uint32_t r = 0; r < R; ++r) {
+        int bk = 0;
+        double bv = D[(size_t)r * K] + lambda * Rr[(size_t)r * K];
+        for (int k = 1; k < K; ++k) {
+            double v = D[(size_t)r * K + k] + lambda * Rr[(size_t)r * K + k];
+            if (v < bv) { bv = v; bk = k; }
+        }
+        choice[r] = bk;
+        L += Rr[(size_t)r * K + bk];
+    }
+    return L;
+}
+
+/* Refines `fields` (the baseline quantisation at scale s) and `sigma` in place.  Candidates k = 0..K-1 use
+ * scales rho_k * s; each is refit with Eq. 13; D[r][k] is the row's squared error with the stored fp32 scale.
+ * T sweeps alternate between a shared model fitted to the current selections (counts + 1/2 over the value
+ * range spanned by all candidates, per table) and a common rate penalty lambda that keeps the modelled code
+ * length within the budget of Eq. 15.  If the refined tensor's alphabets no longer fit 2^b the baseline is
+ * kept. */
+static void rdo_refine(const float *W, uint32_t R, uint32_t C, const float *mu, float s, int b, uint32_t V,
+                       const epo_opts *o, int32_t *fields, float *sigma) {
+    const int K = o->rdo_candidates > 64 ? 64 : o->rdo_candidates;
+    const uint32_t per_row = C / 8;
+    const uint64_t nvec = (uint64_t)R * per_row;
+    double rho[64];
+    epo_rdo_ratios(K, rho);
+    int32_t **cf = (int32_t **)malloc(sizeof(int32_t *) * K);
+    float **cs = (float **)malloc(sizeof(float *) * K);
+    double *D = (double *)malloc(sizeof(double) * (size_t)R * K);
+    double *Rr = (double *)malloc(sizeof(double) * (size_t)R * K);
+    for (int k = 0; k < K; ++k) {
+        cf[k] = (int32_t *)malloc(sizeof(int32_t) * 9 * nvec);
+        cs[k] = (float *)malloc(sizeof(float) * R);
+        if (k == 0) { memcpy(cf[0], fields, sizeof(int32_t) * 9 * nvec); memcpy(cs[0], sigma, sizeof(float) * R); }
+        else {
+            float sk = (float)(rho[k] * (double)s);
+#pragma omp parallel for schedule(static)
+            for (int64_t r = 0; r < (int64_t)R; ++r)
+                quantise_row(W + (size_t)r * C, C, mu[r], sk, cf[k] + 9 * (size_t)r * per_row);
+            epo_refit(W, R, C, cf[k], sk, mu, cs[k]);
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < (int64_t)R; ++r) {
+            double acc = 0.0;
+            for (uint32_t v = 0; v < per_row; ++v) {
+                int32_t q[8];
+                epo_point2_from_fields(cf[k] + 9 * ((size_t)r * per_row + v), q);
+                for (int j = 0; j < 8; ++j) {
+                    double d = (double)W[(size_t)r * C + 8 * v + j] - (double)cs[k][r] * (0.5 * (double)q[j]);
+                    acc += d * d;
+                }
+            }
+            D[(size_t)r * K + k] = acc;
+        }
+    }
+    /* value range of every table over all candidates */
+    int32_t lo[EPO_NT], hi[EPO_NT];
+    int used[EPO_NT];
+    for (int i = 0; i < EPO_NT; ++i) { used[i] = 0; lo[i] = hi[i] = 0; }
+    for (int k = 0; k < K; ++k)
+        for (uint64_t v = 0; v < nvec; ++v) {
+            const int32_t *a = cf[k] + 9 * v;
+            for (int j = 0; j < 9; ++j) {
+                int ti = tab_of(a[0], j);
+                if (!used[ti]) { used[ti] = 1; lo[ti] = hi[ti] = a[j]; }
+                else { if (a[j] < lo[ti]) lo[ti] = a[j]; if (a[j] > hi[ti]) hi[ti] = a[j]; }
+            }
+        }
+    double *nl[EPO_NT];
+    uint64_t *cnt[EPO_NT];
+    for (int i = 0; i < EPO_NT; ++i) {
+        size_t w = used[i] ? (size_t)((int64_t)hi[i] - lo[i] + 1) : 0;
+        nl[i] = (double *)malloc(sizeof(double) * (w ? w : 1));
+        cnt[i] = (uint64_t *)malloc(sizeof(uint64_t) * (w ? w : 1));
+    }
+    int *sel = (int *)calloc(R, sizeof(int)), *khat = (int *)malloc(sizeof(int) * R), *tmp = (int *)malloc(sizeof(int) * R);
+    int32_t *mix = (int32_t *)malloc(sizeof(int32_t) * 9 * nvec);
+    epo_tab t[EPO_NT];
+    tabs_count(cf[0], nvec, t);
+    tabs_normalise(t, b);
+    const double B = estimate_bits(t, b, nvec, R, V, o->retained_bits, NULL) / 8.0;   /* the baseline's estimated bytes */
+    tabs_free(t);
+    for (int sweep = 0; sweep < o->rdo_sweeps; ++sweep) {
+        for (uint32_t r = 0; r < R; ++r)
+            memcpy(mix + 9 * (size_t)r * per_row, cf[sel[r]] + 9 * (size_t)r * per_row, sizeof(int32_t) * 9 * per_row);
+        /* shared model of the current selections, half a count added to every value of the spanned range */
+        uint64_t tot[EPO_NT];
+        for (int i = 0; i < EPO_NT; ++i) {
+            tot[i] = 0;
+            if (used[i]) memset(cnt[i], 0, sizeof(uint64_t) * (size_t)((int64_t)hi[i] - lo[i] + 1));
+        }
+        for (uint64_t v = 0; v < nvec; ++v) {
+            const int32_t *a = mix + 9 * v;
+            for (int j = 0; j < 9; ++j) { int ti = tab_of(a[0], j); cnt[ti][a[j] - lo[ti]]++; tot[ti]++; }
+        }
+        for (int i = 0; i < EPO_NT; ++i) {
+            if (!used[i]) continue;
+            size_t w = (size_t)((int64_t)hi[i] - lo[i] + 1);
+            double den = (double)tot[i] + 0.5 * (double)w;
+            for (size_t z = 0; z < w; ++z) nl[i][z] = -log2(((double)cnt[i][z] + 0.5) / den);
+        }
+        /* Eq. 14 for every row and candidate */
+#pragma omp parallel for schedule(static)
+        for (int64_t r = 0; r < (int64_t)R; ++r)
+            for (int k = 0; k < K; ++k) {
+                double acc = 0.0;
+                for (uint32_t v = 0; v < per_row; ++v) {
+                    const int32_t *a = cf[k] + 9 * ((size_t)r * per_row + v);
+                    for (int j = 0; j < 9; ++j) { int ti = tab_of(a[0], j); acc += nl[ti][a[j] - lo[ti]]; }
+                }
+                Rr[(size_t)r * K + k] = acc;
+            }
+        /* Eq. 15: budget from the baseline's estimated bytes and the current mixture's */
+        tabs_count(mix, nvec, t);
+        uint32_t worst = 0;
+        for (int i = 0; i < EPO_NT; ++i) { uint32_t ob = tabs_observed(t, i); if (ob > worst) worst = ob; }
+        if (worst > (1u << b)) { tabs_free(t); break; }
+        tabs_normalise(t, b);
+        const double Bmix = estimate_bits(t, b, nvec, R, V, o->retained_bits, NULL) / 8.0;
+        tabs_free(t);
+        double cur = 0.0, dcur = 0.0;
+        for (uint32_t r = 0; r < R; ++r) { cur += Rr[(size_t)r * K + sel[r]]; dcur += D[(size_t)r * K + sel[r]]; }
+        const double budget = cur + 8.0 * (B - Bmix);
+        /* Eq. 16 with a common lambda */
+        double L = rdo_choose(D, Rr, R, K, 0.0, khat);
+        if (L > budget) {
+            double lam_lo = 0.0, lam_hi = (cur > 0.0 && dcur > 0.0) ? dcur / cur : 1e-12;
+            int ok = 0;
+            for (int d = 0; d < 64; ++d) {
+                if (rdo_choose(D, Rr, R, K, lam_hi, tmp) <= budget) { ok = 1; break; }
+                lam_lo = lam_hi;
+                lam_hi *= 2.0;
+            }
+            if (ok) {
+                memcpy(khat, tmp, sizeof(int) * R);
+                for (int it = 0; it < 20; ++it) {
+                    double lam = (lam_lo == 0.0) ? 0.5 * lam_hi : sqrt(lam_lo * lam_hi);
+                    if (rdo_choose(D, Rr, R, K, lam, tmp) > budget) lam_lo = lam;
+                    else { lam_hi = lam; memcpy(khat, tmp, sizeof(int) * R); }
+                }
+            } else {
+                memcpy(khat, sel, sizeof(int) * R);     /* no penalty meets the budget: keep the current selection */
+            }
+        }
+        memcpy(sel, khat, sizeof(int) * R);
+    }
+    for (uint32_t r = 0; r < R; ++r)
+        memcpy(mix + 9 * (size_t)r * per_row, cf[sel[r]] + 9 * (size_t)r * per_row, sizeof(int32_t) * 9 * per_row);
+    tabs_count(mix, nvec, t);
+    uint32_t worst = 0;
+    for (int i = 0; i < EPO_NT; ++i) { uint32_t ob = tabs_observed(t, i); if (ob > worst) worst = ob; }
+    tabs_free(t);
+    if (worst <= (1u << b)) {
+        memcpy(fields, mix, sizeof(int32_t) * 9 * nvec);
+        for (uint32_t r = 0; r < R; ++r) sigma[r] = cs[sel[r]][r];
+    }
+    for (int i = 0; i < EPO_NT; ++i) { free(nl[i]); free(cnt[i]); }
+    for (int k = 0; k < K; ++k) { free(cf[k]); free(cs[k]); }
+    free(cf); free(cs); free(D); free(Rr); free(sel); free(khat); free(tmp); free(mix);
+}
+
 /* --------------------------------- Algorithm 1 + packing: the whole encoder */
 int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const epo_opts *opts_in,
                uint8_t **blob_out, size_t *n_out, epo_report *rep) {
@@ -914,6 +1106,7 @@ int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const 
     }
     float *sigma = (float *)malloc(sizeof(float) * R);
     epo_refit(W, R, C, fields, s32, mu, sigma);
+    if (o.rdo_candidates > 1) rdo_refine(W, R, C, mu, s32, b, V, &o, fields, sigma);
     double cce = 0.0;
     int rc = epo_pack(fields, R, C, b, V, sigma, s32, blob_out, n_out, &cce);
     if (!rc && rep) {

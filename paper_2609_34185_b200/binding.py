@@ -31,7 +31,7 @@ class EncodeOpts(C.Structure):
     _fields_ = [("bracket_lo", C.c_double), ("bracket_hi", C.c_double), ("search_steps", C.c_int32),
                 ("sample_vectors", C.c_uint32), ("tile_vectors", C.c_uint32), ("b_start", C.c_int32),
                 ("b_max", C.c_int32), ("retained_bits", C.c_double), ("polish_steps", C.c_int32), ("polish_retained_bits", C.c_double),
-                ("threads", C.c_int32)]
+                ("threads", C.c_int32), ("rdo_candidates", C.c_int32), ("rdo_sweeps", C.c_int32)]
 
 
 class EncodeReport(C.Structure):

@@ -269,6 +269,22 @@ int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, con
     return EP_OK;
 }
 
+// ---- Sec. 3.5 / Alg. 2: candidate ratios ---------------------------------------------------------------
+std::vector<double> rdo_ratios(int K) {
+    std::vector<double> cut = {std::log(0.70), 0.0, std::log(1.45)};   // sorted log-points, the two bounds included
+    std::vector<double> rho = {1.0};
+    while (int(rho.size()) < K) {
+        size_t at = 0;
+        double widest = -1.0;
+        for (size_t j = 0; j + 1 < cut.size(); ++j)
+            if (cut[j + 1] - cut[j] > widest) { widest = cut[j + 1] - cut[j]; at = j; }   // first one on ties
+        const double mid = 0.5 * (cut[at] + cut[at + 1]);
+        cut.insert(cut.begin() + long(at) + 1, mid);
+        rho.push_back(std::exp(mid));
+    }
+    return rho;
+}
+
 // ---- Algorithm 1 + rate correction + packing, over a back end ---------------------------------------
 int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts &o, ep_blob **out) {
     const uint64_t nvec = uint64_t(R) * (C / 8);
@@ -334,6 +350,7 @@ int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, con
             break;
         }
     }
+    if (o.rdo_candidates > 1 && (rc = be.refine(s, b, V, o, full))) return rc;
     full.normalise(b);
     ep_blob *blob = new ep_blob();
     rc = be.finish(s, b, V, full, blob);
@@ -537,8 +554,158 @@ public:
     }
     int finish(float s, int b, uint32_t V, const Model &m, ep_blob *out) override {
         std::vector<float> sigma(R_);
-        refit(W_, R_, C_, fields_.data(), s, mu_.data(), sigma.data(), threads_);
+        if (refined_sigma_.empty()) refit(W_, R_, C_, fields_.data(), s, mu_.data(), sigma.data(), threads_);
+        else sigma = refined_sigma_;
         return pack_fields_host(fields_.data(), R_, C_, b, V, m, sigma.data(), s, threads_, out);
+    }
+
+    // Sec. 3.5 / Alg. 2.  Candidate k quantises every row at rho_k * s and refits its scale (Eq. 13); D is the
+    // row's squared error with the stored fp32 scale.  Each sweep fits one shared model to the rows' current
+    // choices (every value of the range spanned by all candidates gets half a count more), prices every
+    // candidate (Eq. 14), sets the budget of Eq. 15 from the baseline's and the mixture's estimated bytes, and
+    // picks per row argmin D + lambda R (Eq. 16) with the smallest common lambda found that meets the budget.
+    int refine(float s, int b, uint32_t V, const ep_encode_opts &o, Model &m) override {
+        const int K = o.rdo_candidates;
+        const uint32_t per_row = C_ / 8;
+        const uint64_t nvec = uint64_t(R_) * per_row;
+        const std::vector<double> rho = rdo_ratios(K);
+        struct Candidate { std::vector<int32_t> fields; std::vector<float> sigma; };
+        std::vector<Candidate> cand(K);
+        std::vector<double> D(size_t(R_) * K), cost(size_t(R_) * K);
+        for (int k = 0; k < K; ++k) {
+            Candidate &c = cand[k];
+            c.sigma.resize(R_);
+            if (k == 0) {
+                c.fields = fields_;
+                refit(W_, R_, C_, c.fields.data(), s, mu_.data(), c.sigma.data(), threads_);
+            } else {
+                const float sk = float(rho[k] * double(s));
+                c.fields.resize(size_t(nvec) * 9);
+                quantise_rows(W_, C_, mu_.data(), nullptr, R_, sk, c.fields.data(), threads_);
+                refit(W_, R_, C_, c.fields.data(), sk, mu_.data(), c.sigma.data(), threads_);
+            }
+            parallel_for(R_, threads_, [&](uint64_t lo, uint64_t hi, int) {
+                for (uint64_t r = lo; r < hi; ++r) {
+                    double err = 0.0;
+                    const double sg = double(c.sigma[r]);
+                    for (uint32_t v = 0; v < per_row; ++v) {
+                        const int32_t *q = c.fields.data() + 9 * (r * per_row + v);
+                        int32_t s7 = 0, two_p[8];
+                        for (int j = 0; j < 7; ++j) { two_p[j] = 2 * q[1 + j] + q[0]; s7 += q[1 + j]; }
+                        two_p[7] = 2 * (2 * q[8] + (s7 & 1)) + q[0];
+                        for (int j = 0; j < 8; ++j) {
+                            const double d = double(W_[r * C_ + 8 * v + j]) - sg * (0.5 * double(two_p[j]));
+                            err += d * d;
+                        }
+                    }
+                    D[r * K + k] = err;
+                }
+            });
+        }
+        // value range of every table over all candidates
+        int64_t lo[EP_NUM_TABLES], hi[EP_NUM_TABLES];
+        bool used[EP_NUM_TABLES] = {};
+        for (const Candidate &c : cand)
+            for (uint64_t v = 0; v < nvec; ++v) {
+                const int32_t *q = c.fields.data() + 9 * v;
+                for (int j = 0; j < 9; ++j) {
+                    const int t = table_id(q[0], j);
+                    if (!used[t]) { used[t] = true; lo[t] = hi[t] = q[j]; }
+                    else { lo[t] = std::min<int64_t>(lo[t], q[j]); hi[t] = std::max<int64_t>(hi[t], q[j]); }
+                }
+            }
+        std::vector<double> price[EP_NUM_TABLES];      // -log2 of the smoothed probability
+        std::vector<uint64_t> seen[EP_NUM_TABLES];
+        for (int t = 0; t < EP_NUM_TABLES; ++t)
+            if (used[t]) { price[t].resize(size_t(hi[t] - lo[t] + 1)); seen[t].resize(price[t].size()); }
+        auto choose = [&](double lambda, std::vector<int> &pick) {   // kappa_lambda and L(lambda)
+            double L = 0.0;
+            for (uint32_t r = 0; r < R_; ++r) {
+                int best = 0;
+                double bv = D[size_t(r) * K] + lambda * cost[size_t(r) * K];
+                for (int k = 1; k < K; ++k) {
+                    const double v = D[size_t(r) * K + k] + lambda * cost[size_t(r) * K + k];
+                    if (v < bv) { bv = v; best = k; }
+                }
+                pick[r] = best;
+                L += cost[size_t(r) * K + best];
+            }
+            return L;
+        };
+        auto gather = [&](const std::vector<int> &pick, std::vector<int32_t> &dst) {
+            for (uint32_t r = 0; r < R_; ++r)
+                std::copy_n(cand[pick[r]].fields.begin() + long(9 * uint64_t(r) * per_row), 9 * per_row,
+                            dst.begin() + long(9 * uint64_t(r) * per_row));
+        };
+        Model base;
+        base.count(cand[0].fields.data(), nvec, threads_);
+        base.normalise(b);
+        const double B = estimate_bits(base, b, nvec, R_, V, o.retained_bits, nullptr) / 8.0;
+        std::vector<int> sel(R_, 0), hat(R_), trial(R_);
+        std::vector<int32_t> mix(size_t(nvec) * 9);
+        for (int sweep = 0; sweep < o.rdo_sweeps; ++sweep) {
+            gather(sel, mix);
+            uint64_t total[EP_NUM_TABLES] = {};
+            for (int t = 0; t < EP_NUM_TABLES; ++t) std::fill(seen[t].begin(), seen[t].end(), 0);
+            for (uint64_t v = 0; v < nvec; ++v) {
+                const int32_t *q = mix.data() + 9 * v;
+                for (int j = 0; j < 9; ++j) { const int t = table_id(q[0], j); seen[t][size_t(q[j] - lo[t])]++; total[t]++; }
+            }
+            for (int t = 0; t < EP_NUM_TABLES; ++t) {
+                if (!used[t]) continue;
+                const double den = double(total[t]) + 0.5 * double(price[t].size());
+                for (size_t z = 0; z < price[t].size(); ++z) price[t][z] = -std::log2((double(seen[t][z]) + 0.5) / den);
+            }
+            parallel_for(R_, threads_, [&](uint64_t a, uint64_t e, int) {
+                for (uint64_t r = a; r < e; ++r)
+                    for (int k = 0; k < K; ++k) {
+                        double bits = 0.0;
+                        for (uint32_t v = 0; v < per_row; ++v) {
+                            const int32_t *q = cand[k].fields.data() + 9 * (r * per_row + v);
+                            for (int j = 0; j < 9; ++j) { const int t = table_id(q[0], j); bits += price[t][size_t(q[j] - lo[t])]; }
+                        }
+                        cost[r * K + k] = bits;
+                    }
+            });
+            Model mm;
+            mm.count(mix.data(), nvec, threads_);
+            if (mm.worst_observed() > (1u << b)) break;
+            mm.normalise(b);
+            const double Bmix = estimate_bits(mm, b, nvec, R_, V, o.retained_bits, nullptr) / 8.0;
+            double cur = 0.0, dcur = 0.0;
+            for (uint32_t r = 0; r < R_; ++r) { cur += cost[size_t(r) * K + sel[r]]; dcur += D[size_t(r) * K + sel[r]]; }
+            const double budget = cur + 8.0 * (B - Bmix);
+            if (choose(0.0, hat) > budget) {
+                double lam_lo = 0.0, lam_hi = (cur > 0.0 && dcur > 0.0) ? dcur / cur : 1e-12;
+                bool bracketed = false;
+                for (int d = 0; d < 64; ++d) {
+                    if (choose(lam_hi, trial) <= budget) { bracketed = true; break; }
+                    lam_lo = lam_hi;
+                    lam_hi *= 2.0;
+                }
+                if (bracketed) {
+                    hat = trial;
+                    for (int it = 0; it < 20; ++it) {
+                        const double lam = lam_lo == 0.0 ? 0.5 * lam_hi : std::sqrt(lam_lo * lam_hi);
+                        if (choose(lam, trial) > budget) lam_lo = lam;
+                        else { lam_hi = lam; hat = trial; }
+                    }
+                } else {
+                    hat = sel;       // no penalty meets the budget: keep the current selection
+                }
+            }
+            sel = hat;
+        }
+        gather(sel, mix);
+        Model refined;
+        refined.count(mix.data(), nvec, threads_);
+        if (refined.worst_observed() <= (1u << b)) {     // otherwise the baseline stays
+            fields_.swap(mix);
+            refined_sigma_.resize(R_);
+            for (uint32_t r = 0; r < R_; ++r) refined_sigma_[r] = cand[sel[r]].sigma[r];
+            m = refined;
+        }
+        return EP_OK;
     }
 
 private:
@@ -548,6 +715,7 @@ private:
     std::vector<uint32_t> rows_;
     std::vector<float> mu_;
     std::vector<int32_t> sfields_, fields_;
+    std::vector<float> refined_sigma_;
 };
 
 }  // namespace
@@ -568,13 +736,15 @@ extern "C" void ep_encode_opts_default(ep_encode_opts *o) {
     o->polish_steps = 3;
     o->polish_retained_bits = 8.0;
     o->threads = 0;
+    o->rdo_candidates = 1;
+    o->rdo_sweeps = 1;
 }
 
 namespace ep {
 int check_encode_args(uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts &o) {
     if (R == 0 || C == 0 || C % 8 != 0 || !(target_bpp > 0.0)) return EP_ERR_BAD_ARG;
     if (uint64_t(R) * (C / 8) >= (1ull << 32)) return EP_ERR_BAD_ARG;
-    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.polish_steps < 0 || o.b_max > 15 ||
+    if (!(o.bracket_lo > 0.0) || !(o.bracket_hi > o.bracket_lo) || o.search_steps < 0 || o.polish_steps < 0 || o.rdo_candidates < 1 || o.rdo_candidates > 64 || o.rdo_sweeps < 0 || o.b_max > 15 ||
         o.b_max < 9 || (o.b_start != 0 && (o.b_start < 9 || o.b_start > o.b_max)))
         return EP_ERR_BAD_ARG;
     return EP_OK;

@@ -62,7 +62,13 @@ struct EncodeBackend {
     // refit the row scales of the kept quantisation (Eq. 13), encode the tiles under the normalised
     // full-tensor model m and assemble the blob
     virtual int finish(float s, int b, uint32_t V, const Model &m, ep_blob *out) = 0;
+    // per-row rate-distortion refinement of the kept quantisation (Sec. 3.5, Alg. 2); on success `m` holds the
+    // counts of the refined fields and finish() uses the refined row scales.  Optional.
+    virtual int refine(float /*s*/, int /*b*/, uint32_t /*V*/, const ep_encode_opts & /*o*/, Model & /*m*/) { return EP_ERR_UNSUPPORTED; }
 };
+
+// the K nested candidate ratios of Alg. 2: 1 first, then log-midpoints of the widest remaining interval of [0.70, 1.45]
+std::vector<double> rdo_ratios(int K);
 
 // Algorithm 1, the rate-correction stage and the final packing over a back end.
 int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts &o, ep_blob **out);

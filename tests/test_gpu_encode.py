@@ -50,3 +50,10 @@ def test_device_encoder_falls_back_cleanly_on_huge_coordinates():
         ep.encode_device(torch.from_numpy(W).cuda(), 8.0)
     assert ei.value.status == -3
     assert ep.validate(ep.encode(W, 8.0).data) == 0          # the host encoder still serves it
+
+
+def test_device_encoder_leaves_the_per_row_refinement_to_the_host():
+    W = synth.gaussian_rows(32, 512, 11)
+    with pytest.raises(ep.EntroPackError) as ei:
+        ep.encode_device(torch.from_numpy(W).cuda(), 4.0, rdo_candidates=3)
+    assert ei.value.status == -3
