@@ -110,6 +110,24 @@ def test_batch_decode_matches_single():
     assert ep.last_device_status() == 0
 
 
+def test_streams_without_payload_words_and_many_jobs():
+    # an all-zero matrix has one symbol per table: no payload word at all
+    zero = ep.encode(np.zeros((32, 512), np.float32), 4.0, tile_vectors=64)
+    assert zero.info.total_words == 0
+    _check_all_types(zero.data)
+    const = ep.encode(np.tile(np.arange(1, 257, dtype=np.float32), (8, 1)), 5.0, tile_vectors=32)
+    _check_all_types(const.data)
+    # more tensors than one launch takes (16): decode_many splits them
+    blobs = [ep.encode(synth.gaussian_rows(32, 256 + 8 * i, 600 + i), 3.0 + 0.1 * i, tile_vectors=40 + i) for i in range(19)]
+    devs = [ep.upload(b) for b in blobs]
+    outs = [torch.empty((b.info.R, b.info.C), dtype=torch.float16, device="cuda") for b in blobs]
+    ep.decode_many(devs, ep.FP16, outs)
+    torch.cuda.synchronize()
+    for b, o in zip(blobs, outs):
+        assert np.array_equal(_bits(o), oracle.decode(b.data, oracle.FP16)[0])
+    assert ep.last_device_status() == 0
+
+
 def test_damaged_payload_is_flagged_not_fatal():
     W = synth.gaussian_rows(64, 1024, 9)
     blob = ep.encode(W, 4.0, tile_vectors=128)

@@ -108,3 +108,15 @@ def test_validate_rejects_damaged_structure():
     assert broken(swap_offsets) == -2                                                   # offsets not monotone
     with pytest.raises(ep.EntroPackError):
         ep.blob_info(good[:40])
+
+
+def test_suggested_tile_size_fills_whole_rounds_of_slots():
+    slots = 148 * 32
+    for R, C, bpp in ((8192, 8192, 4.0), (8192, 8192, 2.0), (8192, 8192, 6.0), (10240, 3840, 4.0), (5120, 17408, 3.5)):
+        V = ep.suggest_tile_vectors(R, C, bpp, slots)
+        assert V <= ep.default_tile_vectors(bpp) and V % 32 == 0
+        tiles = -(-(R * C // 8) // V)
+        rounds = -(-tiles // slots)
+        assert tiles > 0.93 * rounds * slots                      # the last round is nearly full
+    assert ep.suggest_tile_vectors(512, 512, 4.0, slots) == ep.default_tile_vectors(4.0) // 4    # small tensor: floor
+    assert ep.suggest_tile_vectors(4096, 4096, 3.0, 0) == ep.default_tile_vectors(3.0)
