@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true",
                     help="c4 only: after the main line's measurement also time every target rate 2.0, 2.5 .. 6.0 "
                          "(throughput and stored vs target bpp per rate, in the JSON key 'sweep')")
+    ap.add_argument("--gemm-curve", action="store_true",
+                    help="also time decode-then-GEMM against a GEMM on resident BF16 weights (10240x3840 layer, 4 bpp)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -229,6 +231,56 @@ def run_reference(args):
 
 
 # ---- the GPU arm ---------------------------------------------------------------------------------------
+
+def decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms):
+    """Overhead of reconstructing a layer before each use (the experiment of Sec. "Reconstruction cost and tile
+    overhead", right panel): y = x W^T with W a 10240 x 3840 BF16 layer, x holding 256 .. 16384 tokens, once on
+    resident dense weights and once as decode + the same product.  The product is the library's (torch.matmul);
+    only the decode is this repository's kernel.  Median of 15 flushed repetitions each."""
+    from paper_2609_34185_b200 import synth
+    R, C, bpp = 10240, 3840, 4.0
+    W = synth.gaussian_rows(R, C, 77)
+    V = pick_tile_vectors(-1, W.shape, bpp, 32 * n_sms)
+    blob = ep.encode(W, bpp, tile_vectors=V)
+    d = ep.upload(blob, device=dev)
+    Wd = torch.empty(R, C, dtype=torch.bfloat16, device=dev)
+    ep.decode(d, ep.BF16, out=Wd, stream=stream)
+    g = torch.Generator(device=dev)
+    g.manual_seed(78)
+
+    def median_ms(fn):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(15):
+            flush.fill_(0)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    rows = []
+    for tokens in (256, 1024, 4096, 16384):
+        x = torch.randn(tokens, C, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        y = torch.empty(tokens, R, dtype=torch.bfloat16, device=dev)
+
+        def dense():
+            torch.matmul(x, Wd.t(), out=y)
+
+        def with_decode():
+            ep.decode(d, ep.BF16, out=Wd, stream=stream)
+            torch.matmul(x, Wd.t(), out=y)
+
+        t_dense, t_both = median_ms(dense), median_ms(with_decode)
+        rows.append({"tokens": tokens, "gemm_ms": t_dense, "decode_gemm_ms": t_both,
+                     "overhead_pct": 100.0 * (t_both - t_dense) / t_dense})
+        del x, y
+    return {"layer": [R, C], "target_bpp": bpp, "stored_bpp": blob.stored_bpp, "tile_vectors": blob.info.V,
+            "rows": rows}
+
 
 def main():
     args = parse_args()
@@ -450,6 +502,10 @@ def main():
                           "effective_GBps": nbytes / (med * 1e-3) / 1e9})
             del dd
 
+    gemm_curve = None
+    if args.gemm_curve and rank == 0:
+        gemm_curve = decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -496,7 +552,7 @@ def main():
                        "warm_ms_per_step_no_flush": warm_ms, "rel_l2_first_tensor": rel_l2_first},
             "effective_GBps": eff_gbs, "pct_of_measured_hbm": 100.0 * eff_gbs / peak, "pct_of_8TBps": 100.0 * eff_gbs / 8000.0,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "per_layer_ms": per_layer_ms, "sweep": sweep,
+            "per_layer_ms": per_layer_ms, "sweep": sweep, "decode_then_gemm": gemm_curve,
             "clocks": clocks}
     print(json.dumps(line), flush=True)
     if world > 1:

@@ -457,15 +457,17 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 
 // ---- the hot loop in PTX -------------------------------------------------------------------------------
 // All full groups of one tile.  Written as one asm statement so that every branch can be marked
-// warp-uniform (bra.uni) and the rare work - refilling the payload ring, moving to the next row - sits
-// out of line.  Per group: 9 x rans step, Eq. 5 / Eq. 19 on eight weights, one vector store.
+// warp-uniform (bra.uni) and the rare work - refilling the payload ring, moving to the next row, leaving
+// the loop - sits out of line behind ONE warp vote per group.  Per group: 9 x rans step, Eq. 5 / Eq. 19
+// on eight weights, one vector store.
 //
 // Register roles (asm operands):
 //   x      rANS state                      wa    cursor (shared-memory byte address)
 //   wthr   cursor value that triggers the next ring service (next 512-byte chunk boundary)
 //   wbase  wa - (byte position of the cursor relative to a0)
-//   col,row  this lane's block column inside its row / row index;  sig = row scale bits
-//   doff   byte offset of this lane's block in the output;  left = groups still to do
+//   doff   byte offset of this lane's block in the output
+//   chg    value of doff at which this lane enters its next row;  row = row index;  sig = row scale bits
+//   lim    min(chg, endo): the fast path compares doff with this alone;  endo = doff after the last group
 //   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
 //                     the payload bytes left from there (may be <= 0)
 #define EP_S_FQ(E)                                              \
@@ -576,21 +578,16 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 #define EP_FULL_GROUPS_ASM(STORE, GROUP_BYTES)                                                                        \
     asm volatile(                                                                                                     \
         "{\n\t"                                                                                                       \
-        ".reg .pred p, ps, pw, pa, pl, pq, pv, pm, pm1, plow;\n\t"                                                    \
-        ".reg .b32 u, f, q, bias, bal, t, w, coff, tab, kc, par, pos, cur, lim, n, slot, d;\n\t"                      \
+        ".reg .pred p, ps, pw, pa, pl, pq, pr, pv, pm;\n\t"                                                           \
+        ".reg .b32 u, f, q, bias, bal, t, w, coff, tab, kc, par, pos, cur, clim, n, slot, d, mlim;\n\t"               \
         ".reg .b32 e0, e1, e2, e3, e4, e5, e6, e7, e8, x1, x2, x3, x4, x5, x6, x7, x8, o0, o1, o2, o3;\n\t"           \
         ".reg .b16 h0, h1, h2, h3;\n\t"                                                                               \
         ".reg .f32 w0, w1, w2, w3, w4, w5, w6, w7;\n\t"                                                               \
         ".reg .b64 kk, ss, p0, p1, p2, p3, ad, src;\n\t"                                                              \
-        "setp.lt.u32 plow, %22, 128;\n\t"                                                                             \
-        "setp.eq.u32 pl, %8, 0;\n\t"                                                                                  \
-        "vote.sync.all.pred pl, pl, 0xffffffff;\n\t"                                                                  \
+        "setp.ge.u32 pl, %7, %23;\n\t"                                                                                \
+        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"                                                                  \
         "@pl bra.uni EP_DONE;\n\t"                                                                                    \
         "EP_LOOP:\n\t"                                                                                                \
-        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
-        "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
-        "@ps bra.uni EP_SERVICE;\n\t"                                                                                 \
-        "EP_RESUME:\n\t"                                                                                              \
         EP_S_STEP("e0", "%15", "131072")                                                                              \
         "and.b32 coff, e0, 0xFF800;\n\t"                                                                              \
         "add.u32 tab, %15, coff;\n\t"                                                                                 \
@@ -627,46 +624,47 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "add.s64 ad, ad, %19;\n\t"                                                                                    \
         STORE                                                                                                         \
         "add.u32 %7, %7, " #GROUP_BYTES ";\n\t"                                                                       \
-        "add.u32 %4, %4, 32;\n\t"                                                                                     \
-        "setp.ge.u32 pw, %4, %17;\n\t"                                                                                \
-        "vote.sync.any.pred pa, pw, 0xffffffff;\n\t"                                                                  \
-        "@pa bra.uni EP_ROWCHG;\n\t"                                                                                  \
-        "EP_ROWDONE:\n\t"                                                                                             \
-        "sub.u32 %8, %8, 1;\n\t"                                                                                      \
-        "setp.ne.u32 pl, %8, 0;\n\t"                                                                                  \
-        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */        \
-        "@pl bra.uni EP_LOOP;\n\t"                                                                                    \
-        "bra.uni EP_DONE;\n\t"                                                                                        \
-        /* ---- some lane moved to the next row: reload its scale ---- */                                             \
-        "EP_ROWCHG:\n\t"                                                                                              \
-        "@pw sub.u32 %4, %4, %17;\n\t"                                                                                \
+        /* one vote for everything rare: the cursor crossed a chunk boundary, or this lane reached lim */             \
+        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
+        "setp.ge.or.u32 pq, %7, %8, ps;\n\t"                                                                          \
+        "vote.sync.any.pred pq, pq, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */        \
+        "@!pq bra.uni EP_LOOP;\n\t"                                                                                   \
+        "setp.ge.u32 pr, %7, %8;\n\t"                                                                                 \
+        "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                                  \
+        "@!pr bra.uni EP_SVCCHK;\n\t"                                                                                 \
+        /* ---- some lane moved to the next row (reload its scale), or the tile's full groups are done ---- */        \
+        "setp.ge.u32 pw, %7, %4;\n\t"                                                                                 \
+        "@pw add.u32 %4, %4, %17;\n\t"                                                                                \
         "@pw add.u32 %5, %5, 1;\n\t"                                                                                  \
-        "min.u32 t, %5, %23;\n\t"                                                                                     \
+        "min.u32 t, %5, %22;\n\t"                                                                                     \
         "mul.wide.u32 ad, t, 4;\n\t"                                                                                  \
         "add.s64 ad, ad, %20;\n\t"                                                                                    \
         "@pw ld.global.nc.b32 %6, [ad];\n\t"                                                                          \
-        "bra.uni EP_ROWDONE;\n\t"                                                                                     \
+        "min.u32 %8, %4, %23;\n\t"                                                                                    \
+        "setp.ge.u32 pl, %7, %23;\n\t"                                                                                \
+        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"                                                                  \
+        "@pl bra.uni EP_DONE;\n\t"                                                                                    \
+        "EP_SVCCHK:\n\t"                                                                                              \
+        "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
+        "@!ps bra.uni EP_LOOP;\n\t"                                                                                   \
         /* ---- the cursor entered a new 512-byte chunk: request chunks up to cur+3, wait for all but the newest */   \
-        "EP_SERVICE:\n\t"                                                                                             \
         "sub.u32 pos, %1, %3;\n\t"                                                                                    \
         "shr.u32 cur, pos, 9;\n\t"                                                                                    \
-        "add.u32 lim, cur, 4;\n\t"                                                                                    \
+        "add.u32 clim, cur, 4;\n\t"                                                                                   \
+        "sub.u32 t, %24, %16;\n\t"                     /* 16 * lane */                                                \
+        "setp.lt.u32 pm, t, 128;\n\t"                                                                                 \
+        "selp.u32 mlim, 2, 1, pm;\n\t"                 /* slot 0 is mirrored whole, slot 1 by lanes 0..7 */           \
         "EP_SVC_LOOP:\n\t"                                                                                            \
-        "setp.ge.u32 pq, %11, lim;\n\t"                                                                               \
+        "setp.ge.u32 pq, %11, clim;\n\t"                                                                              \
         "@pq bra.uni EP_SVC_DONE;\n\t"                                                                                \
         "min.s32 n, %10, 16;\n\t"                                                                                     \
         "max.s32 n, n, 0;\n\t"                                                                                        \
         "setp.gt.s32 pv, %10, 0;\n\t"                                                                                 \
         "selp.b64 src, %9, %21, pv;\n\t"                                                                              \
         "and.b32 slot, %11, 3;\n\t"                                                                                   \
-        "shl.b32 d, slot, 9;\n\t"                                                                                     \
-        "add.u32 d, d, %16;\n\t"                                                                                      \
-        "add.u32 d, d, %22;\n\t"                                                                                      \
+        "mad.lo.u32 d, slot, 512, %24;\n\t"                                                                           \
         "cp.async.cg.shared.global [d], [src], 16, n;\n\t"                                                            \
-        "setp.eq.u32 pm, slot, 0;\n\t"                                                                                \
-        "setp.eq.u32 pm1, slot, 1;\n\t"                                                                               \
-        "and.pred pm1, pm1, plow;\n\t"                                                                                \
-        "or.pred pm, pm, pm1;\n\t"                                                                                    \
+        "setp.lt.u32 pm, slot, mlim;\n\t"                                                                             \
         "@pm cp.async.cg.shared.global [d+2048], [src], 16, n;\n\t"                                                   \
         "cp.async.commit_group;\n\t"                                                                                  \
         "add.s64 %9, %9, 512;\n\t"                                                                                    \
@@ -682,14 +680,14 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "shl.b32 t, cur, 9;\n\t"                                                                                      \
         "add.u32 t, t, 512;\n\t"                                                                                      \
         "add.u32 %2, %3, t;\n\t"                                                                                      \
-        "bra.uni EP_RESUME;\n\t"                                                                                      \
+        "bra.uni EP_LOOP;\n\t"                                                                                        \
         "EP_DONE:\n\t"                                                                                                \
         "}"                                                                                                           \
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
-        : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(col), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
-          "+&r"(left), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                          \
-        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(per_row), "r"(k0_bits), "l"(out_base),        \
-          "l"(scales), "l"(a0), "r"(lane16), "r"(row_max)                                                             \
+        : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(chg), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
+          "+&r"(lim), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                           \
+        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(row_bytes), "r"(k0_bits), "l"(out_base),         \
+          "l"(scales), "l"(a0), "r"(row_max), "r"(endo), "r"(ring_lane)                                               \
         : "memory")
 
 // One tile of a tensor whose rows hold at least 32 blocks: the full groups in PTX, a last partial group
@@ -722,16 +720,22 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     uint64_t srcp = a0 + 2048u + lane16;          // this lane's part of chunk 4
     uint32_t rem = room - (2048u + lane16);       // signed in the asm: may be negative
     uint32_t nextc = 4;
+    const uint32_t ring_lane = ring + lane16;
     const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
     const uint32_t v = v0 + lane;
-    uint32_t row = v / per_row, col = v - row * per_row;
+    uint32_t row = v / per_row;
     const float *scales = J.scales;
     uint32_t sig = __float_as_uint(__ldg(scales + row));
     uint32_t doff = v * Out<DT>::kBlockBytes;
     const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
-    // The group count is the same in all lanes but comes from loaded data, which the compiler treats as possibly
-    // different per lane; the loop therefore branches on warp votes of it (see the asm), never on the value itself.
-    uint32_t left = nv >> 5;                           // may be 0: the asm then falls straight through
+    // The loop runs on byte offsets into the output: this lane leaves its row when doff reaches chg and the tile's
+    // full groups are done when it reaches endo.  The group count is the same in all lanes but comes from loaded
+    // data, which the compiler treats as possibly different per lane; the loop therefore branches on warp votes of
+    // these comparisons (see the asm), never on the values themselves.  nv >> 5 may be 0: the asm falls through.
+    const uint32_t row_bytes = per_row * Out<DT>::kBlockBytes;
+    uint32_t chg = (row + 1u) * row_bytes;
+    const uint32_t endo = doff + (nv >> 5) * (32u * Out<DT>::kBlockBytes);
+    uint32_t lim = min(chg, endo);
     const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
     if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
     else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
@@ -1095,8 +1099,9 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
             (reinterpret_cast<uintptr_t>(jb.d_out) & 15))
             return EP_ERR_BAD_ARG;
         if (I.table_K[0] == 0 || I.table_min[0] < 0 || int64_t(I.table_min[0]) + I.table_K[0] > 2) return EP_ERR_BAD_STREAM;
-        // 32-bit byte offsets into the output and a signed 32-bit payload remainder in the kernels
-        if (uint64_t(I.R) * I.C * 4u >= (1ull << 32) || I.total_words >= (1ull << 30)) return EP_ERR_UNSUPPORTED;
+        // 32-bit byte offsets into the output (one row and one group beyond the end still representable) and a
+        // signed 32-bit payload remainder in the kernels
+        if ((uint64_t(I.R) + 1u) * I.C * 4u + 1024u >= (1ull << 32) || I.total_words >= (1ull << 30)) return EP_ERR_UNSUPPORTED;
         if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; tiles_total += I.n_tiles; }
         else large[n_large++] = &jb;
     }
