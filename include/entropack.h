@@ -182,7 +182,7 @@ int ep_validate(const void *blob, size_t n);
 /* ---- device decoder ----------------------------------------------------------------------- */
 
 /* Scratch bytes the decoder needs for this tensor: 0 when the symbol lookup tables fit shared
- * memory (b <= 11 and coordinate range <= 512), else room for 17 tables of 2^b 8-byte entries. */
+ * memory (b <= 11 and coordinate range <= 1024, no single-symbol table at b = 11), else room for 17 tables of 2^b 8-byte entries. */
 size_t ep_decode_scratch_bytes(const ep_info *info);
 
 /* Fused decode of one tensor (Sec. 3.7): rANS symbol decode (Eq. 18) -> inverse field transform

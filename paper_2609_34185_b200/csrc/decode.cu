@@ -6,10 +6,11 @@
 // Mapping: one warp per tile, one rANS state per lane (the paper's layout); a CTA of 32 warps
 // builds the seventeen slot->(frequency, offset, value) lookup tables once in shared memory from the
 // stream's frequency tables and then streams tiles through them.  A lookup entry is one 32-bit word
-//     [31:20] f      [19:11] code     [10:0] u - F
+//     [31:21] f      [20:11] code     [10:0] u - F
 // where `code` is the symbol's coordinate relative to an even base zlo (z - zlo; 2m - zlo for the m
-// field; 32c for the coset, which makes (entry & 0xFF800) the byte offset of coset c's tables).
-// (entry & 0xFF800) | 0x45800000 is the fp32 number 4096 + code, so one subtraction of
+// field; 32c for the coset, which makes (entry & 0x1FF800) the byte offset of coset c's tables).
+// f < 2^11 always: a table with a single symbol at b = 11 (f = 2^11) goes to the large-table path.
+// (entry & 0x1FF800) | 0x45800000 is the fp32 number 4096 + code, so one subtraction of
 // 4096 - zlo - c/2 yields the lattice coordinate p exactly, and one fp32 multiply by the row scale
 // gives the product of Eq. 19 with the same operands and rounding as the definition.
 //
@@ -39,7 +40,7 @@ constexpr uint32_t kRingBytes = 2048;                  // four 512-byte chunks p
 constexpr uint32_t kRingMirror = 640;                  // >= 9 steps * 32 words * 2 bytes + one lane span
 constexpr uint32_t kRingStride = kRingBytes + kRingMirror;
 constexpr uint32_t kSmemBytes = kLutBytes + kWarps * kRingStride;   // 225280
-constexpr uint32_t kCodeMask = 0x000FF800u;
+constexpr uint32_t kCodeMask = 0x001FF800u;            // 10-bit code field
 constexpr uint32_t kExp4096 = 0x45800000u;             // fp32 bit pattern of 4096.0
 
 __device__ unsigned int g_ep_status = 0;
@@ -161,7 +162,8 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
         const uint32_t first = run + incl - f;
         const int32_t v = tmin + int32_t(j);
         const uint32_t code = t == 0 ? uint32_t(v) * 32u : uint32_t((is_m ? 2 * v : v) - J.zlo);
-        const uint32_t entry = (f << 20) | ((code & 0x1FFu) << 11);
+        const uint32_t entry = (f << 21) | ((code & 0x3FFu) << 11);
+        if (f >= kLutEntries) atomicOr(&g_ep_status, 1u);   // not a stream the launcher sends here: f does not fit its field
 #pragma unroll
         for (uint32_t u = 0; u < 4; ++u)
             if (u < f && first + u < kLutEntries) sts32(base + 4u * (first + u), entry | u);
@@ -196,7 +198,7 @@ __device__ __forceinline__ uint32_t rans_step(uint32_t &x, uint32_t table_addr, 
         "shl.b32 u, u, 2;\n\t"
         "add.u32 u, u, %5;\n\t"
         "ld.shared.u32 %0, [u + %7];\n\t"
-        "shr.u32 f, %0, 20;\n\t"
+        "shr.u32 f, %0, 21;\n\t"
         "and.b32 bias, %0, 0x7FF;\n\t"
         "shr.u32 q, %1, %4;\n\t"
         "mad.lo.u32 %1, f, q, bias;\n\t"
@@ -225,7 +227,7 @@ __device__ __forceinline__ uint32_t rans_step_tail(uint32_t &x, uint32_t table_a
     bool need = false;
     if (act) {
         e = lds32(table_addr + ((x & mask) << 2));
-        x = (e >> 20) * (x >> b) + (e & 0x7FFu);
+        x = (e >> 21) * (x >> b) + (e & 0x7FFu);
         need = x < ep::kStateLow;
     }
     const uint32_t bal = __ballot_sync(0xFFFFFFFFu, need);
@@ -471,7 +473,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
 //   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
 //                     the payload bytes left from there (may be <= 0)
 #define EP_S_FQ(E)                                              \
-    "shr.u32 f, " E ", 20;\n\t"                                 \
+    "shr.u32 f, " E ", 21;\n\t"                                 \
     "shr.u32 q, %0, %14;\n\t"
 #define EP_S_FETCH                                              \
     "and.b32 t, bal, %12;\n\t"                                  \
@@ -589,7 +591,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "@pl bra.uni EP_DONE;\n\t"                                                                                    \
         "EP_LOOP:\n\t"                                                                                                \
         EP_S_STEP("e0", "%15", "131072")                                                                              \
-        "and.b32 coff, e0, 0xFF800;\n\t"                                                                              \
+        "and.b32 coff, e0, 0x1FF800;\n\t"                                                                              \
         "add.u32 tab, %15, coff;\n\t"                                                                                 \
         EP_S_STEP("e1", "tab", "0")                                                                                   \
         EP_S_STEP("e2", "tab", "8192")                                                                                \
@@ -602,18 +604,18 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         /* Eq. 5: 4096 + code as fp32, minus kc = 4096 - zlo - c/2 (one ulp = 2^-11, c/2 = 1024 ulps) */              \
         "shr.u32 t, coff, 6;\n\t"                                                                                     \
         "sub.u32 kc, %18, t;\n\t"                                                                                     \
-        "lop3.b32 x1, e1, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x2, e2, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x3, e3, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x4, e4, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x5, e5, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x6, e6, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x7, e7, 0xFF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x1, e1, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x2, e2, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x3, e3, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x4, e4, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x5, e5, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x6, e6, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
+        "lop3.b32 x7, e7, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
         "lop3.b32 par, e1, e2, e3, 0x96;\n\t"                                                                         \
         "lop3.b32 par, par, e4, e5, 0x96;\n\t"                                                                        \
         "lop3.b32 par, par, e6, e7, 0x96;\n\t"                                                                        \
         "lop3.b32 par, par, 0x800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x8, e8, 0xFF800, par, 0xEA;\n\t"                                                                    \
+        "lop3.b32 x8, e8, 0x1FF800, par, 0xEA;\n\t"                                                                    \
         "mov.b64 kk, {kc, kc};\n\t"                                                                                   \
         "mov.b64 ss, {%6, %6};\n\t"                                                                                   \
         EP_S_PAIR("p0", "x1", "x2", "w0", "w1")                                                                       \
@@ -624,11 +626,11 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "add.s64 ad, ad, %19;\n\t"                                                                                    \
         STORE                                                                                                         \
         "add.u32 %7, %7, " #GROUP_BYTES ";\n\t"                                                                       \
-        /* one vote for everything rare: the cursor crossed a chunk boundary, or this lane reached lim */             \
-        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
-        "setp.ge.or.u32 pq, %7, %8, ps;\n\t"                                                                          \
-        "vote.sync.any.pred pq, pq, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */        \
-        "@!pq bra.uni EP_LOOP;\n\t"                                                                                   \
+        /* one vote for everything rare: go on only if no lane crossed a chunk boundary or reached its lim */        \
+        "setp.lt.u32 ps, %1, %2;\n\t"                                                                                 \
+        "setp.lt.and.u32 pq, %7, %8, ps;\n\t"                                                                         \
+        "vote.sync.all.pred pq, pq, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */         \
+        "@pq bra.uni EP_LOOP;\n\t"                                                                                    \
         "setp.ge.u32 pr, %7, %8;\n\t"                                                                                 \
         "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                                  \
         "@!pr bra.uni EP_SVCCHK;\n\t"                                                                                 \
@@ -645,6 +647,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"                                                                  \
         "@pl bra.uni EP_DONE;\n\t"                                                                                    \
         "EP_SVCCHK:\n\t"                                                                                              \
+        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
         "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
         "@!ps bra.uni EP_LOOP;\n\t"                                                                                   \
         /* ---- the cursor entered a new 512-byte chunk: request chunks up to cur+3, wait for all but the newest */   \
@@ -656,6 +659,7 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
         "selp.u32 mlim, 2, 1, pm;\n\t"                 /* slot 0 is mirrored whole, slot 1 by lanes 0..7 */           \
         "EP_SVC_LOOP:\n\t"                                                                                            \
         "setp.ge.u32 pq, %11, clim;\n\t"                                                                              \
+        "vote.sync.any.pred pq, pq, 0xffffffff;\n\t"                                                                  \
         "@pq bra.uni EP_SVC_DONE;\n\t"                                                                                \
         "min.s32 n, %10, 16;\n\t"                                                                                     \
         "max.s32 n, n, 0;\n\t"                                                                                        \
@@ -978,9 +982,12 @@ bool fits_smem_tables(const ep_info &I) {
     if (I.b > 11) return false;
     const Range r = coord_range(I);
     const int64_t zlo = even_base(r);
-    if (r.any && r.hi - zlo > 511) return false;
-    if (zlo < -512) return false;
-    for (int t = 0; t < EP_NUM_TABLES; ++t) if (I.table_K[t] > kLutEntries) return false;
+    if (r.any && r.hi - zlo > 1023) return false;     // 10-bit code field
+    if (zlo < -1024) return false;                    // 4096 - zlo - c/2 stays below 8192: same fp32 exponent as 4096 + code
+    for (int t = 0; t < EP_NUM_TABLES; ++t) {
+        if (I.table_K[t] > kLutEntries) return false;
+        if (I.b == 11 && I.table_K[t] == 1) return false;   // a lone symbol has f = 2^11: one bit more than the f field
+    }
     return true;
 }
 

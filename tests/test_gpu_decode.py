@@ -157,7 +157,7 @@ def test_decode_argument_checks():
         ep.decode_tensor(d.info, 0, d.d_tile_index, d.d_row_scales, ep.BF16, out.data_ptr())
 
 
-# ---- streams whose lookup tables do not fit shared memory (b >= 12 or coordinate range > 512) -----
+# ---- streams whose lookup tables do not fit shared memory (b >= 12 or coordinate range > 1024) -----
 
 def test_large_table_path_high_precision_and_high_rate():
     W = synth.laplace_rows(96, 1024, 77)
@@ -187,6 +187,46 @@ def test_large_table_path_wide_coordinate_range():
     blob = ep.pack_fields(fields, 6, 512, 11, 50, np.linspace(0.01, 0.02, 6).astype(np.float32))
     assert ep.decode_scratch_bytes(blob.info) > 0
     _check_all_types(blob.data)
+
+
+def test_coordinate_range_up_to_1024_stays_on_the_shared_memory_path():
+    # the table entry's code field holds ten bits: coordinates spread over 513 .. 1024 values need no scratch
+    rng = np.random.default_rng(4)
+    n = 8 * 64
+    fields = np.zeros((n, 9), np.int32)
+    fields[:, 0] = rng.integers(0, 2, n)
+    fields[:, 1:] = np.rint(rng.standard_normal((n, 8)) * 6).astype(np.int32)
+    fields[3, 2] = 500
+    fields[90, 7] = -520          # z range -520 .. 500: 1021 values, even base -520
+    fields[200, 8] = 250          # m = 250 stands for z8 = 500 or 501
+    fields[201, 8] = -260         # and z8 = -520 or -519
+    blob = ep.pack_fields(fields, 8, 512, 11, 64, np.linspace(0.01, 0.03, 8).astype(np.float32))
+    assert ep.decode_scratch_bytes(blob.info) == 0
+    _check_all_types(blob.data)
+    # one value more on either side no longer fits
+    fields[4, 1] = 504
+    blob = ep.pack_fields(fields, 8, 512, 11, 64, np.linspace(0.01, 0.03, 8).astype(np.float32))
+    assert ep.decode_scratch_bytes(blob.info) > 0
+    _check_all_types(blob.data)
+    # Laplace rows at 7 bpp: b = 11 with coordinates beyond +-256
+    blob = ep.encode(synth.laplace_rows(512, 4096, 4), 7.0)
+    assert blob.info.b == 11 and blob.info.coord_max - blob.info.coord_min > 512
+    assert ep.decode_scratch_bytes(blob.info) == 0
+    _check_all_types(blob.data)
+
+
+def test_single_symbol_table_at_b11_takes_the_large_table_path():
+    # a lone symbol has frequency 2^11, one bit more than the shared-memory entry's frequency field
+    rng = np.random.default_rng(5)
+    n = 4 * 64
+    fields = np.zeros((n, 9), np.int32)                      # coset always 0: the coset table has one symbol
+    fields[:, 1:] = np.rint(rng.standard_normal((n, 8)) * 3).astype(np.int32)
+    blob = ep.pack_fields(fields, 4, 512, 11, 40, np.full(4, 0.02, np.float32))
+    assert blob.info.table_K[0] == 1 and ep.decode_scratch_bytes(blob.info) > 0
+    _check_all_types(blob.data)
+    blob10 = ep.pack_fields(fields, 4, 512, 10, 40, np.full(4, 0.02, np.float32))
+    assert ep.decode_scratch_bytes(blob10.info) == 0        # f = 2^10 fits
+    _check_all_types(blob10.data)
 
 
 def test_large_table_path_needs_scratch_and_mixes_in_a_batch():
