@@ -182,7 +182,8 @@ int ep_validate(const void *blob, size_t n);
 /* ---- device decoder ----------------------------------------------------------------------- */
 
 /* Scratch bytes the decoder needs for this tensor: 0 when the symbol lookup tables fit shared
- * memory (b <= 11 and coordinate range <= 1024, no single-symbol table at b = 11), else room for 17 tables of 2^b 8-byte entries. */
+ * memory (b <= 11 and coordinate range <= 1024, no single-symbol table at b = 11), else room
+ * for 17 tables of 2^b four-byte entries. */
 size_t ep_decode_scratch_bytes(const ep_info *info);
 
 /* Fused decode of one tensor (Sec. 3.7): rANS symbol decode (Eq. 18) -> inverse field transform
@@ -197,7 +198,7 @@ int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_ti
 int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
 
 /* Largest probability precision b served by ep_decode_tensor_static: its built-in table area holds
- * 17 tables of 2^13 eight-byte entries = 1 114 112 bytes of device memory per GPU that loads the library. */
+ * 17 tables of 2^13 four-byte entries = 557 056 bytes of device memory per GPU that loads the library. */
 #define EP_STATIC_MAX_B 13
 
 /* (No counterpart in the paper: an integration aid of this library.)

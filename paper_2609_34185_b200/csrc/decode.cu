@@ -801,10 +801,14 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
 }
 
 // ======================================================================================================
-// Large-table path: b >= 12 or a coordinate range above 512.  The seventeen tables (2^b slots of 8 bytes:
-// {f | (u - F) << 16, value}) are built into caller-provided scratch by one launch and read through L1/L2
-// by the decode launch that follows on the same stream.  Same tile / lane / word order as above; payload
-// words are read straight from global memory with the index clamped to the payload.
+// Large-table path: b >= 12, a coordinate range above 1024, or a single-symbol table at b = 11.  The
+// seventeen tables (2^b slots of 4 bytes: symbol index << 16 | u - F) are built into caller-provided
+// scratch by one launch and read through L1/L2 by the decode launch that follows on the same stream; a
+// symbol's frequency comes from the stream's own frequency arrays (a few KB, resident in L1) and its value
+// is the table's minimum plus the index.  Slots are hit uniformly at random, so the traffic between L2 and
+// L1 is what bounds this path: four-byte entries halve the table set (278 KB at b = 12, most of it
+// L1-resident).  Same tile / lane / word order as above; payload words are read straight from global
+// memory with the index clamped to the payload.
 // ======================================================================================================
 
 struct GJobParams {
@@ -812,7 +816,7 @@ struct GJobParams {
     const uint32_t *tile_index;
     const float *scales;
     void *out;
-    uint2 *lut;                   // scratch: 17 << b entries
+    uint32_t *lut;                // scratch: 17 << b entries
     uint32_t off_tables;          // byte offset of the table section (directory, then frequencies)
     uint32_t off_payload;
     uint32_t total_words;
@@ -838,7 +842,6 @@ __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_cons
     const GJobParams &J = P.job[blockIdx.y];
     const uint32_t t = blockIdx.x, tid = threadIdx.x;
     const uint8_t *dir = J.stream + J.off_tables;
-    const int32_t tmin = reinterpret_cast<const int32_t *>(dir)[t];
     const uint32_t *Ks = reinterpret_cast<const uint32_t *>(dir) + EP_NUM_TABLES;
     const uint32_t K = Ks[t];
     if (K == 0) return;
@@ -862,44 +865,60 @@ __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_cons
     for (uint32_t j = j0; j < j1; ++j) { F[j] = uint16_t(run); run += fq[j]; }
     __syncthreads();
     const uint32_t M = 1u << J.b;
-    uint2 *lut = J.lut + (size_t(t) << J.b);
+    uint32_t *lut = J.lut + (size_t(t) << J.b);
     for (uint32_t u = tid; u < M; u += blockDim.x) {
         uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u; F[K] = 2^b > u
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
             if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
         }
-        const uint32_t f = uint32_t(F[lo + 1]) - uint32_t(F[lo]);
-        lut[u] = make_uint2(f | ((u - uint32_t(F[lo])) << 16), uint32_t(tmin + int32_t(lo)));
+        lut[u] = (lo << 16) | (u - uint32_t(F[lo]));                 // K <= 65535 and u - F < 2^15
     }
 }
 
-__device__ __forceinline__ int32_t grans_step(uint32_t &x, const uint2 *table, uint32_t mask, uint32_t b, uint32_t &ptr,
-                                              const uint16_t *pay, uint32_t lt, bool act, uint32_t last_word) {
-    int32_t value = 0;
+// one symbol: returns its index inside table t's symbol range (0 for an idle lane)
+__device__ __forceinline__ uint32_t grans_step(uint32_t &x, const uint32_t *table, const uint16_t *freq, uint32_t mask,
+                                               uint32_t b, uint32_t &ptr, const uint16_t *pay, uint32_t lt, bool act,
+                                               uint32_t last_word) {
+    uint32_t sym = 0;
     bool need = false;
     if (act) {
-        const uint2 e = __ldg(table + (x & mask));
-        x = (e.x & 0xFFFFu) * (x >> b) + (e.x >> 16);
-        value = int32_t(e.y);
+        const uint32_t e = __ldg(table + (x & mask));
+        sym = e >> 16;
+        x = uint32_t(__ldg(freq + sym)) * (x >> b) + (e & 0xFFFFu);
         need = x < ep::kStateLow;
     }
     const uint32_t bal = __ballot_sync(0xFFFFFFFFu, need);
     if (need) x = (x << 16) | __ldg(pay + min(ptr + __popc(bal & lt), last_word));
     ptr += __popc(bal);
-    return value;
+    return sym;
 }
 
 template <int DT>
 __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_constant__ GBatchParams P) {
+    __shared__ uint32_t s_foff[EP_NUM_TABLES];     // start of table t's frequencies, in u16 units
+    __shared__ int32_t s_tmin[EP_NUM_TABLES];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     int j = 0;
     while (j + 1 < P.n_jobs && blockIdx.x >= P.job[j + 1].cta_begin) ++j;
     const GJobParams &J = P.job[j];
+    const uint8_t *dir = J.stream + J.off_tables;
+    if (threadIdx.x == 0) {
+        const uint32_t *Ks = reinterpret_cast<const uint32_t *>(dir) + EP_NUM_TABLES;
+        uint32_t acc = 0;
+        for (int t = 0; t < EP_NUM_TABLES; ++t) {
+            s_foff[t] = acc;
+            s_tmin[t] = reinterpret_cast<const int32_t *>(dir)[t];
+            acc += Ks[t];
+        }
+    }
+    __syncthreads();
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(dir + 8 * EP_NUM_TABLES);
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
     const uint16_t *pay = reinterpret_cast<const uint16_t *>(J.stream + J.off_payload);
     const uint32_t last_word = J.total_words ? J.total_words - 1u : 0u;
     const uint32_t cta = blockIdx.x - J.cta_begin;
+    const uint32_t foff0 = s_foff[0];
     for (uint32_t tile = cta * kGWarps + warp; tile < J.n_tiles; tile += J.cta_count * kGWarps) {
         const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
         uint32_t x = rec[lane];
@@ -911,11 +930,12 @@ __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_
             const uint32_t i = g * 32u + lane;
             const bool act = i < nv;
             int32_t fld[9];
-            fld[0] = grans_step(x, J.lut, mask, b, ptr, pay, lt, act, last_word);
-            const uint2 *tabs = J.lut + (size_t(1 + 8 * (fld[0] & 1)) << b);
+            fld[0] = int32_t(grans_step(x, J.lut, fq + foff0, mask, b, ptr, pay, lt, act, last_word)) + s_tmin[0];
+            const uint32_t t0 = 1u + 8u * uint32_t(fld[0] & 1);          // first coordinate table of this coset
 #pragma unroll
-            for (int k = 1; k <= 8; ++k)
-                fld[k] = grans_step(x, tabs + (size_t(k - 1) << b), mask, b, ptr, pay, lt, act, last_word);
+            for (uint32_t k = 0; k < 8; ++k)
+                fld[k + 1] = int32_t(grans_step(x, J.lut + (size_t(t0 + k) << b), fq + s_foff[t0 + k], mask, b, ptr, pay, lt,
+                                                act, last_word)) + s_tmin[t0 + k];
             if (!act) continue;
             const uint32_t v = v0 + i;
             if constexpr (DT == EP_FIELDS_I32) {
@@ -1011,7 +1031,7 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
 extern "C" size_t ep_decode_scratch_bytes(const ep_info *info) {
     if (!info) return 0;
     if (fits_smem_tables(*info)) return 0;
-    return size_t(EP_NUM_TABLES) * (size_t(1) << info->b) * 8u;
+    return size_t(EP_NUM_TABLES) * (size_t(1) << info->b) * 4u;
 }
 
 namespace {
@@ -1031,7 +1051,7 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
     for (int i = 0; i < n_jobs; ++i) {
         const ep_decode_job &jb = *jobs[i];
         const ep_info &I = *jb.info;
-        const size_t need = size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 8u;
+        const size_t need = size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 4u;
         if (!jb.d_scratch || jb.scratch_bytes < need || (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255)) return EP_ERR_SCRATCH;
         for (int t = 0; t < EP_NUM_TABLES; ++t) {
             if (I.table_K[t] > 65535u) return EP_ERR_UNSUPPORTED;
@@ -1042,7 +1062,7 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
         J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
         J.scales = jb.d_row_scales;
         J.out = jb.d_out;
-        J.lut = static_cast<uint2 *>(jb.d_scratch);
+        J.lut = static_cast<uint32_t *>(jb.d_scratch);
         J.off_tables = I.off_tables;
         J.off_payload = I.off_payload;
         J.total_words = uint32_t(I.total_words);
@@ -1204,7 +1224,7 @@ extern "C" int ep_last_device_status(void *stream) {
 // caller scratch.  One area per device, shared by every call: calls that overlap on the GPU race on it.
 namespace {
 
-constexpr size_t kStaticTableBytes = size_t(EP_NUM_TABLES) * (size_t(1) << EP_STATIC_MAX_B) * 8u;   // 1 114 112
+constexpr size_t kStaticTableBytes = size_t(EP_NUM_TABLES) * (size_t(1) << EP_STATIC_MAX_B) * 4u;   // 557 056
 static __device__ __align__(256) unsigned char g_ep_static_tables[kStaticTableBytes];
 
 // In host code `g_ep_static_tables` is only a handle for the runtime, not an address a kernel could use:
