@@ -304,6 +304,7 @@ void epo_normalise_freqs(const uint64_t *n, uint32_t K, int b, uint32_t *f) {
         for (uint32_t j = 1; j < K; ++j) if (f[j] > f[jm]) jm = j;
         uint64_t take = sum - M;
         if (take > (uint64_t)f[jm] - 1) take = f[jm] - 1;
+        if (take == 0) break;   /* more than 2^b observed symbols: no valid table exists (callers test the fit first) */
         f[jm] -= (uint32_t)take;
         sum -= take;
     }
@@ -1035,6 +1036,12 @@ int epo_encode(const float *W, uint32_t R, uint32_t C, double target_bpp, const 
                 quantise_row(W + (size_t)srows[i] * C, C, mu[srows[i]], sq, sf + 9 * (size_t)i * (C / 8));
             epo_tab t[EPO_NT];
             tabs_count(sf, svec, t);
+            /* Reading (the paper does not say): a sampled table with more than 2^b observed symbols cannot be given
+             * b-bit frequencies at all, so this scale is too fine at this precision; the search moves on as if its
+             * rate were above the target.  The precision loop below raises b if the coarser scale still does not fit. */
+            int sample_fits = 1;
+            for (int i = 0; i < EPO_NT; ++i) if (tabs_observed(t, i) > (1u << b)) sample_fits = 0;
+            if (!sample_fits) { tabs_free(t); lo = s; continue; }
             tabs_normalise(t, b);
             double bits = estimate_bits(t, b, svec, ns, V, o.retained_bits, NULL);
             tabs_free(t);

@@ -132,6 +132,7 @@ void Model::normalise(int b) {
         while (sum > M) {
             const uint32_t j = largest();
             const uint64_t take = std::min<uint64_t>(sum - M, uint64_t(tb.f[j]) - 1);
+            if (take == 0) break;   // over 2^b observed symbols: callers check worst_observed() before relying on the sum
             tb.f[j] -= uint32_t(take);
             sum -= take;
         }
@@ -304,6 +305,9 @@ int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, con
             const double mid = std::sqrt(lo * hi);
             Model m;
             if ((rc = be.count_sample(float(mid), m))) return rc;
+            // more observed symbols than 2^b slots: no b-bit table exists for this scale; treat it as too fine
+            // (rate above the target).  If the scale found this way still overflows on the full tensor, b goes up.
+            if (m.worst_observed() > (1u << b)) { lo = mid; continue; }
             m.normalise(b);
             const double bits = estimate_bits(m, b, svec, rows.size(), V, o.retained_bits, nullptr);
             last_rate = bits / (8.0 * double(svec));

@@ -46,6 +46,24 @@ def test_other_distributions_and_threads():
         assert abs(a.stored_bpp - bpp) < 0.02 * bpp
 
 
+@pytest.mark.timeout(120)
+def test_search_survives_sample_alphabets_beyond_the_precision():
+    # low starting precision at a high rate: the fine end of the scale search sees more than 2^b symbols per
+    # table in the sample; such a scale counts as too fine (no b-bit table exists for it) and the search goes on
+    W = synth.laplace_rows(256, 2048, 11)
+    for b0, bpp in ((9, 8.0), (9, 7.0), (10, 8.0)):
+        a = ep.encode(W, bpp, b_start=b0)
+        o, rep = oracle.encode(W, bpp, oracle.default_opts(b_start=b0))
+        assert np.array_equal(a.data, o)
+        assert max(a.info.table_K) <= 1 << a.info.b
+        assert abs(a.stored_bpp - bpp) < 0.01 * bpp
+        back, _ = oracle.decode(a.data, oracle.FP32)
+        assert oracle.rel_l2(W, back) < 0.02
+    # frequency normalisation itself ends even when no valid table exists (more symbols than slots)
+    f = oracle.normalise_freqs(np.ones(600, np.uint64), 9)
+    assert f.min() == 1 and f.sum() == 600
+
+
 def test_library_stream_decodes_with_the_oracle():
     W = synth.laplace_rows(64, 1024, 8)
     blob = ep.encode(W, 4.0, tile_vectors=77)
