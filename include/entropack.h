@@ -222,7 +222,10 @@ int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const voi
 /* Device-side integrity word.  The kernel ORs in a flag when a tile does not end with every state
  * at 2^15 and its word pointer at the next tile's offset (a damaged stream).  This call
  * synchronises `stream`, returns EP_OK or EP_ERR_BAD_STREAM / EP_ERR_CUDA, and clears the word.
- * For tests and debugging; not needed on the hot path. */
+ * For tests and debugging; not needed on the hot path.  The decode kernels take every address bound
+ * from `info` (sizes, counts, offsets), never from the stream's contents: damaged tables, tile records
+ * or payload give wrong weights and this flag, not an access outside the buffers `info` describes.
+ * `info` itself must match the buffers (ep_blob_info / ep_validate on the host copy). */
 int ep_last_device_status(void *stream);
 
 /* ---- misc --------------------------------------------------------------------------------- */

@@ -178,6 +178,9 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
         }
         run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
+    // frequencies of a damaged stream may sum to less than 2^b: no slot keeps what an earlier CTA left there
+    // (the coset entry's code field is added to a shared-memory address)
+    for (uint32_t u = run + lane; u < (1u << J.b) && u < kLutEntries; u += 32) sts32(base + 4u * u, 0u);
   }
 }
 
@@ -318,7 +321,8 @@ __device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &wa, uint32_t
     uint32_t e[9];
     e[0] = TAIL ? rans_step_tail(x, lut_addr + kCosetTableOff, mask, b, wa, lt, act)
                 : rans_step<kCosetTableOff>(x, lut_addr, mask, b, wa, lt);
-    const uint32_t coff = e[0] & kCodeMask;          // 0 or 65536: byte offset of this coset's tables
+    // 0 or 65536: byte offset of this coset's tables (one bit only, so that a damaged table cannot point elsewhere)
+    const uint32_t coff = e[0] & 0x10000u;
     const uint32_t tab = lut_addr + coff;
     if (TAIL) {
 #pragma unroll
@@ -402,7 +406,7 @@ template <int DT, bool WIDE>
 __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
     uint32_t x = rec[lane];
-    const uint32_t off = rec[32];
+    const uint32_t off = min(rec[32], J.total_words);   // a damaged index must not move reads outside the payload
     const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
     const uint32_t v0 = tile * J.V;
     const uint32_t nv = min(J.V, J.n_vec - v0);
@@ -703,7 +707,7 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
                                                  uint32_t ring, uint32_t lane) {
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
     uint32_t x = rec[lane];
-    const uint32_t off = rec[32];
+    const uint32_t off = min(rec[32], J.total_words);   // a damaged index must not move reads outside the payload
     const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
     const uint32_t v0 = tile * J.V;
     const uint32_t nv = valid ? min(J.V, J.n_vec - v0) : 0u;
