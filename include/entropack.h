@@ -161,7 +161,11 @@ int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int32_t b, uin
  * aligned), d_workspace a 256-byte aligned device buffer of ep_encode_device_workspace_bytes() bytes
  * (about 54 bytes per 8-weight block).  The call enqueues on `stream` and synchronises it several times;
  * it returns the finished host blob.  EP_ERR_UNSUPPORTED (use ep_encode instead) if a lattice coordinate
- * exceeds +-4095 or the tables hold more than 40960 symbols in total. */
+ * exceeds +-4095 or the tables hold more than 40960 symbols in total.
+ * The blob of this call lives in page-locked host memory (the device copies the payload straight into it,
+ * and a later upload of the blob runs at full bus speed).  Page-locking costs milliseconds, so ep_blob_free
+ * keeps the buffer of the most recently freed such blob (one per process at most, the larger one when two
+ * compete) for the next call whose blob fits; a model converted tensor by tensor allocates once or twice. */
 size_t ep_encode_device_workspace_bytes(uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts);
 int ep_encode_device(const float *d_W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts,
                      void *d_workspace, size_t workspace_bytes, void *stream, ep_blob **out);

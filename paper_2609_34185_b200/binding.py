@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+import weakref
 
 import numpy as np
 
@@ -153,8 +154,9 @@ def _take(handle: C.c_void_p) -> Blob:
     n = L.ep_blob_bytes(handle)
     rep = EncodeReport()
     L.ep_blob_report(handle, C.byref(rep))
-    data = np.ctypeslib.as_array(C.cast(L.ep_blob_data(handle), C.POINTER(C.c_uint8)), shape=(n,)).copy()
-    L.ep_blob_free(handle)
+    # no copy: the array views the library's buffer, which is freed when the array (and every view of it) is gone
+    data = np.ctypeslib.as_array(C.cast(L.ep_blob_data(handle), C.POINTER(C.c_uint8)), shape=(n,))
+    weakref.finalize(data, L.ep_blob_free, handle)
     return Blob(data, rep.as_dict())
 
 

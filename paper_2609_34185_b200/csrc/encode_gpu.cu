@@ -8,6 +8,8 @@
 // order written with explicit add / multiply intrinsics so that nothing is fused.
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include <algorithm>
 #include <cmath>
 #include <cstring>
@@ -293,6 +295,43 @@ Workspace carve(uint8_t *base, uint32_t R, uint32_t C, uint32_t V) {
         if ((call) != cudaSuccess) return EP_ERR_CUDA; \
     } while (0)
 
+// Page-locked host memory for finished blobs.  Locking tens of MB costs milliseconds, so the buffer of the
+// most recently freed blob is kept (one at most) and handed to the next encode that fits into it.
+std::mutex g_pinned_lock;
+uint8_t *g_pinned_spare = nullptr;
+size_t g_pinned_spare_cap = 0;
+
+uint8_t *pinned_acquire(size_t n, size_t *cap) {
+    {
+        std::lock_guard<std::mutex> hold(g_pinned_lock);
+        if (g_pinned_spare && g_pinned_spare_cap >= n) {
+            uint8_t *p = g_pinned_spare;
+            *cap = g_pinned_spare_cap;
+            g_pinned_spare = nullptr;
+            g_pinned_spare_cap = 0;
+            return p;
+        }
+    }
+    const size_t want = n + n / 8 + 4096;           // headroom: the next tensor of a model is rarely the same size
+    void *p = nullptr;
+    if (cudaHostAlloc(&p, want, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    *cap = want;
+    return static_cast<uint8_t *>(p);
+}
+
+void pinned_release(uint8_t *p, size_t cap) {
+    uint8_t *drop = p;
+    {
+        std::lock_guard<std::mutex> hold(g_pinned_lock);
+        if (cap > g_pinned_spare_cap) {               // keep the larger of the two
+            drop = g_pinned_spare;
+            g_pinned_spare = p;
+            g_pinned_spare_cap = cap;
+        }
+    }
+    if (drop) cudaFreeHost(drop);
+}
+
 class DeviceBackend final : public EncodeBackend {
 public:
     DeviceBackend(const float *dW, uint32_t R, uint32_t C, uint32_t V, uint8_t *ws, cudaStream_t st)
@@ -340,16 +379,22 @@ public:
         EP_CUDA(cudaMemcpyAsync(w_.offsets, offsets.data(), 4ull * (n_tiles + 1), cudaMemcpyHostToDevice, st_));
         compact_kernel<<<(n_tiles + 7) / 8, 256, 0, st_>>>(w_.scratch, cap, w_.counts, w_.offsets, n_tiles, w_.payload);
         EP_CUDA(cudaGetLastError());
-        std::vector<uint16_t> payload(size_t(total) + 1);
         std::vector<uint32_t> states(size_t(n_tiles) * 32);
         std::vector<float> sigma(R_);
-        if (total) EP_CUDA(cudaMemcpyAsync(payload.data(), w_.payload, 2ull * total, cudaMemcpyDeviceToHost, st_));
         EP_CUDA(cudaMemcpyAsync(states.data(), w_.states, 128ull * n_tiles, cudaMemcpyDeviceToHost, st_));
         EP_CUDA(cudaMemcpyAsync(sigma.data(), w_.sigma, 4ull * R_, cudaMemcpyDeviceToHost, st_));
         EP_CUDA(cudaStreamSynchronize(st_));
-        std::vector<const uint16_t *> ptr(n_tiles);
-        for (uint32_t t = 0; t < n_tiles; ++t) ptr[t] = payload.data() + offsets[t];
-        return assemble_blob(m, R_, C_, b, V, sigma.data(), s, states.data(), ptr.data(), counts.data(), out);
+        // everything but the payload is laid out on the host; the compacted payload is copied straight into its place
+        uint64_t payload_at = 0;
+        out->acquire = pinned_acquire;
+        out->release = pinned_release;
+        const int rc = assemble_blob(m, R_, C_, b, V, sigma.data(), s, states.data(), nullptr, counts.data(), out, &payload_at);
+        if (rc) return rc;
+        if (total) {
+            EP_CUDA(cudaMemcpyAsync(out->data() + payload_at, w_.payload, 2ull * total, cudaMemcpyDeviceToHost, st_));
+            EP_CUDA(cudaStreamSynchronize(st_));
+        }
+        return EP_OK;
     }
 
 private:

@@ -207,7 +207,8 @@ std::vector<uint32_t> sample_rows(uint32_t R, uint32_t C, uint32_t budget_vector
 
 // header + tables + scales + tile index + payload
 int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
-                  const uint32_t *states, const uint16_t *const *tile_words, const uint32_t *tile_len, ep_blob *out) {
+                  const uint32_t *states, const uint16_t *const *tile_words, const uint32_t *tile_len, ep_blob *out,
+                  uint64_t *payload_offset) {
     const uint64_t nvec = uint64_t(R) * (C / 8);
     const uint32_t n_tiles = uint32_t((nvec + V - 1) / V);
     uint64_t total_words = 0;
@@ -230,9 +231,10 @@ int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, con
     const uint64_t off_tables = kHeaderBytes, off_scales = off_tables + tb_bytes, off_tiles = off_scales + 4ull * R;
     const uint64_t off_payload = off_tiles + uint64_t(kTileRecordBytes) * n_tiles + 4, total = off_payload + 2 * total_words;
     if (total >= (1ull << 32)) return EP_ERR_UNSUPPORTED;   // section offsets are 32-bit
-    std::vector<uint8_t> &B = out->bytes;
-    B.assign(size_t(total), 0);
-    uint8_t *p = B.data();
+    uint8_t *p = out->allocate(size_t(total));   // uninitialised: everything before the payload is zeroed here,
+    if (!p) return EP_ERR_NOMEM;                 // the payload is written whole below or by the caller
+    std::memset(p, 0, size_t(off_payload));
+    if (payload_offset) *payload_offset = off_payload;
     store_le<uint32_t>(p, kMagic);
     store_le<uint16_t>(p + 4, 1);
     p[6] = uint8_t(b);
@@ -263,7 +265,7 @@ int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, con
         uint8_t *rec = p + off_tiles + uint64_t(kTileRecordBytes) * t;
         std::memcpy(rec, states + size_t(t) * kStates, 4 * kStates);
         store_le<uint32_t>(rec + 4 * kStates, uint32_t(at));
-        if (tile_len[t]) std::memcpy(p + off_payload + 2 * at, tile_words[t], 2ull * tile_len[t]);
+        if (tile_words && tile_len[t]) std::memcpy(p + off_payload + 2 * at, tile_words[t], 2ull * tile_len[t]);
         at += tile_len[t];
     }
     store_le<uint32_t>(p + off_tiles + uint64_t(kTileRecordBytes) * n_tiles, uint32_t(at));
@@ -361,8 +363,8 @@ int run_encode(EncodeBackend &be, uint32_t R, uint32_t C, double target_bpp, con
     if (rc) { delete blob; return rc; }
     blob->report.s = double(s);
     blob->report.b = b;
-    blob->report.bytes = blob->bytes.size();
-    blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
+    blob->report.bytes = blob->size();
+    blob->report.stored_bpp = 8.0 * double(blob->size()) / (double(R) * double(C));
     blob->report.est_bpp_sample = last_rate;
     blob->report.cce_bits = full.cross_entropy_bits(b);
     blob->report.sample_rows = uint32_t(rows.size());
@@ -792,8 +794,8 @@ extern "C" int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int
         if (rc) { delete blob; return rc; }
         blob->report.s = double(s_info);
         blob->report.b = b;
-        blob->report.bytes = blob->bytes.size();
-        blob->report.stored_bpp = 8.0 * double(blob->bytes.size()) / (double(R) * double(C));
+        blob->report.bytes = blob->size();
+        blob->report.stored_bpp = 8.0 * double(blob->size()) / (double(R) * double(C));
         blob->report.cce_bits = m.cross_entropy_bits(b);
         *out = blob;
         return EP_OK;
@@ -804,8 +806,8 @@ extern "C" int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int
     }
 }
 
-extern "C" const void *ep_blob_data(const ep_blob *b) { return b ? b->bytes.data() : nullptr; }
-extern "C" size_t ep_blob_bytes(const ep_blob *b) { return b ? b->bytes.size() : 0; }
+extern "C" const void *ep_blob_data(const ep_blob *b) { return b ? b->data() : nullptr; }
+extern "C" size_t ep_blob_bytes(const ep_blob *b) { return b ? b->size() : 0; }
 extern "C" int ep_blob_report(const ep_blob *b, ep_encode_report *out) {
     if (!b || !out) return EP_ERR_BAD_ARG;
     *out = b->report;

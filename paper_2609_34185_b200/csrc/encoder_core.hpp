@@ -4,13 +4,54 @@
 // (encode_gpu.cu).  Both back ends produce byte-identical streams for the same input.
 #pragma once
 #include <cstdint>
+#include <memory>
+#include <new>
+#include <utility>
 #include <vector>
 
 #include "stream.hpp"
 
+// allocator whose resize() leaves new bytes uninitialised (a blob of tens of MB is written exactly once)
+template <class T>
+struct ep_no_init_allocator : std::allocator<T> {
+    template <class U> struct rebind { using other = ep_no_init_allocator<U>; };
+    ep_no_init_allocator() = default;
+    template <class U> ep_no_init_allocator(const ep_no_init_allocator<U> &) {}
+    template <class U> void construct(U *p) { ::new (static_cast<void *>(p)) U; }
+    template <class U, class... A> void construct(U *p, A &&...a) { ::new (static_cast<void *>(p)) U(std::forward<A>(a)...); }
+};
+
+// Host storage of a stored representation.  By default ordinary heap memory; a back end may install its
+// own source (the GPU back end: page-locked memory, which the device copies into at full bus speed and
+// which a later upload reads at full speed too) before the blob is assembled.
 struct ep_blob {
-    std::vector<uint8_t> bytes;
+    std::vector<uint8_t, ep_no_init_allocator<uint8_t>> heap;
+    uint8_t *ext = nullptr;                                  // storage obtained through `acquire`
+    size_t ext_size = 0, ext_cap = 0;
+    uint8_t *(*acquire)(size_t n, size_t *cap) = nullptr;    // nullptr on failure
+    void (*release)(uint8_t *p, size_t cap) = nullptr;
     ep_encode_report report{};
+
+    ep_blob() = default;
+    ep_blob(const ep_blob &) = delete;
+    ep_blob &operator=(const ep_blob &) = delete;
+    ~ep_blob() { if (ext && release) release(ext, ext_cap); }
+    // n bytes of uninitialised storage (replaces what the blob held); nullptr if the source has none
+    uint8_t *allocate(size_t n) {
+        if (acquire) {
+            if (ext && release) release(ext, ext_cap);
+            ext_size = ext_cap = 0;
+            ext = acquire(n, &ext_cap);
+            if (!ext) return nullptr;
+            ext_size = n;
+            return ext;
+        }
+        heap.resize(n);
+        return heap.data();
+    }
+    const uint8_t *data() const { return ext ? ext : heap.data(); }
+    uint8_t *data() { return ext ? ext : heap.data(); }
+    size_t size() const { return ext ? ext_size : heap.size(); }
 };
 
 namespace ep {
@@ -49,9 +90,11 @@ double estimate_bits(const Model &m, int b, uint64_t nvec, uint64_t rows, uint32
 std::vector<uint32_t> sample_rows(uint32_t R, uint32_t C, uint32_t budget_vectors);
 
 // header + tables + scales + tile index + payload; `states` holds 32 words per tile, tile t's payload is
-// tile_words[t] .. + tile_len[t]
+// tile_words[t] .. + tile_len[t].  With tile_words == nullptr the payload section is left unwritten for the
+// caller to fill in place: it starts at out->bytes.data() + *payload_offset and holds the tiles back to back.
 int assemble_blob(const Model &m, uint32_t R, uint32_t C, int b, uint32_t V, const float *sigma, float s_info,
-                  const uint32_t *states, const uint16_t *const *tile_words, const uint32_t *tile_len, ep_blob *out);
+                  const uint32_t *states, const uint16_t *const *tile_words, const uint32_t *tile_len, ep_blob *out,
+                  uint64_t *payload_offset = nullptr);
 
 // What a back end must provide.  Each call returns an ep_status.
 struct EncodeBackend {

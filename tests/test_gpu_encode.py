@@ -57,3 +57,32 @@ def test_device_encoder_leaves_the_per_row_refinement_to_the_host():
     with pytest.raises(ep.EntroPackError) as ei:
         ep.encode_device(torch.from_numpy(W).cuda(), 4.0, rdo_candidates=3)
     assert ei.value.status == -3
+
+
+def test_device_encoder_blobs_keep_their_bytes_while_buffers_are_reused():
+    # finished blobs live in page-locked memory and a freed blob's buffer serves a later encode: a blob that is
+    # still alive must never be overwritten, a reused buffer must give the same bytes as a fresh one
+    import gc
+    Wa, Wb = synth.gaussian_rows(256, 1024, 71), synth.laplace_rows(192, 2048, 72)
+    da, db = torch.from_numpy(Wa).cuda(), torch.from_numpy(Wb).cuda()
+    ref_a, ref_b = ep.encode(Wa, 4.0).data.copy(), ep.encode(Wb, 3.0).data.copy()
+    a1 = ep.encode_device(da, 4.0)
+    b1 = ep.encode_device(db, 3.0)                 # a1 alive: must come from another buffer
+    assert np.array_equal(a1.data, ref_a) and np.array_equal(b1.data, ref_b)
+    view = a1.data[100:200]
+    keep = view.copy()
+    del a1
+    gc.collect()                                   # `view` still holds the buffer
+    b2 = ep.encode_device(db, 3.0)
+    assert np.array_equal(view, keep) and np.array_equal(b2.data, ref_b)
+    del view, b1, b2
+    gc.collect()
+    for _ in range(3):                             # now buffers come back from the spare slot
+        a = ep.encode_device(da, 4.0)
+        assert np.array_equal(a.data, ref_a)
+        del a
+        gc.collect()
+        b = ep.encode_device(db, 3.0)
+        assert np.array_equal(b.data, ref_b)
+        del b
+        gc.collect()
