@@ -131,10 +131,13 @@ typedef struct {
     const void *d_tile_index;   /* device: the tile-index section (132*n_tiles + 4 bytes); 4-byte aligned */
     const float *d_row_scales;  /* device: R fp32 row scales (the blob's, or the caller's own) */
     int32_t out_dtype;          /* ep_dtype */
-    void *d_out;                /* device: R*C elements of out_dtype, row-major; 16-byte aligned */
+    void *d_out;                /* device: R*C elements of out_dtype, row-major; 16-byte aligned (8 bytes are
+                                   enough for the one-byte types, 4 for EP_FIELDS_I32) */
     void *d_scratch;            /* device: ep_decode_scratch_bytes(info) bytes, 256-byte aligned; may be
                                    NULL when that size is 0 */
     size_t scratch_bytes;
+    uint32_t tile_begin;        /* a range of tiles to decode, for a caller that owns a shard of the tensor */
+    uint32_t tile_count;        /* (both 0 = the whole tensor); see ep_decode_tiles */
 } ep_decode_job;
 
 /* ---- host encoder ------------------------------------------------------------------------- */
@@ -196,6 +199,17 @@ size_t ep_decode_scratch_bytes(const ep_info *info);
 int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_tile_index,
                      const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
                      size_t scratch_bytes, void *stream);
+
+/* Tiles are independently decodable (Sec. 3.6): this call decodes tiles [tile_begin, tile_begin + tile_count)
+ * only, i.e. blocks [tile_begin * V, min((tile_begin + tile_count) * V, R*C/8)) of the row-major block
+ * sequence, and writes nothing else.  d_out is still the address of element (0, 0) of the full tensor: a
+ * caller that holds only its shard passes shard_base - first_block * 8 * sizeof(element) (which must keep
+ * d_out's alignment; it is never dereferenced outside the shard).  d_row_scales is indexed by the tensor's row
+ * numbers likewise.  tile_count >= 1, tile_begin + tile_count <= n_tiles, else EP_ERR_BAD_ARG.  With this,
+ * ranks of a tensor-parallel job decode disjoint row ranges of one stream without any exchange. */
+int ep_decode_tiles(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                    const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
+                    size_t scratch_bytes, uint32_t tile_begin, uint32_t tile_count, void *stream);
 
 /* The same for up to EP_MAX_BATCH tensors in one kernel launch (independent tiles of all tensors
  * share the grid).  Jobs needing scratch get their lookup tables built by one extra launch first. */

@@ -61,7 +61,8 @@ class Info(C.Structure):
 class DecodeJob(C.Structure):
     _fields_ = [("info", C.POINTER(Info)), ("d_stream", C.c_void_p), ("d_tile_index", C.c_void_p),
                 ("d_row_scales", C.c_void_p), ("out_dtype", C.c_int32), ("d_out", C.c_void_p),
-                ("d_scratch", C.c_void_p), ("scratch_bytes", C.c_size_t)]
+                ("d_scratch", C.c_void_p), ("scratch_bytes", C.c_size_t),
+                ("tile_begin", C.c_uint32), ("tile_count", C.c_uint32)]
 
 
 _lib = None
@@ -96,6 +97,8 @@ def load():
     L.ep_decode_scratch_bytes.argtypes = [C.POINTER(Info)]
     L.ep_decode_tensor.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ep_decode_tiles.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                  C.c_void_p, C.c_size_t, C.c_uint32, C.c_uint32, C.c_void_p]
     L.ep_decode_tensor_static.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                           C.c_void_p]
     L.ep_decode_batch.argtypes = [C.POINTER(DecodeJob), C.c_int32, C.c_void_p]
@@ -231,6 +234,15 @@ def decode_tensor(info: Info, d_stream: int, d_tile_index: int, d_row_scales: in
                                    d_scratch or None, scratch_bytes, stream or None), "ep_decode_tensor")
 
 
+def decode_tiles(info: Info, d_stream: int, d_tile_index: int, d_row_scales: int, out_dtype: int, d_out: int,
+                 tile_begin: int, tile_count: int, d_scratch: int = 0, scratch_bytes: int = 0, stream: int = 0) -> None:
+    """ep_decode_tiles: decode tiles [tile_begin, tile_begin + tile_count) only; d_out is the address element
+    (0, 0) of the full tensor has (or would have: a shard holder passes its base minus the shard's offset)."""
+    _check(load().ep_decode_tiles(C.byref(info), d_stream, d_tile_index, d_row_scales, out_dtype, d_out,
+                                  d_scratch or None, scratch_bytes, tile_begin, tile_count, stream or None),
+           "ep_decode_tiles")
+
+
 def decode_tensor_static(info: Info, d_stream: int, d_tile_index: int, d_row_scales: int, out_dtype: int, d_out: int,
                          stream: int = 0) -> None:
     """ep_decode_tensor_static: the same decode for callers that cannot allocate a scratch buffer; large lookup
@@ -311,6 +323,24 @@ def decode(dblob: DeviceBlob, out_dtype: int = BF16, out=None, row_scales=None, 
     decode_tensor(I, dblob.d_stream, dblob.d_tile_index, sc, out_dtype, out.data_ptr(),
                   dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
                   dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
+    return out
+
+
+def decode_tile_range(dblob: DeviceBlob, tiles: range, out_dtype: int = BF16, out=None, stream=None):
+    """Decode a contiguous range of tiles into a buffer that holds exactly their blocks: a flat tensor of
+    (blocks of the range) * 8 elements, allocated here unless given.  The shard of a tensor-parallel rank."""
+    torch = _torch()
+    I = dblob.info
+    nvec = I.R * (I.C // 8)
+    first, last = tiles.start * I.V, min(tiles.stop * I.V, nvec)
+    esize = DTYPE_BYTES[out_dtype]
+    if out is None:
+        out = torch.empty((last - first) * 8, dtype=_out_torch_dtype(out_dtype), device=dblob.dev.device)
+    assert out.numel() >= (last - first) * 8 and out.data_ptr() % 16 == 0
+    decode_tiles(I, dblob.d_stream, dblob.d_tile_index, dblob.d_row_scales, out_dtype,
+                 out.data_ptr() - first * 8 * esize, tiles.start, len(tiles),
+                 dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
+                 dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
     return out
 
 

@@ -55,10 +55,11 @@ struct JobParams {
     uint32_t total_words;
     uint32_t n_vec;
     uint32_t per_row;             // C / 8
-    uint32_t V, n_tiles, b;
+    uint32_t V, n_tiles, b;       // n_tiles: tiles of the whole tensor
+    uint32_t tile0, tile_cnt;     // the tiles this launch decodes: [tile0, tile0 + tile_cnt)
     int32_t zlo;                  // even, <= -2
     uint32_t cta_begin, cta_count;
-    uint32_t iters;               // ceil(n_tiles / (cta_count * warps)): every warp runs this many rounds
+    uint32_t iters;               // ceil(tile_cnt / (cta_count * warps)): every warp runs this many rounds
     int16_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint16_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
@@ -782,22 +783,23 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
     build_tables_smem(J, lut_addr, warp, lane);
     __syncthreads();
     const uint32_t cta = blockIdx.x - J.cta_begin;
-    // Rounds over the tiles: warp w of CTA c takes tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and the
+    // Rounds over the job's tiles: warp w of CTA c takes the job's tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and the
     // test for a CTA past the end depend on blockIdx and kernel parameters only, so the compiler sees warp-uniform
     // control flow and puts no divergence guards around the warp votes of the hot loop; inside the one CTA that
     // straddles the end, a warp past the last tile goes through the same code with zero groups to do.
     const bool wide = J.per_row >= 32u;
     for (uint32_t i = 0; i < J.iters; ++i) {
         const uint32_t base = (cta + i * J.cta_count) * kWarps;
-        if (base >= J.n_tiles) break;
-        const uint32_t tile = base + warp;
+        if (base >= J.tile_cnt) break;
+        const bool mine = base + warp < J.tile_cnt;
+        const uint32_t tile = J.tile0 + min(base + warp, J.tile_cnt - 1u);
         if constexpr (DT != EP_FIELDS_I32) {
             if (wide && J.V < (1u << 20)) {
-                decode_tile_fast<DT>(J, min(tile, J.n_tiles - 1u), tile < J.n_tiles, lut_addr, ring, lane);
+                decode_tile_fast<DT>(J, tile, mine, lut_addr, ring, lane);
                 continue;
             }
         }
-        if (tile < J.n_tiles) {
+        if (mine) {
             if (wide) decode_tile<DT, true>(J, tile, lut_addr, ring, lane);
             else decode_tile<DT, false>(J, tile, lut_addr, ring, lane);
         }
@@ -827,6 +829,7 @@ struct GJobParams {
     uint32_t n_vec;
     uint32_t per_row;
     uint32_t V, n_tiles, b;
+    uint32_t tile0, tile_cnt;     // the tiles this launch decodes
     uint32_t cta_begin, cta_count;
 };
 
@@ -923,7 +926,8 @@ __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_
     const uint32_t last_word = J.total_words ? J.total_words - 1u : 0u;
     const uint32_t cta = blockIdx.x - J.cta_begin;
     const uint32_t foff0 = s_foff[0];
-    for (uint32_t tile = cta * kGWarps + warp; tile < J.n_tiles; tile += J.cta_count * kGWarps) {
+    for (uint32_t local = cta * kGWarps + warp; local < J.tile_cnt; local += J.cta_count * kGWarps) {
+        const uint32_t tile = J.tile0 + local;
         const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
         uint32_t x = rec[lane];
         uint32_t ptr = rec[32];
@@ -966,6 +970,10 @@ __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_
 }
 
 // ---- host side -----------------------------------------------------------------------------------
+
+// the tiles a job asks for: its range, or the whole tensor when both range fields are 0
+inline uint32_t job_tile0(const ep_decode_job &jb) { return jb.tile_count ? jb.tile_begin : 0u; }
+inline uint32_t job_tiles(const ep_decode_job &jb) { return jb.tile_count ? jb.tile_count : jb.info->n_tiles; }
 
 int g_num_sms = 0;
 
@@ -1075,7 +1083,9 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
         J.V = I.V;
         J.n_tiles = I.n_tiles;
         J.b = I.b;
-        const uint64_t want = (uint64_t(I.n_tiles) + kGWarps - 1) / kGWarps;
+        J.tile0 = job_tile0(jb);
+        J.tile_cnt = job_tiles(jb);
+        const uint64_t want = (uint64_t(J.tile_cnt) + kGWarps - 1) / kGWarps;
         const uint64_t cap = uint64_t(sms) * 8u;
         J.cta_begin = next;
         J.cta_count = uint32_t(want < cap ? want : cap);
@@ -1126,14 +1136,19 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         if (dt != EP_FIELDS_I32 && !jb.d_row_scales) return EP_ERR_BAD_ARG;
         const ep_info &I = *jb.info;
         if (I.C == 0 || I.C % 8 || I.R == 0 || I.V == 0 || I.b < 9 || I.b > 15 || I.J != ep::kStates) return EP_ERR_BAD_ARG;
+        // one vector store per block: 16 bytes for the two-byte types (two of them for FP32), 8 for the one-byte types
+        const uintptr_t out_mask = dt == EP_FIELDS_I32 ? 3u : (dt == EP_FP8_E4M3 || dt == EP_FP8_E5M2 || dt == EP_INT8 || dt == EP_UINT8) ? 7u : 15u;
         if ((reinterpret_cast<uintptr_t>(jb.d_stream) & 3) || (reinterpret_cast<uintptr_t>(jb.d_tile_index) & 3) ||
-            (reinterpret_cast<uintptr_t>(jb.d_out) & 15))
+            (reinterpret_cast<uintptr_t>(jb.d_out) & out_mask))
             return EP_ERR_BAD_ARG;
         if (I.table_K[0] == 0 || I.table_min[0] < 0 || int64_t(I.table_min[0]) + I.table_K[0] > 2) return EP_ERR_BAD_STREAM;
         // 32-bit byte offsets into the output (one row and one group beyond the end still representable) and a
         // signed 32-bit payload remainder in the kernels
         if ((uint64_t(I.R) + 1u) * I.C * 4u + 1024u >= (1ull << 32) || I.total_words >= (1ull << 30)) return EP_ERR_UNSUPPORTED;
-        if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; tiles_total += I.n_tiles; }
+        if (jb.tile_count != 0 || jb.tile_begin != 0) {     // a tile range: inside the tensor and not empty
+            if (jb.tile_count == 0 || jb.tile_begin >= I.n_tiles || jb.tile_count > I.n_tiles - jb.tile_begin) return EP_ERR_BAD_ARG;
+        }
+        if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; tiles_total += job_tiles(jb); }
         else large[n_large++] = &jb;
     }
     if (n_large) {
@@ -1152,8 +1167,9 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         const ep_decode_job &jb = *fast[i];
         const ep_info &I = *jb.info;
         JobParams &J = P.job[i];
-        const uint64_t want = (uint64_t(I.n_tiles) + kWarps - 1) / kWarps;
-        uint64_t share = (budget * I.n_tiles + tiles_total - 1) / tiles_total;
+        const uint32_t my_tiles = job_tiles(jb);
+        const uint64_t want = (uint64_t(my_tiles) + kWarps - 1) / kWarps;
+        uint64_t share = (budget * my_tiles + tiles_total - 1) / tiles_total;
         if (share < 1) share = 1;
         if (share > want) share = want;
         J.stream = static_cast<const uint8_t *>(jb.d_stream);
@@ -1167,12 +1183,14 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.per_row = I.C / 8;
         J.V = I.V;
         J.n_tiles = I.n_tiles;
+        J.tile0 = job_tile0(jb);
+        J.tile_cnt = my_tiles;
         J.b = I.b;
         J.zlo = int32_t(even_base(coord_range(I)));
         J.cta_begin = next;
         J.cta_count = uint32_t(share);
         const uint32_t round_tiles = J.cta_count * uint32_t(kWarps);
-        J.iters = (J.n_tiles + round_tiles - 1u) / round_tiles;
+        J.iters = (J.tile_cnt + round_tiles - 1u) / round_tiles;
         uint32_t acc = 0;
         for (int t = 0; t < EP_NUM_TABLES; ++t) {
             J.tmin[t] = int16_t(I.table_min[t]);
@@ -1197,6 +1215,24 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     return e == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
+extern "C" int ep_decode_tiles(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                               const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
+                               size_t scratch_bytes, uint32_t tile_begin, uint32_t tile_count, void *stream) {
+    if (tile_count == 0) return EP_ERR_BAD_ARG;
+    ep_decode_job jb;
+    jb.info = info;
+    jb.d_stream = d_stream;
+    jb.d_tile_index = d_tile_index;
+    jb.d_row_scales = d_row_scales;
+    jb.out_dtype = out_dtype;
+    jb.d_out = d_out;
+    jb.d_scratch = d_scratch;
+    jb.scratch_bytes = scratch_bytes;
+    jb.tile_begin = tile_begin;
+    jb.tile_count = tile_count;
+    return ep_decode_batch(&jb, 1, stream);
+}
+
 extern "C" int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_tile_index,
                                 const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
                                 size_t scratch_bytes, void *stream) {
@@ -1209,6 +1245,8 @@ extern "C" int ep_decode_tensor(const ep_info *info, const void *d_stream, const
     jb.d_out = d_out;
     jb.d_scratch = d_scratch;
     jb.scratch_bytes = scratch_bytes;
+    jb.tile_begin = 0;
+    jb.tile_count = 0;
     return ep_decode_batch(&jb, 1, stream);
 }
 

@@ -283,3 +283,52 @@ def test_config3_one_wide_tensor_fp8_and_int8_containers():
         else:
             Wc = np.clip(np.rint(Wc), -128, 127).astype(np.float32)
         _full_compare(Wc, 2.5, dt)
+
+
+# ---- tile ranges: the shard of a tensor-parallel rank ------------------------------------------------
+
+def test_tile_ranges_tile_the_tensor_and_write_nothing_else():
+    from paper_2609_34185_b200.sharding import shard_range
+    for W, bpp, V, dt, odt in ((synth.gaussian_rows(96, 1024, 21), 4.0, 100, ep.BF16, oracle.BF16),
+                               (synth.laplace_rows(40, 264, 22), 3.0, 33, ep.FP8_E4M3, oracle.E4M3),
+                               (synth.laplace_rows(64, 2048, 23), 8.0, 0, ep.FP16, oracle.FP16)):      # b = 12 path
+        blob = ep.encode(W, bpp, tile_vectors=V)
+        d = ep.upload(blob)
+        I = blob.info
+        ref, _ = oracle.decode(blob.data, odt)
+        ref = np.ascontiguousarray(ref).reshape(-1).view(np.uint8)
+        es = ep.DTYPE_BYTES[dt]
+        nvec = I.R * (I.C // 8)
+        for world in (1, 2, 3, 5):
+            pieces = []
+            for rank in range(world):
+                tiles = shard_range(I.n_tiles, world, rank)
+                if len(tiles) == 0:
+                    continue
+                out = ep.decode_tile_range(d, tiles, dt)
+                torch.cuda.synchronize()
+                first, last = tiles.start * I.V, min(tiles.stop * I.V, nvec)
+                got = out.view(torch.uint8).cpu().numpy().reshape(-1)
+                assert got.size == (last - first) * 8 * es
+                assert np.array_equal(got, ref[first * 8 * es:last * 8 * es]), (W.shape, world, rank)
+                part, _ = oracle.decode(blob.data, odt, tiles=(tiles.start, tiles.stop))     # the oracle's own range decode
+                part = np.ascontiguousarray(part).reshape(-1).view(np.uint8)
+                assert np.array_equal(got, part[first * 8 * es:last * 8 * es])
+                pieces.append(got)
+            assert np.array_equal(np.concatenate(pieces), ref)
+        # in place in a full-size buffer: bytes outside the range keep their fill value
+        full = torch.full((I.R * I.C * es,), 0xA5, dtype=torch.uint8, device="cuda")
+        t0, cnt = I.n_tiles // 3, max(1, I.n_tiles // 3)
+        ep.decode_tiles(I, d.d_stream, d.d_tile_index, d.d_row_scales, dt, full.data_ptr(), t0, cnt,
+                        d.scratch.data_ptr() if d.scratch is not None else 0,
+                        d.scratch.numel() if d.scratch is not None else 0)
+        torch.cuda.synchronize()
+        got = full.cpu().numpy()
+        a, b = t0 * I.V * 8 * es, min((t0 + cnt) * I.V, nvec) * 8 * es
+        assert np.array_equal(got[a:b], ref[a:b]) and np.all(got[:a] == 0xA5) and np.all(got[b:] == 0xA5)
+        assert ep.last_device_status() == 0
+        for bad in ((I.n_tiles, 1), (0, I.n_tiles + 1), (1, 0)):
+            with pytest.raises(ep.EntroPackError):
+                ep.decode_tiles(I, d.d_stream, d.d_tile_index, d.d_row_scales, dt, full.data_ptr(), bad[0], bad[1],
+                                d.scratch.data_ptr() if d.scratch is not None else 0,
+                                d.scratch.numel() if d.scratch is not None else 0)

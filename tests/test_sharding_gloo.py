@@ -40,6 +40,16 @@ def _worker(rank, world, port, q):
         assert 0 <= r0 < r1 <= shapes[i][0]
         nbytes += len(blob)
         params += W.size
+    # one tensor split by tile ranges (the shard of a tensor-parallel rank): the ranks' ranges are disjoint and
+    # cover the tensor, so the sum of their zero-filled partial decodes is the full decode
+    Wt = synth.laplace_rows(48, 512, 950)
+    bt = ep.encode(Wt, 3.0, tile_vectors=100, threads=2)
+    tiles = shard_range(bt.info.n_tiles, world, rank)
+    part, _ = oracle.decode(bt.data, oracle.BF16, tiles=(tiles.start, tiles.stop))
+    acc = torch.from_numpy(part.astype(np.int64))
+    dist.all_reduce(acc)                                         # test-only: the product path exchanges nothing
+    full, _ = oracle.decode(bt.data, oracle.BF16)
+    assert np.array_equal(acc.numpy(), full.astype(np.int64))
     t = torch.tensor([float(nbytes), float(params)], dtype=torch.float64)
     dist.all_reduce(t)                                           # whole-job totals
     tm = torch.tensor([1.0 + rank], dtype=torch.float64)
