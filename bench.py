@@ -44,8 +44,8 @@ def parse_args():
     ap.add_argument("--workload", default="c4", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--bpp", type=float, default=None, help="target bits/param (default: the workload's)")
     ap.add_argument("--tile-vectors", type=int, default=-1,
-                    help="V; 0 = the paper's default for the target rate; -1 (default) = ep_suggest_tile_vectors: "
-                         "the largest V up to the paper's default that fills whole rounds of the GPU's tile slots")
+                    help="V; 0 = the paper's default for the target rate; -1 (default) = ep_suggest_tile_vectors[_batch]: "
+                         "a V up to the paper's default that fills whole rounds of the GPU's tile slots")
     ap.add_argument("--dtype", default=None, choices=[None, "bf16", "fp16", "fp8", "int8"])
     ap.add_argument("--layers", type=int, default=48, help="c5: resident layers")
     ap.add_argument("--distinct-layers", type=int, default=2, help="c5: distinct layers actually encoded")
@@ -91,21 +91,25 @@ def make_workload(args):
     raise ValueError(w)
 
 
-def pick_tile_vectors(V, shape, bpp, slots):
-    """V < 0: single tensors get ep_suggest_tile_vectors for the GPU's tile slots; tensors of a batch (slots == 0)
-    share the grid, there the paper's default is kept but capped at its 4 bpp value (1820 vectors): the 3640-vector
-    default of the lowest rates leaves too few tiles per tensor to balance a batch."""
+def pick_tile_vectors(V, shape, bpp, slots, batch_shapes=None):
+    """V < 0: a single tensor gets ep_suggest_tile_vectors for the GPU's tile slots; the tensors of a batch (decoded by
+    one launch, `batch_shapes`) get ep_suggest_tile_vectors_batch for the GPU's SMs: one multiple of 32 up to the
+    paper's default for which the rounds of all tensors split evenly over the CTAs."""
     import paper_2609_34185_b200 as ep
     if V >= 0:
         return V
-    if slots:
-        return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots)
-    return min(ep.default_tile_vectors(bpp), 1820)
+    if batch_shapes is not None and len(batch_shapes) > 1:
+        return ep.suggest_tile_vectors_batch(batch_shapes, bpp, slots // 32)
+    return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots)
 
 
 def encode_layers(layers, bpp, V, slots):
     import paper_2609_34185_b200 as ep
-    return [[ep.encode(W, bpp, tile_vectors=pick_tile_vectors(V, W.shape, bpp, slots)) for W in mats] for mats in layers]
+    out = []
+    for mats in layers:
+        shapes = [W.shape for W in mats]
+        out.append([ep.encode(W, bpp, tile_vectors=pick_tile_vectors(V, W.shape, bpp, slots, shapes)) for W in mats])
+    return out
 
 
 # ---- clocks ------------------------------------------------------------------------------------------
@@ -207,7 +211,8 @@ def run_reference(args):
     name, dtype_name, bpp, layers = make_workload(args)
     V = args.tile_vectors
     import paper_2609_34185_b200 as ep
-    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 32))
+    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 32,
+                                                                       [W.shape for W in layers[0]]))
     I = blob.info
     # each step decodes a leading tile range (repeated if short) sized so that the whole run stays near a minute
     params, tiles, reps, threads = oracle_sample(blob, dtype_name, min(0.5, 60.0 / max(1, args.steps + args.warmup)))
@@ -308,9 +313,8 @@ def main():
 
     # every rank decodes its own replica of the workload: tiles and tensors are independent, no collective
     n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    # a single tensor gets one 32-warp CTA per SM
-    single = sum(len(m) for m in layers) == len(layers)
-    slots = 32 * n_sms if single else 0
+    # one 32-warp CTA per SM: 32 tile slots each
+    slots = 32 * n_sms
     blobs = encode_layers(layers, bpp, args.tile_vectors, slots)
     n_layers = args.layers if args.workload == "c5" else len(blobs)
     resident = [[ep.upload(b, device=dev) for b in blobs[l % len(blobs)]] for l in range(n_layers)]

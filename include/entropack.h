@@ -258,6 +258,13 @@ uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile
  * leaves SMs idle (App. "Tile layout and storage": tile size trades storage against parallelism).
  * Never below a quarter of the default (small tensors); returns the default when decode_slots is 0. */
 uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint32_t decode_slots);
+
+/* The same question for tensors that are decoded together by one ep_decode_batch launch (the blocks of a
+ * transformer layer): one tile size for all of them, a multiple of 32 not above the paper's default, chosen
+ * so that the rounds of all tensors (32 tiles per CTA and round) split over `decode_ctas` CTAs (the SM count:
+ * 148 on a B200) with the shortest last round.  R[i] x C[i] are the n tensor shapes. */
+uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint32_t *C, uint32_t n, double target_bpp,
+                                       uint32_t decode_ctas);
 int ep_version(void);
 
 #ifdef __cplusplus

@@ -107,6 +107,8 @@ def load():
     L.ep_strerror.argtypes = [C.c_int]
     L.ep_default_tile_vectors.restype = C.c_uint32
     L.ep_default_tile_vectors.argtypes = [C.c_double]
+    L.ep_suggest_tile_vectors_batch.restype = C.c_uint32
+    L.ep_suggest_tile_vectors_batch.argtypes = [C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.c_uint32, C.c_double, C.c_uint32]
     L.ep_suggest_tile_vectors.restype = C.c_uint32
     L.ep_suggest_tile_vectors.argtypes = [C.c_uint32, C.c_uint32, C.c_double, C.c_uint32]
     L.ep_encode_opts_default.argtypes = [C.POINTER(EncodeOpts)]
@@ -134,6 +136,14 @@ def default_tile_vectors(target_bpp: float) -> int:
 def suggest_tile_vectors(R: int, Cc: int, target_bpp: float, decode_slots: int = 148 * 32) -> int:
     """ep_suggest_tile_vectors: tile size that fills whole rounds of `decode_slots` concurrent tiles."""
     return load().ep_suggest_tile_vectors(R, Cc, float(target_bpp), decode_slots)
+
+
+def suggest_tile_vectors_batch(shapes, target_bpp: float, decode_ctas: int) -> int:
+    """ep_suggest_tile_vectors_batch: one tile size for tensors decoded together by one batched launch."""
+    n = len(shapes)
+    Rs = (C.c_uint32 * n)(*[int(s[0]) for s in shapes])
+    Cs = (C.c_uint32 * n)(*[int(s[1]) for s in shapes])
+    return int(load().ep_suggest_tile_vectors_batch(Rs, Cs, n, float(target_bpp), int(decode_ctas)))
 
 
 class Blob:

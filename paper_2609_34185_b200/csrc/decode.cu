@@ -27,10 +27,7 @@
 
 namespace {
 
-#ifndef EP_THREADS
-#define EP_THREADS 1024
-#endif
-constexpr int kThreads = EP_THREADS;
+constexpr int kThreads = 1024;                         // one CTA per SM: 32 warps = 32 tiles in flight
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kLutEntries = 2048;                 // 2^11 slots per table
 constexpr uint32_t kLutStride = kLutEntries * 4;       // bytes per table in shared memory
@@ -58,8 +55,9 @@ struct JobParams {
     uint32_t V, n_tiles, b;       // n_tiles: tiles of the whole tensor
     uint32_t tile0, tile_cnt;     // the tiles this launch decodes: [tile0, tile0 + tile_cnt)
     int32_t zlo;                  // even, <= -2
-    uint32_t cta_begin, cta_count;
-    uint32_t iters;               // ceil(tile_cnt / (cta_count * warps)): every warp runs this many rounds
+    uint32_t rounds;              // ceil(tile_cnt / warps): in one round the 32 warps of a CTA take 32 consecutive tiles
+    uint32_t round_cost;          // work of one round in groups of 32 vectors (ceil(V / 32))
+    uint32_t cost_begin;          // sum of rounds * round_cost over the jobs before this one
     int16_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint16_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
@@ -67,6 +65,7 @@ struct JobParams {
 
 struct BatchParams {
     JobParams job[EP_MAX_BATCH];
+    uint32_t cost_per_cta;        // ceil(sum of rounds * round_cost over all jobs / CTAs of the launch)
     int32_t n_jobs;
 };
 
@@ -358,14 +357,8 @@ __device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &wa, uint32_t
         for (int k = 1; k <= 7; ++k) xb[k - 1] = (e[k] & kCodeMask) | kExp4096;
         xb[7] = (e[8] & kCodeMask) | par | kExp4096;
         float w[8];
-#ifdef EP_SCALAR_FP32
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w[i] = __fmul_rn(__fsub_rn(__uint_as_float(xb[i]), __uint_as_float(kc)), sigma);
-        (void)kk; (void)ss;
-#else
 #pragma unroll
         for (int i = 0; i < 8; i += 2) unpack64(mul2(sub2(pack64(xb[i], xb[i + 1]), kk), ss), w[i], w[i + 1]);
-#endif
         Out<DT>::store(dst, w);
     }
 }
@@ -771,37 +764,50 @@ __device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t ti
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
 }
 
-template <int DT>
+// One persistent CTA per SM.  The rounds of all jobs of the launch form one list (job after job); CTA k takes the
+// rounds whose cumulative cost at their start lies in [k, k + 1) * ceil(total / gridDim.x) - a contiguous stretch,
+// usually inside one job - and rebuilds the lookup tables when the stretch crosses into the next job.  Everything
+// that steers this (loop bounds, job changes) depends on blockIdx and kernel parameters only, so the compiler
+// sees warp-uniform control flow and puts no divergence guards around the warp votes of the hot loop; in the last
+// round of a job a warp past the job's last tile goes through the same code with zero groups to do.
+// SINGLE: the launch has one job (the common single-tensor call); its parameters then sit at fixed offsets of
+// the parameter block and the job loop disappears.
+template <int DT, bool SINGLE>
 __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __grid_constant__ BatchParams P) {
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    int j = 0;
-    while (j + 1 < P.n_jobs && blockIdx.x >= P.job[j + 1].cta_begin) ++j;
-    const JobParams &J = P.job[j];
     const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
     const uint32_t ring = lut_addr + kLutBytes + warp * kRingStride;
-    build_tables_smem(J, lut_addr, warp, lane);
-    __syncthreads();
-    const uint32_t cta = blockIdx.x - J.cta_begin;
-    // Rounds over the job's tiles: warp w of CTA c takes the job's tile (c + i * cta_count) * 32 + w in round i.  Loop bounds and the
-    // test for a CTA past the end depend on blockIdx and kernel parameters only, so the compiler sees warp-uniform
-    // control flow and puts no divergence guards around the warp votes of the hot loop; inside the one CTA that
-    // straddles the end, a warp past the last tile goes through the same code with zero groups to do.
-    const bool wide = J.per_row >= 32u;
-    for (uint32_t i = 0; i < J.iters; ++i) {
-        const uint32_t base = (cta + i * J.cta_count) * kWarps;
-        if (base >= J.tile_cnt) break;
-        const bool mine = base + warp < J.tile_cnt;
-        const uint32_t tile = J.tile0 + min(base + warp, J.tile_cnt - 1u);
-        if constexpr (DT != EP_FIELDS_I32) {
-            if (wide && J.V < (1u << 20)) {
-                decode_tile_fast<DT>(J, tile, mine, lut_addr, ring, lane);
-                continue;
+    bool tables_in_use = false;
+    const int n_jobs = SINGLE ? 1 : P.n_jobs;
+    for (int j = 0; j < n_jobs; ++j) {
+        const JobParams &J = P.job[SINGLE ? 0 : j];
+        // rounds r of this job with cost_begin + r * round_cost in [lo, hi), this CTA's share of the total cost
+        // (recomputed per job rather than kept in registers across the decode loops)
+        const uint32_t lo = P.cost_per_cta * blockIdx.x, hi = lo + P.cost_per_cta;      // below 2^31 (see the launcher)
+        const uint32_t a = lo > J.cost_begin ? lo - J.cost_begin : 0u, b = hi > J.cost_begin ? hi - J.cost_begin : 0u;
+        const uint32_t r0 = min((a + J.round_cost - 1u) / J.round_cost, J.rounds);
+        const uint32_t r1 = min((b + J.round_cost - 1u) / J.round_cost, J.rounds);
+        if (r0 >= r1) continue;
+        if (tables_in_use) __syncthreads();          // every warp is done with the previous job's tables
+        build_tables_smem(J, lut_addr, warp, lane);
+        __syncthreads();
+        tables_in_use = true;
+        const bool wide = J.per_row >= 32u;
+        for (uint32_t r = r0; r < r1; ++r) {
+            const uint32_t base = r * kWarps;
+            const bool mine = base + warp < J.tile_cnt;
+            const uint32_t tile = J.tile0 + min(base + warp, J.tile_cnt - 1u);
+            if constexpr (DT != EP_FIELDS_I32) {
+                if (wide && J.V < (1u << 20)) {
+                    decode_tile_fast<DT>(J, tile, mine, lut_addr, ring, lane);
+                    continue;
+                }
             }
-        }
-        if (mine) {
-            if (wide) decode_tile<DT, true>(J, tile, lut_addr, ring, lane);
-            else decode_tile<DT, false>(J, tile, lut_addr, ring, lane);
+            if (mine) {
+                if (wide) decode_tile<DT, true>(J, tile, lut_addr, ring, lane);
+                else decode_tile<DT, false>(J, tile, lut_addr, ring, lane);
+            }
         }
     }
 }
@@ -1030,11 +1036,14 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
+        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    ep_decode_smem_kernel<DT><<<grid, kThreads, kSmemBytes, st>>>(P);
+    if (P.n_jobs == 1) ep_decode_smem_kernel<DT, true><<<grid, kThreads, kSmemBytes, st>>>(P);
+    else ep_decode_smem_kernel<DT, false><<<grid, kThreads, kSmemBytes, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -1128,7 +1137,6 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         return EP_ERR_BAD_ARG;
     const ep_decode_job *fast[EP_MAX_BATCH], *large[EP_MAX_BATCH];
     int n_jobs = 0, n_large = 0;
-    uint64_t tiles_total = 0;
     for (int i = 0; i < n_in; ++i) {
         const ep_decode_job &jb = jobs_in[i];
         if (!jb.info || !jb.d_stream || !jb.d_tile_index || !jb.d_out) return EP_ERR_BAD_ARG;
@@ -1148,7 +1156,7 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         if (jb.tile_count != 0 || jb.tile_begin != 0) {     // a tile range: inside the tensor and not empty
             if (jb.tile_count == 0 || jb.tile_begin >= I.n_tiles || jb.tile_count > I.n_tiles - jb.tile_begin) return EP_ERR_BAD_ARG;
         }
-        if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; tiles_total += job_tiles(jb); }
+        if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; }
         else large[n_large++] = &jb;
     }
     if (n_large) {
@@ -1159,19 +1167,14 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     BatchParams P;
     std::memset(&P, 0, sizeof(P));
     P.n_jobs = n_jobs;
-    // persistent CTAs: a single tensor gets one CTA per SM (or fewer if it has under 32 tiles per SM);
-    // a batch shares twice the SM count in proportion to the tensors' tile counts
-    const uint64_t budget = n_jobs == 1 ? uint64_t(sms) : 2ull * sms;
-    uint32_t next = 0;
+    // persistent CTAs, one per SM (fewer if the launch has fewer rounds than SMs); the kernel splits the
+    // cost-weighted list of all rounds evenly over them
+    uint64_t rounds_total = 0, cost = 0;
     for (int i = 0; i < n_jobs; ++i) {
         const ep_decode_job &jb = *fast[i];
         const ep_info &I = *jb.info;
         JobParams &J = P.job[i];
         const uint32_t my_tiles = job_tiles(jb);
-        const uint64_t want = (uint64_t(my_tiles) + kWarps - 1) / kWarps;
-        uint64_t share = (budget * my_tiles + tiles_total - 1) / tiles_total;
-        if (share < 1) share = 1;
-        if (share > want) share = want;
         J.stream = static_cast<const uint8_t *>(jb.d_stream);
         J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
         J.scales = jb.d_row_scales;
@@ -1187,10 +1190,11 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.tile_cnt = my_tiles;
         J.b = I.b;
         J.zlo = int32_t(even_base(coord_range(I)));
-        J.cta_begin = next;
-        J.cta_count = uint32_t(share);
-        const uint32_t round_tiles = J.cta_count * uint32_t(kWarps);
-        J.iters = (J.tile_cnt + round_tiles - 1u) / round_tiles;
+        J.rounds = (my_tiles + uint32_t(kWarps) - 1u) / uint32_t(kWarps);
+        J.round_cost = (I.V + 31u) / 32u;
+        J.cost_begin = uint32_t(cost);
+        cost += uint64_t(J.rounds) * J.round_cost;
+        rounds_total += J.rounds;
         uint32_t acc = 0;
         for (int t = 0; t < EP_NUM_TABLES; ++t) {
             J.tmin[t] = int16_t(I.table_min[t]);
@@ -1198,8 +1202,11 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
             J.foff[t] = uint16_t(acc);
             acc += I.table_K[t];
         }
-        next += uint32_t(share);
     }
+    const uint32_t next = uint32_t(rounds_total < uint64_t(sms) ? rounds_total : uint64_t(sms));   // grid size
+    // a tensor has under 2^27 blocks, so sixteen of them cost under 2^26 groups: 32-bit arithmetic in the kernel
+    if (cost + next >= (1ull << 31)) return EP_ERR_UNSUPPORTED;
+    P.cost_per_cta = uint32_t((cost + next - 1u) / next);
     cudaError_t e;
     switch (dt) {
     case EP_BF16: e = launch_smem<EP_BF16>(P, next, st); break;

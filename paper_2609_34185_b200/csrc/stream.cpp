@@ -137,4 +137,28 @@ extern "C" uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double targe
     }
 }
 
+extern "C" uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint32_t *C, uint32_t n, double target_bpp,
+                                                  uint32_t decode_ctas) {
+    const uint32_t vmax = ep_default_tile_vectors(target_bpp);
+    if (!R || !C || n == 0 || decode_ctas == 0) return vmax;
+    // One launch decodes all n tensors: a CTA takes 32 tiles per round, the rounds of all tensors are split evenly
+    // over the CTAs, so the launch lasts ceil(rounds / CTAs) rounds of ceil(V / 32) groups each (plus a small
+    // fixed cost per round: tile set-up and the last, partly idle steps).  Take the multiple of 32 that makes this
+    // shortest; on ties the larger tile (less metadata).  Never below a quarter of the paper's default.
+    const uint32_t lo = (vmax / 4u > 32u ? vmax / 4u : 32u);
+    uint32_t best_v = vmax;
+    uint64_t best_cost = ~0ull;
+    for (uint32_t V = (lo + 31u) & ~31u; V <= vmax; V += 32u) {
+        uint64_t rounds = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint64_t nvec = uint64_t(R[i]) * (C[i] / 8u);
+            const uint64_t tiles = (nvec + V - 1u) / V;
+            rounds += (tiles + 31u) / 32u;
+        }
+        const uint64_t cost = ((rounds + decode_ctas - 1u) / decode_ctas) * (V / 32u + 2u);
+        if (cost <= best_cost) { best_cost = cost; best_v = V; }
+    }
+    return best_v;
+}
+
 extern "C" int ep_version(void) { return 1; }

@@ -332,3 +332,31 @@ def test_tile_ranges_tile_the_tensor_and_write_nothing_else():
                 ep.decode_tiles(I, d.d_stream, d.d_tile_index, d.d_row_scales, dt, full.data_ptr(), bad[0], bad[1],
                                 d.scratch.data_ptr() if d.scratch is not None else 0,
                                 d.scratch.numel() if d.scratch is not None else 0)
+
+
+def test_batch_shares_cross_jobs_with_different_tile_sizes():
+    # the launch's rounds are split over the CTAs by cost (groups per round): tiny tensors make one CTA's share
+    # span several jobs (tables rebuilt in between), a big one spreads over many CTAs, tile sizes differ per job
+    rng = np.random.default_rng(12)
+    specs = [(8, 256, 32), (16, 512, 33), (8, 264, 5), (2048, 2048, 455), (32, 256, 100), (64, 1024, 1792),
+             (8, 8, 0), (512, 4096, 1820), (24, 512, 64), (1024, 1024, 96), (8, 512, 1), (40, 2048, 640),
+             (16, 256, 0), (256, 256, 128), (8, 1024, 31), (128, 8192, 3640)]
+    blobs, outs = [], []
+    for i, (R, C, V) in enumerate(specs):
+        W = synth.gaussian_rows(R, C, 500 + i) if i % 2 else synth.laplace_rows(R, C, 500 + i)
+        blobs.append(ep.encode(W, float(rng.choice([2.0, 3.0, 4.0, 5.0])), tile_vectors=V))
+        outs.append(torch.empty((R, C), dtype=torch.float16, device="cuda"))
+    ds = [ep.upload(b) for b in blobs]
+    ep.decode_many(ds, ep.FP16, outs)
+    torch.cuda.synchronize()
+    for b, o in zip(blobs, outs):
+        ref, _ = oracle.decode(b.data, oracle.FP16)
+        assert np.array_equal(_bits(o), ref), (b.info.R, b.info.C, b.info.V)
+    assert ep.last_device_status() == 0
+    # the same tensors in the opposite order (other shares, other job boundaries) and as fields
+    outs2 = [torch.empty((b.info.R * b.info.C // 8, 9), dtype=torch.int32, device="cuda") for b in blobs]
+    ep.decode_many(ds[::-1], ep.FIELDS_I32, outs2[::-1])
+    torch.cuda.synchronize()
+    for b, o in zip(blobs, outs2):
+        _, f = oracle.decode(b.data, oracle.BF16, want_fields=True)
+        assert np.array_equal(o.cpu().numpy(), f)
