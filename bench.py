@@ -54,6 +54,8 @@ def parse_args():
                          "(throughput and stored vs target bpp per rate, in the JSON key 'sweep')")
     ap.add_argument("--gemm-curve", action="store_true",
                     help="also time decode-then-GEMM against a GEMM on resident BF16 weights (10240x3840 layer, 4 bpp)")
+    ap.add_argument("--graph", action="store_true",
+                    help="record the step's launches once in a CUDA graph and replay it in the timed region")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -337,15 +339,16 @@ def main():
     launches_per_step = sum((len(r) + ep.binding.MAX_BATCH - 1) // ep.binding.MAX_BATCH for r in resident)
     stream = torch.cuda.current_stream()
 
-    def decode_layer(l):
+    def decode_layer(l, st=None):
+        st = stream if st is None else st
         if len(resident[l]) == 1:
-            ep.decode(resident[l][0], DT, out=outs_by_layer[l][0], stream=stream)
+            ep.decode(resident[l][0], DT, out=outs_by_layer[l][0], stream=st)
         else:
-            ep.decode_many(resident[l], DT, outs_by_layer[l], stream=stream)
+            ep.decode_many(resident[l], DT, outs_by_layer[l], stream=st)
 
-    def step():
+    def step(st=None):
         for l in range(n_layers):
-            decode_layer(l)
+            decode_layer(l, st)
 
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
 
@@ -366,13 +369,26 @@ def main():
     if ep.last_device_status() != 0:
         raise RuntimeError("decoder reported an inconsistent stream during warm-up")
     barrier()
+    run_step = step
+    if args.graph:
+        graph = torch.cuda.CUDAGraph()
+        cap = torch.cuda.Stream(device=dev)
+        cap.wait_stream(stream)
+        with torch.cuda.stream(cap):
+            with torch.cuda.graph(graph, stream=cap):
+                step(cap)
+        stream.wait_stream(cap)
+        run_step = graph.replay
+        for _ in range(2):
+            run_step()
+        barrier()
     mark = sampler.mark()
     evs = []
     for _ in range(args.steps):
         flush.fill_(0)      # L2 flush between timed iterations, outside the events
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record(stream)
-        step()
+        run_step()
         e.record(stream)
         evs.append((s, e))
     barrier()
@@ -552,6 +568,7 @@ def main():
             "config": {"workload": name, "target_bpp": bpp, "stored_bpp": stored, "tile_vectors": b0.info.V,
                        "tiles_first_tensor": b0.info.n_tiles, "b": b0.info.b, "out_dtype": dtype_name,
                        "params_per_step": params_per_step, "l2": "flushed between timed steps (512 MB write)",
+                       "launch": "cuda graph replay" if args.graph else "direct",
                        "min_ms": min(times_ms), "median_ms": statistics.median(times_ms),
                        "warm_ms_per_step_no_flush": warm_ms, "rel_l2_first_tensor": rel_l2_first},
             "effective_GBps": eff_gbs, "pct_of_measured_hbm": 100.0 * eff_gbs / peak, "pct_of_8TBps": 100.0 * eff_gbs / 8000.0,

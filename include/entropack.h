@@ -195,7 +195,9 @@ size_t ep_decode_scratch_bytes(const ep_info *info);
 
 /* Fused decode of one tensor (Sec. 3.7): rANS symbol decode (Eq. 18) -> inverse field transform
  * (Eq. 5) -> multiply by the fp32 row scale -> snap to out_dtype (Eq. 19) -> store.  Enqueues on
- * `stream` and returns; see ep_decode_job for the pointer arguments. */
+ * `stream` and returns; see ep_decode_job for the pointer arguments.  The first decode call per output
+ * type on a device also sets an attribute of the kernel (its shared-memory size); after that a call does
+ * nothing but enqueue its launches, so it can be recorded in a stream capture and replayed as a CUDA graph. */
 int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_tile_index,
                      const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
                      size_t scratch_bytes, void *stream);

@@ -360,3 +360,34 @@ def test_batch_shares_cross_jobs_with_different_tile_sizes():
     for b, o in zip(blobs, outs2):
         _, f = oracle.decode(b.data, oracle.BF16, want_fields=True)
         assert np.array_equal(o.cpu().numpy(), f)
+
+
+def test_decode_calls_can_be_captured_in_a_cuda_graph_and_replayed():
+    # a decode call only enqueues kernels on the given stream (after the first call per output type has set the
+    # kernel's shared-memory attribute), so a layer's launches can be recorded once and replayed
+    Ws = [synth.gaussian_rows(128, 1024, 61), synth.laplace_rows(64, 2048, 62), synth.gaussian_rows(96, 512, 63)]
+    blobs = [ep.encode(W, 4.0) for W in Ws] + [ep.encode(Ws[0], 4.0, b_start=12)]      # the last one needs scratch
+    ds = [ep.upload(b) for b in blobs]
+    outs = [torch.zeros((b.info.R, b.info.C), dtype=torch.bfloat16, device="cuda") for b in blobs]
+    ep.decode_many(ds, ep.BF16, outs)                  # warm-up outside the capture
+    torch.cuda.synchronize()
+    for o in outs:
+        o.zero_()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            ep.decode_many(ds[:3], ep.BF16, outs[:3], stream=side)
+            ep.decode(ds[3], ep.BF16, out=outs[3], stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for rep in range(2):
+        for o in outs:
+            o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for b, o in zip(blobs, outs):
+            ref, _ = oracle.decode(b.data, oracle.BF16)
+            assert np.array_equal(_bits(o), ref)
+    assert ep.last_device_status() == 0
