@@ -39,6 +39,7 @@ constexpr uint32_t kRingStride = kRingBytes + kRingMirror;
 constexpr uint32_t kSmemBytes = kLutBytes + kWarps * kRingStride;   // 225280
 constexpr uint32_t kCodeMask = 0x001FF800u;            // 10-bit code field
 constexpr uint32_t kExp4096 = 0x45800000u;             // fp32 bit pattern of 4096.0
+constexpr uint32_t kOwnSlots = 16;                     // table build: slots of a symbol that its own lane writes
 
 __device__ unsigned int g_ep_status = 0;
 
@@ -84,6 +85,8 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, uint64_t src, uint32_t 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // two fp32 lanes per instruction (sm_100 packed fp32), operands kept as 64-bit register pairs
 __device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi) {
@@ -139,8 +142,9 @@ __device__ __forceinline__ uint32_t cvt_s8(float v) {
 
 // ---- lookup-table construction (per CTA, from the stream's frequency tables) ---------------------
 // Warp t fills table t.  Symbols are taken 32 at a time: a warp scan gives each lane its symbol's
-// first slot, every lane writes the first four slots of its own symbol, and symbols with more than
-// four slots are then filled by the whole warp.
+// first slot, every lane writes the first sixteen slots of its own symbol, and the few symbols with more
+// slots than that are then filled by the whole warp, one after the other (that loop is serial: its length,
+// not the number of stores, is what the build time depends on).
 __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t lut_addr, uint32_t warp, uint32_t lane) {
   for (uint32_t t = warp; t < EP_NUM_TABLES; t += kWarps) {
     const uint32_t K = J.tK[t];
@@ -165,16 +169,16 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
         const uint32_t entry = (f << 21) | ((code & 0x3FFu) << 11);
         if (f >= kLutEntries) atomicOr(&g_ep_status, 1u);   // not a stream the launcher sends here: f does not fit its field
 #pragma unroll
-        for (uint32_t u = 0; u < 4; ++u)
+        for (uint32_t u = 0; u < kOwnSlots; ++u)
             if (u < f && first + u < kLutEntries) sts32(base + 4u * (first + u), entry | u);
-        uint32_t big = __ballot_sync(0xFFFFFFFFu, f > 4);
+        uint32_t big = __ballot_sync(0xFFFFFFFFu, f > kOwnSlots);
         while (big) {
             const int i = __ffs(big) - 1;
             big &= big - 1;
             const uint32_t fi = __shfl_sync(0xFFFFFFFFu, f, i);
             const uint32_t Fi = __shfl_sync(0xFFFFFFFFu, first, i);
             const uint32_t ei = __shfl_sync(0xFFFFFFFFu, entry, i);
-            for (uint32_t u = 4 + lane; u < fi && Fi + u < kLutEntries; u += 32) sts32(base + 4u * (Fi + u), ei | u);
+            for (uint32_t u = kOwnSlots + lane; u < fi && Fi + u < kLutEntries; u += 32) sts32(base + 4u * (Fi + u), ei | u);
         }
         run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
@@ -789,6 +793,14 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
         const uint32_t r0 = min((a + J.round_cost - 1u) / J.round_cost, J.rounds);
         const uint32_t r1 = min((b + J.round_cost - 1u) / J.round_cost, J.rounds);
         if (r0 >= r1) continue;
+        {   // while the tables are built, bring this warp's first tile record and the start of its payload into L2
+            const uint32_t t_first = J.tile0 + min(r0 * kWarps + warp, J.tile_cnt - 1u);
+            const uint32_t *rec = J.tile_index + size_t(t_first) * 33u;
+            if (lane < 2) prefetch_l2(rec + 32u * lane);                     // the record spans two 128-byte lines
+            const uint32_t off = min(rec[32], J.total_words);
+            const uint64_t at = 2ull * off + 128u * lane;                      // 4 KB: the ring's first fill and more
+            if (at < 2ull * J.total_words) prefetch_l2(J.stream + J.off_payload + at);
+        }
         if (tables_in_use) __syncthreads();          // every warp is done with the previous job's tables
         build_tables_smem(J, lut_addr, warp, lane);
         __syncthreads();
