@@ -32,7 +32,7 @@ FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEA
 
 # dram bytes (read + write) per launch measured with ncu for the default workload, filled in from
 # profiles/ after a capture; None = not captured for this workload
-NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 41798656 + 75799296}   # dram read + write of one launch
+NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 41855744 + 76059904}   # dram read + write of one launch
 
 
 def parse_args():
