@@ -285,6 +285,39 @@ def test_config3_one_wide_tensor_fp8_and_int8_containers():
         _full_compare(Wc, 2.5, dt)
 
 
+def test_config4_with_the_tile_size_the_bench_uses():
+    V = ep.suggest_tile_vectors(8192, 8192, 4.0, 32 * torch.cuda.get_device_properties(0).multi_processor_count)
+    blob = _full_compare(synth.config4(), 4.0, ep.FP16, V)
+    assert blob.info.V == V
+
+
+def test_config5_one_layer_batched_as_the_bench_times_it():
+    # the seven tensors of one layer at full size (372 M parameters), one tile size from ep_suggest_tile_vectors_batch,
+    # streams from the GPU encoder, one batched launch into one reused BF16 buffer: every weight against the oracle
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    V = ep.suggest_tile_vectors_batch(synth.BLOCK_SHAPES, 3.5, sms)
+    blobs = []
+    for i in range(7):
+        W = synth.config5_tensor(0, i)
+        blobs.append(ep.encode_device(torch.from_numpy(W).cuda(), 3.5, tile_vectors=V))
+        del W
+    total = sum(b.info.R * b.info.C for b in blobs)
+    assert abs(8.0 * sum(len(b) for b in blobs) / total - 3.5) < 0.035
+    buf = torch.empty(total, dtype=torch.bfloat16, device="cuda")
+    outs, at = [], 0
+    for b in blobs:
+        n = b.info.R * b.info.C
+        outs.append(buf[at:at + n].view(b.info.R, b.info.C))
+        at += n
+    ds = [ep.upload(b) for b in blobs]
+    ep.decode_many(ds, ep.BF16, outs)
+    torch.cuda.synchronize()
+    assert ep.last_device_status() == 0
+    for b, o in zip(blobs, outs):
+        ref, _ = oracle.decode(b.data, oracle.BF16)
+        assert np.array_equal(_bits(o), ref), (b.info.R, b.info.C)
+
+
 # ---- tile ranges: the shard of a tensor-parallel rank ------------------------------------------------
 
 def test_tile_ranges_tile_the_tensor_and_write_nothing_else():
