@@ -544,39 +544,35 @@ __device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, u
     "mov.b32 o0, {h0, h1};\n\t"                                 \
     "mov.b32 o1, {h2, h3};\n\t"                                 \
     "st.global.v2.b32 [ad], {o0, o1};\n\t"
+/* one-byte integers: round to nearest even into s32 (out-of-range values end at INT_MIN / INT_MAX, NaN at 0), then
+   saturate and pack four at a time: cvt.pack d, a, b, c gives (c << 16) | sat(a) << 8 | sat(b) */
 #define EP_S_STORE_UINT8                                        \
-    "cvt.rni.sat.u8.f32 o0, w0;\n\t"                            \
-    "cvt.rni.sat.u8.f32 o2, w1;\n\t"                            \
-    "bfi.b32 o0, o2, o0, 8, 8;\n\t"                             \
-    "cvt.rni.sat.u8.f32 o2, w2;\n\t"                            \
-    "bfi.b32 o0, o2, o0, 16, 8;\n\t"                            \
-    "cvt.rni.sat.u8.f32 o2, w3;\n\t"                            \
-    "bfi.b32 o0, o2, o0, 24, 8;\n\t"                            \
-    "cvt.rni.sat.u8.f32 o1, w4;\n\t"                            \
-    "cvt.rni.sat.u8.f32 o2, w5;\n\t"                            \
-    "bfi.b32 o1, o2, o1, 8, 8;\n\t"                             \
-    "cvt.rni.sat.u8.f32 o2, w6;\n\t"                            \
-    "bfi.b32 o1, o2, o1, 16, 8;\n\t"                            \
-    "cvt.rni.sat.u8.f32 o2, w7;\n\t"                            \
-    "bfi.b32 o1, o2, o1, 24, 8;\n\t"                            \
+    "cvt.rni.s32.f32 x1, w0;\n\t"                               \
+    "cvt.rni.s32.f32 x2, w1;\n\t"                               \
+    "cvt.rni.s32.f32 x3, w2;\n\t"                               \
+    "cvt.rni.s32.f32 x4, w3;\n\t"                               \
+    "cvt.rni.s32.f32 x5, w4;\n\t"                               \
+    "cvt.rni.s32.f32 x6, w5;\n\t"                               \
+    "cvt.rni.s32.f32 x7, w6;\n\t"                               \
+    "cvt.rni.s32.f32 x8, w7;\n\t"                               \
+    "cvt.pack.sat.u8.s32.b32 o2, x4, x3, 0;\n\t"                \
+    "cvt.pack.sat.u8.s32.b32 o0, x2, x1, o2;\n\t"               \
+    "cvt.pack.sat.u8.s32.b32 o3, x8, x7, 0;\n\t"                \
+    "cvt.pack.sat.u8.s32.b32 o1, x6, x5, o3;\n\t"               \
     "st.global.v2.b32 [ad], {o0, o1};\n\t"
 #define EP_S_STORE_INT8                                         \
-    "cvt.rni.sat.s8.f32 o0, w0;\n\t"                            \
-    "cvt.rni.sat.s8.f32 o2, w1;\n\t"                            \
-    "and.b32 o0, o0, 0xFF;\n\t"                                 \
-    "bfi.b32 o0, o2, o0, 8, 8;\n\t"                             \
-    "cvt.rni.sat.s8.f32 o2, w2;\n\t"                            \
-    "bfi.b32 o0, o2, o0, 16, 8;\n\t"                            \
-    "cvt.rni.sat.s8.f32 o2, w3;\n\t"                            \
-    "bfi.b32 o0, o2, o0, 24, 8;\n\t"                            \
-    "cvt.rni.sat.s8.f32 o1, w4;\n\t"                            \
-    "cvt.rni.sat.s8.f32 o2, w5;\n\t"                            \
-    "and.b32 o1, o1, 0xFF;\n\t"                                 \
-    "bfi.b32 o1, o2, o1, 8, 8;\n\t"                             \
-    "cvt.rni.sat.s8.f32 o2, w6;\n\t"                            \
-    "bfi.b32 o1, o2, o1, 16, 8;\n\t"                            \
-    "cvt.rni.sat.s8.f32 o2, w7;\n\t"                            \
-    "bfi.b32 o1, o2, o1, 24, 8;\n\t"                            \
+    "cvt.rni.s32.f32 x1, w0;\n\t"                               \
+    "cvt.rni.s32.f32 x2, w1;\n\t"                               \
+    "cvt.rni.s32.f32 x3, w2;\n\t"                               \
+    "cvt.rni.s32.f32 x4, w3;\n\t"                               \
+    "cvt.rni.s32.f32 x5, w4;\n\t"                               \
+    "cvt.rni.s32.f32 x6, w5;\n\t"                               \
+    "cvt.rni.s32.f32 x7, w6;\n\t"                               \
+    "cvt.rni.s32.f32 x8, w7;\n\t"                               \
+    "cvt.pack.sat.s8.s32.b32 o2, x4, x3, 0;\n\t"                \
+    "cvt.pack.sat.s8.s32.b32 o0, x2, x1, o2;\n\t"               \
+    "cvt.pack.sat.s8.s32.b32 o3, x8, x7, 0;\n\t"                \
+    "cvt.pack.sat.s8.s32.b32 o1, x6, x5, o3;\n\t"               \
     "st.global.v2.b32 [ad], {o0, o1};\n\t"
 
 #define EP_FULL_GROUPS_ASM(STORE, GROUP_BYTES)                                                                        \
