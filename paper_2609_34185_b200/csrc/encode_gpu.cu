@@ -36,11 +36,29 @@ constexpr uint32_t kMaxTableSymbols = 40960;   // sum of K over the 17 tables th
 __global__ void row_rms_kernel(const float *__restrict__ W, uint32_t R, uint32_t C, float *__restrict__ mu) {
     const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= R) return;
-    const float *x = W + size_t(r) * C;
+    // the sum is one serial chain (the host's order); the loads are not: eight 16-byte loads are in flight per pass
+    const float4 *x = reinterpret_cast<const float4 *>(W + size_t(r) * C);     // rows start 16-byte aligned: C % 8 == 0
+    const uint32_t n4 = C / 4;
     double acc = 0.0;
-    for (uint32_t j = 0; j < C; ++j) {
-        const double v = double(x[j]);
-        acc = __dadd_rn(acc, __dmul_rn(v, v));
+    uint32_t j = 0;
+    for (; j + 8 <= n4; j += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __ldg(x + j + k);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            acc = __dadd_rn(acc, __dmul_rn(double(v[k].x), double(v[k].x)));
+            acc = __dadd_rn(acc, __dmul_rn(double(v[k].y), double(v[k].y)));
+            acc = __dadd_rn(acc, __dmul_rn(double(v[k].z), double(v[k].z)));
+            acc = __dadd_rn(acc, __dmul_rn(double(v[k].w), double(v[k].w)));
+        }
+    }
+    for (; j < n4; ++j) {
+        const float4 v = __ldg(x + j);
+        acc = __dadd_rn(acc, __dmul_rn(double(v.x), double(v.x)));
+        acc = __dadd_rn(acc, __dmul_rn(double(v.y), double(v.y)));
+        acc = __dadd_rn(acc, __dmul_rn(double(v.z), double(v.z)));
+        acc = __dadd_rn(acc, __dmul_rn(double(v.w), double(v.w)));
     }
     double m = __dsqrt_rn(__ddiv_rn(acc, double(C)));
     if (!(m > 1e-12)) m = 1e-12;
@@ -159,21 +177,40 @@ __global__ void refit_kernel(const float *__restrict__ W, uint32_t R, uint32_t C
     const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= R) return;
     const uint32_t per_row = C / 8;
-    const float *x = W + size_t(r) * C;
+    const float4 *x4 = reinterpret_cast<const float4 *>(W + size_t(r) * C);    // rows start 16-byte aligned: C % 8 == 0
     const int16_t *q = fields + size_t(r) * per_row * 9;
     double xp = 0.0, pp = 0.0;
-    for (uint32_t v = 0; v < per_row; ++v, q += 9) {
-        const double half = 0.5 * double(q[0]);
-        int32_t s7 = 0;
-        for (int j = 0; j < 7; ++j) {
-            const double p = __dadd_rn(double(q[1 + j]), half);
-            xp = __dadd_rn(xp, __dmul_rn(double(x[8 * v + j]), p));
-            pp = __dadd_rn(pp, __dmul_rn(p, p));
-            s7 += q[1 + j];
+    // two serial chains in the host's order; the loads of four blocks are issued together
+    constexpr int kAhead = 4;
+    for (uint32_t v0 = 0; v0 < per_row; v0 += kAhead) {
+        float xv[kAhead][8];
+        int32_t qv[kAhead][9];
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k) {
+            if (v0 + k < per_row) {
+                const float4 a = __ldg(x4 + 2 * (v0 + k)), b = __ldg(x4 + 2 * (v0 + k) + 1);
+                xv[k][0] = a.x; xv[k][1] = a.y; xv[k][2] = a.z; xv[k][3] = a.w;
+                xv[k][4] = b.x; xv[k][5] = b.y; xv[k][6] = b.z; xv[k][7] = b.w;
+#pragma unroll
+                for (int j = 0; j < 9; ++j) qv[k][j] = q[9 * (v0 + k) + j];
+            }
         }
-        const double p8 = __dadd_rn(double(2 * int32_t(q[8]) + (s7 & 1)), half);   // Eq. 5
-        xp = __dadd_rn(xp, __dmul_rn(double(x[8 * v + 7]), p8));
-        pp = __dadd_rn(pp, __dmul_rn(p8, p8));
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k) {
+            if (v0 + k >= per_row) break;
+            const double half = 0.5 * double(qv[k][0]);
+            int32_t s7 = 0;
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                const double p = __dadd_rn(double(qv[k][1 + j]), half);
+                xp = __dadd_rn(xp, __dmul_rn(double(xv[k][j]), p));
+                pp = __dadd_rn(pp, __dmul_rn(p, p));
+                s7 += qv[k][1 + j];
+            }
+            const double p8 = __dadd_rn(double(2 * qv[k][8] + (s7 & 1)), half);   // Eq. 5
+            xp = __dadd_rn(xp, __dmul_rn(double(xv[k][7]), p8));
+            pp = __dadd_rn(pp, __dmul_rn(p8, p8));
+        }
     }
     double sg;
     if (pp > 0.0) {
