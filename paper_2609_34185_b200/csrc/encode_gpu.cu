@@ -332,47 +332,58 @@ Workspace carve(uint8_t *base, uint32_t R, uint32_t C, uint32_t V) {
         if ((call) != cudaSuccess) return EP_ERR_CUDA; \
     } while (0)
 
-// Page-locked host memory for finished blobs.  Locking tens of MB costs milliseconds, so the buffer of the
-// most recently freed blob is kept (one at most) and handed to the next encode that fits into it.
-std::mutex g_pinned_lock;
-uint8_t *g_pinned_spare = nullptr;
-size_t g_pinned_spare_cap = 0;
+// Page-locked host memory: for finished blobs and for the histograms that come back after every counting pass.
+// Locking memory costs milliseconds, so each of the two uses keeps the buffer it last gave back (one at most, the
+// larger one when two compete) for the next request that fits into it.
+struct PinnedSlot {
+    std::mutex lock;
+    uint8_t *spare = nullptr;
+    size_t spare_cap = 0;
 
-uint8_t *pinned_acquire(size_t n, size_t *cap) {
-    {
-        std::lock_guard<std::mutex> hold(g_pinned_lock);
-        if (g_pinned_spare && g_pinned_spare_cap >= n) {
-            uint8_t *p = g_pinned_spare;
-            *cap = g_pinned_spare_cap;
-            g_pinned_spare = nullptr;
-            g_pinned_spare_cap = 0;
-            return p;
+    uint8_t *acquire(size_t n, size_t headroom, size_t *cap) {
+        {
+            std::lock_guard<std::mutex> hold(lock);
+            if (spare && spare_cap >= n) {
+                uint8_t *p = spare;
+                *cap = spare_cap;
+                spare = nullptr;
+                spare_cap = 0;
+                return p;
+            }
         }
+        const size_t want = n + headroom;
+        void *p = nullptr;
+        if (cudaHostAlloc(&p, want, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        *cap = want;
+        return static_cast<uint8_t *>(p);
     }
-    const size_t want = n + n / 8 + 4096;           // headroom: the next tensor of a model is rarely the same size
-    void *p = nullptr;
-    if (cudaHostAlloc(&p, want, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-    *cap = want;
-    return static_cast<uint8_t *>(p);
-}
+    void release(uint8_t *p, size_t cap) {
+        uint8_t *drop = p;
+        {
+            std::lock_guard<std::mutex> hold(lock);
+            if (cap > spare_cap) {               // keep the larger of the two
+                drop = spare;
+                spare = p;
+                spare_cap = cap;
+            }
+        }
+        if (drop) cudaFreeHost(drop);
+    }
+};
+PinnedSlot g_blob_slot, g_hist_slot;
 
-void pinned_release(uint8_t *p, size_t cap) {
-    uint8_t *drop = p;
-    {
-        std::lock_guard<std::mutex> hold(g_pinned_lock);
-        if (cap > g_pinned_spare_cap) {               // keep the larger of the two
-            drop = g_pinned_spare;
-            g_pinned_spare = p;
-            g_pinned_spare_cap = cap;
-        }
-    }
-    if (drop) cudaFreeHost(drop);
-}
+// headroom for blobs: the next tensor of a model is rarely the same size
+uint8_t *pinned_acquire(size_t n, size_t *cap) { return g_blob_slot.acquire(n, n / 8 + 4096, cap); }
+void pinned_release(uint8_t *p, size_t cap) { g_blob_slot.release(p, cap); }
 
 class DeviceBackend final : public EncodeBackend {
 public:
     DeviceBackend(const float *dW, uint32_t R, uint32_t C, uint32_t V, uint8_t *ws, cudaStream_t st)
-        : W_(dW), R_(R), C_(C), V_(V), w_(carve(ws, R, C, V)), st_(st), hist_(size_t(EP_NUM_TABLES) * kHistBins) {}
+        : W_(dW), R_(R), C_(C), V_(V), w_(carve(ws, R, C, V)), st_(st) {
+        hist_ = reinterpret_cast<uint32_t *>(g_hist_slot.acquire(kHistBytes, 0, &hist_cap_));
+        if (!hist_) throw std::bad_alloc();
+    }
+    ~DeviceBackend() override { if (hist_) g_hist_slot.release(reinterpret_cast<uint8_t *>(hist_), hist_cap_); }
 
     int prepare(const std::vector<uint32_t> &sample) override {
         n_sample_ = uint32_t(sample.size());
@@ -444,11 +455,11 @@ private:
         quantise_count_kernel<<<grid, 256, 0, st_>>>(W_, C_, w_.mu, rows, n, s, fields, w_.hist, w_.overflow);
         EP_CUDA(cudaGetLastError());
         int overflow = 0;
-        EP_CUDA(cudaMemcpyAsync(hist_.data(), w_.hist, 4ull * hist_.size(), cudaMemcpyDeviceToHost, st_));
+        EP_CUDA(cudaMemcpyAsync(hist_, w_.hist, kHistBytes, cudaMemcpyDeviceToHost, st_));
         EP_CUDA(cudaMemcpyAsync(&overflow, w_.overflow, 4, cudaMemcpyDeviceToHost, st_));
         EP_CUDA(cudaStreamSynchronize(st_));
         if (overflow) return EP_ERR_UNSUPPORTED;     // a coordinate beyond +-4095: use the host encoder
-        m.from_histograms(hist_.data(), kHistBins, kHistOrigin);
+        m.from_histograms(hist_, kHistBins, kHistOrigin);
         return EP_OK;
     }
 
@@ -456,7 +467,9 @@ private:
     uint32_t R_, C_, V_;
     Workspace w_;
     cudaStream_t st_;
-    std::vector<uint32_t> hist_;
+    static constexpr size_t kHistBytes = 4ull * EP_NUM_TABLES * kHistBins;
+    uint32_t *hist_ = nullptr;       // page-locked: the copy back after each counting pass is a plain DMA
+    size_t hist_cap_ = 0;
     uint32_t n_sample_ = 0;
 };
 
