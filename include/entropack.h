@@ -168,7 +168,8 @@ int ep_pack_fields(const int32_t *fields, uint32_t R, uint32_t C, int32_t b, uin
  * The blob of this call lives in page-locked host memory (the device copies the payload straight into it,
  * and a later upload of the blob runs at full bus speed).  Page-locking costs milliseconds, so ep_blob_free
  * keeps the buffer of the most recently freed such blob (one per process at most, the larger one when two
- * compete) for the next call whose blob fits; a model converted tensor by tensor allocates once or twice. */
+ * compete) for the next call whose blob fits; a model converted tensor by tensor allocates once or twice.
+ * A second page-locked buffer of 0.5 MB (the histograms of the counting passes) is kept the same way. */
 size_t ep_encode_device_workspace_bytes(uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts);
 int ep_encode_device(const float *d_W, uint32_t R, uint32_t C, double target_bpp, const ep_encode_opts *opts,
                      void *d_workspace, size_t workspace_bytes, void *stream, ep_blob **out);
