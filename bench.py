@@ -5,7 +5,7 @@ One "step" is one pass of the whole hot path (rANS decode -> E8 point -> row res
 store) over one workload.  Default workload: the 48-layer stack of transformer-block bundles at 3.5 bpp decoded layer by
 layer into one reused BF16 buffer (config 5 of the baseline, the largest single-GPU configuration and one of the
 two the roofline target is stated on); the other one, the 8192x8192 Laplace tensor at 4.0 bpp to FP16, is
---workload c4.  Other workloads: --workload c2 | c3.
+--workload c4.  Other workloads: --workload c1 | c2 | c3.
 
   python bench.py [--gpus N --steps K --warmup W] [--workload c4 --bpp 4.0 --tile-vectors V]
   python bench.py --impl reference       # the CPU oracle on the same workload (bounded sample per step)
@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--bpp", type=float, default=None, help="target bits/param (default: the workload's)")
     ap.add_argument("--tile-vectors", type=int, default=-1,
                     help="V; 0 = the paper's default for the target rate; -1 (default) = ep_suggest_tile_vectors[_batch]: "
@@ -72,6 +72,10 @@ def make_workload(args):
     w = args.workload
     if w == "c4":
         return "config4: 8192x8192 Laplace rows", args.dtype or "fp16", args.bpp or 4.0, [[synth.config4()]]
+    if w == "c1":
+        if args.tile_vectors < 0:
+            args.tile_vectors = 4096            # the configuration fixes one tile per 64 rows
+        return "config1: 512x512 Gaussian rows, one tile per 64 rows", args.dtype or "bf16", args.bpp or 4.0, [[synth.config1()]]
     if w == "c2":
         return "config2: 4096x4096 Student-t rows", args.dtype or "bf16", args.bpp or 3.0, [[synth.config2()]]
     if w == "c3":
