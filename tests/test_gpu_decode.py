@@ -424,3 +424,38 @@ def test_decode_calls_can_be_captured_in_a_cuda_graph_and_replayed():
             ref, _ = oracle.decode(b.data, oracle.BF16)
             assert np.array_equal(_bits(o), ref)
     assert ep.last_device_status() == 0
+
+
+def test_largest_supported_tensor_byte_offsets_beyond_two_to_the_31():
+    # 30000 x 32768 = 983 M weights: the FP32 output is 3.93 GB, so the kernels' 32-bit byte offsets run close to
+    # their end; one more row would be refused.  Input drawn on the device (seeded), stream from the GPU encoder.
+    R, C = 30000, 32768
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    Wd = torch.randn(R, C, generator=g, device="cuda", dtype=torch.float32) * 0.02
+    blob = ep.encode_device(Wd, 3.0)
+    del Wd
+    assert abs(blob.stored_bpp - 3.0) < 0.03
+    d = ep.upload(blob)
+    for dt, odt in ((ep.FP32, oracle.FP32), (ep.INT8, oracle.INT8)):
+        out = ep.decode(d, dt)
+        torch.cuda.synchronize()
+        ref, _ = oracle.decode(blob.data, odt)
+        got = out.view(torch.uint8).cpu().numpy().reshape(-1)
+        assert np.array_equal(got, np.ascontiguousarray(ref).reshape(-1).view(np.uint8))
+        del out, got, ref
+    assert ep.last_device_status() == 0
+    tiles = range(blob.info.n_tiles - 1000, blob.info.n_tiles)          # a shard at the far end of the offsets
+    sh = ep.decode_tile_range(d, tiles, ep.FP32)
+    torch.cuda.synchronize()
+    part, _ = oracle.decode(blob.data, oracle.FP32, tiles=(tiles.start, tiles.stop))
+    first = tiles.start * blob.info.V * 8
+    assert np.array_equal(sh.view(torch.int32).cpu().numpy(), part.reshape(-1)[first:].view(np.int32))
+    # a tensor whose offsets would not fit is refused, not decoded wrongly
+    import copy
+    big = copy.copy(blob.info)
+    big.R = 32768
+    out = torch.empty(16, dtype=torch.float32, device="cuda")
+    with pytest.raises(ep.EntroPackError) as ei:
+        ep.decode_tensor(big, d.d_stream, d.d_tile_index, d.d_row_scales, ep.FP32, out.data_ptr())
+    assert ei.value.status == -3
