@@ -259,7 +259,7 @@ uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile
  * rounded up to a multiple of 32 vectors when that stays within the default.
  * Larger tiles amortise the 132 bytes of per-tile metadata, but a tensor with fewer tiles than slots
  * leaves SMs idle (App. "Tile layout and storage": tile size trades storage against parallelism).
- * Never below a quarter of the default (small tensors); returns the default when decode_slots is 0. */
+ * Never below a quarter of the default rounded down to a multiple of 32 (small tensors); returns the default when decode_slots is 0. */
 uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint32_t decode_slots);
 
 /* The same question for tensors that are decoded together by one ep_decode_batch launch (the blocks of a

@@ -123,8 +123,9 @@ extern "C" uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double targe
     const uint32_t vmax = ep_default_tile_vectors(target_bpp);
     const uint64_t nvec = uint64_t(R) * (C / 8);
     if (decode_slots == 0 || nvec == 0) return vmax;
-    // a small tensor cannot fill the decoder anyway: never let metadata grow beyond 4x the default's share
-    const uint64_t floor_v = vmax / 4 > 32 ? vmax / 4 : 32;
+    // a small tensor cannot fill the decoder anyway: never let metadata grow beyond about 4x the default's share
+    // (a quarter of the default, rounded down to whole groups of 32 vectors)
+    const uint64_t floor_v = (vmax / 4) / 32 * 32 > 32 ? (vmax / 4) / 32 * 32 : 32;
     // fewest rounds whose tiles are not larger than the default; tile sizes are multiples of 32 vectors (whole
     // groups of 32 rANS states, no partly filled last group) whenever that still fits
     for (uint64_t rounds = 1;; ++rounds) {
@@ -145,10 +146,10 @@ extern "C" uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint3
     // over the CTAs, so the launch lasts ceil(rounds / CTAs) rounds of ceil(V / 32) groups each (plus a small
     // fixed cost per round: tile set-up and the last, partly idle steps).  Take the multiple of 32 that makes this
     // shortest; on ties the larger tile (less metadata).  Never below a quarter of the paper's default.
-    const uint32_t lo = (vmax / 4u > 32u ? vmax / 4u : 32u);
+    const uint32_t lo = (vmax / 4u) / 32u * 32u > 32u ? (vmax / 4u) / 32u * 32u : 32u;   // as in ep_suggest_tile_vectors
     uint32_t best_v = vmax;
     uint64_t best_cost = ~0ull;
-    for (uint32_t V = (lo + 31u) & ~31u; V <= vmax; V += 32u) {
+    for (uint32_t V = lo; V <= vmax; V += 32u) {
         uint64_t rounds = 0;
         for (uint32_t i = 0; i < n; ++i) {
             const uint64_t nvec = uint64_t(R[i]) * (C[i] / 8u);

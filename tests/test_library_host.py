@@ -136,7 +136,7 @@ def test_suggested_tile_size_fills_whole_rounds_of_slots():
         tiles = -(-(R * C // 8) // V)
         rounds = -(-tiles // slots)
         assert tiles > 0.93 * rounds * slots                      # the last round is nearly full
-    assert ep.suggest_tile_vectors(512, 512, 4.0, slots) == ep.default_tile_vectors(4.0) // 4    # small tensor: floor
+    assert ep.suggest_tile_vectors(512, 512, 4.0, slots) == ep.default_tile_vectors(4.0) // 4 // 32 * 32    # small tensor: floor
     assert ep.suggest_tile_vectors(4096, 4096, 3.0, 0) == ep.default_tile_vectors(3.0)
 
 
@@ -151,8 +151,8 @@ def test_suggested_tile_size_for_a_batch_minimises_the_number_of_group_steps():
                         ([(4096, 4096), (4096, 11008), (11008, 4096)], 4.0), ([(256, 256), (128, 1024)], 6.0)):
         V = ep.suggest_tile_vectors_batch(shapes, bpp, ctas)
         vmax = ep.default_tile_vectors(bpp)
-        assert V % 32 == 0 and max(32, vmax // 4) <= V <= vmax
-        lo = -(-max(32, vmax // 4) // 32) * 32
+        lo = max(32, vmax // 4 // 32 * 32)
+        assert V % 32 == 0 and lo <= V <= vmax
         best = min(steps(shapes, v) for v in range(lo, vmax + 1, 32))
         assert steps(shapes, V) == best
         assert all(steps(shapes, v) > best for v in range(V + 32, vmax + 1, 32))      # the largest of the best
