@@ -108,7 +108,7 @@ def pick_tile_vectors(V, shape, bpp, slots, batch_shapes=None):
     if V >= 0:
         return V
     if batch_shapes is not None and len(batch_shapes) > 1:
-        return ep.suggest_tile_vectors_batch(batch_shapes, bpp, slots // 32)
+        return ep.suggest_tile_vectors_batch(batch_shapes, bpp, slots // ep.decode_tiles_per_sm())
     return ep.suggest_tile_vectors(shape[0], shape[1], bpp, slots)
 
 
@@ -234,7 +234,7 @@ def run_reference(args):
     name, dtype_name, bpp, layers = make_workload(args)
     V = args.tile_vectors
     import paper_2609_34185_b200 as ep
-    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 32,
+    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 48,
                                                                        [W.shape for W in layers[0]]))
     I = blob.info
     # each step decodes a leading tile range (repeated if short) sized so that the whole run stays near a minute
@@ -336,8 +336,8 @@ def main():
 
     # every rank decodes its own replica of the workload: tiles and tensors are independent, no collective
     n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    # one 32-warp CTA per SM: 32 tile slots each
-    slots = 32 * n_sms
+    # one persistent CTA per SM, ep_decode_tiles_per_sm() tiles in flight each
+    slots = ep.decode_tiles_per_sm() * n_sms
     blobs = encode_layers(layers, bpp, args.tile_vectors, slots, dev)
     n_layers = args.layers if args.workload == "c5" else len(blobs)
     resident = [[ep.upload(b, device=dev) for b in blobs[l % len(blobs)]] for l in range(n_layers)]

@@ -54,7 +54,6 @@ typedef enum {
     EP_ERR_BAD_STREAM = -2,  /* blob fails structural validation, or the decoder found an inconsistency */
     EP_ERR_UNSUPPORTED = -3, /* valid request this build cannot serve (e.g. offsets beyond 32 bits) */
     EP_ERR_CUDA = -4,        /* a CUDA runtime call failed */
-    EP_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out */
     EP_ERR_NOMEM = -6,       /* host allocation failed */
     EP_ERR_SCRATCH = -7,     /* scratch buffer missing, misaligned or too small */
     EP_ERR_STATIC_LIMIT = -8 /* ep_decode_tensor_static: the stream's tables exceed the built-in area */
@@ -138,6 +137,10 @@ typedef struct {
     size_t scratch_bytes;
     uint32_t tile_begin;        /* a range of tiles to decode, for a caller that owns a shard of the tensor */
     uint32_t tile_count;        /* (both 0 = the whole tensor); see ep_decode_tiles */
+    const void *d_tables;       /* device: lookup tables of this stream as ep_prepare_tables() left them
+                                   (ep_decode_tables_bytes(info) bytes, 256-byte aligned), or NULL: the decode
+                                   then derives them from the stream's frequency tables on every call.  With
+                                   prepared tables d_scratch is not needed */
 } ep_decode_job;
 
 /* ---- host encoder ------------------------------------------------------------------------- */
@@ -193,6 +196,23 @@ int ep_validate(const void *blob, size_t n);
  * memory (b <= 11 and coordinate range <= 1024, no single-symbol table at b = 11), else room
  * for 17 tables of 2^b four-byte entries. */
 size_t ep_decode_scratch_bytes(const ep_info *info);
+
+/* The decoder's lookup tables (App. "Tiled RANS implementation": the low b bits of a state select symbol and
+ * interval) depend on the stream's frequency tables only, and a weight is decoded on every forward call
+ * (Sec. "Reconstruction cost and tile overhead").  A caller that keeps a stream resident can therefore have
+ * them derived once: ep_decode_tables_bytes() is the size of the table image for this stream (128 KB when
+ * the tables fit shared memory, else 17 tables of 2^b four-byte entries), ep_prepare_tables() enqueues one
+ * small launch on `stream` that fills d_tables (device, 256-byte aligned) from the device copy of the blob,
+ * and every later decode of that stream that passes d_tables in its ep_decode_job copies (or reads) the image
+ * instead of rebuilding it.  The image is opaque and valid for this library version, this stream and any
+ * tile range of it.  Errors: EP_ERR_SCRATCH for a missing, misaligned or short buffer. */
+size_t ep_decode_tables_bytes(const ep_info *info);
+int ep_prepare_tables(const ep_info *info, const void *d_stream, void *d_tables, size_t tables_bytes, void *stream);
+
+/* Tiles the decode kernel works on at a time per SM (48: 24 warps, two tiles each); times the SM count this
+ * is the `decode_slots` argument of ep_suggest_tile_vectors (App. "Tile layout and storage": tile size trades
+ * storage against parallelism). */
+uint32_t ep_decode_tiles_per_sm(void);
 
 /* Fused decode of one tensor (Sec. 3.7): rANS symbol decode (Eq. 18) -> inverse field transform
  * (Eq. 5) -> multiply by the fp32 row scale -> snap to out_dtype (Eq. 19) -> store.  Enqueues on
@@ -253,7 +273,7 @@ int ep_last_device_status(void *stream);
 const char *ep_strerror(int status);
 uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile-size defaults */
 
-/* Tile size for a decoder with `decode_slots` concurrent tile slots (32 per SM for this library: 4736 on
+/* Tile size for a decoder with `decode_slots` concurrent tile slots (ep_decode_tiles_per_sm() = 48 per SM for this library: 7104 on
  * a 148-SM B200): the largest V not above the paper's default for the target rate for which the tensor's
  * R*C/8 blocks split into a whole number of rounds of decode_slots tiles (the last round nearly full),
  * rounded up to a multiple of 32 vectors when that stays within the default.
@@ -264,7 +284,7 @@ uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint
 
 /* The same question for tensors that are decoded together by one ep_decode_batch launch (the blocks of a
  * transformer layer): one tile size for all of them, a multiple of 32 not above the paper's default, chosen
- * so that the rounds of all tensors (32 tiles per CTA and round) split over `decode_ctas` CTAs (the SM count:
+ * so that the rounds of all tensors (48 tiles per CTA and round) split over `decode_ctas` CTAs (the SM count:
  * 148 on a B200) with the shortest last round.  R[i] x C[i] are the n tensor shapes. */
 uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint32_t *C, uint32_t n, double target_bpp,
                                        uint32_t decode_ctas);

@@ -62,7 +62,7 @@ class DecodeJob(C.Structure):
     _fields_ = [("info", C.POINTER(Info)), ("d_stream", C.c_void_p), ("d_tile_index", C.c_void_p),
                 ("d_row_scales", C.c_void_p), ("out_dtype", C.c_int32), ("d_out", C.c_void_p),
                 ("d_scratch", C.c_void_p), ("scratch_bytes", C.c_size_t),
-                ("tile_begin", C.c_uint32), ("tile_count", C.c_uint32)]
+                ("tile_begin", C.c_uint32), ("tile_count", C.c_uint32), ("d_tables", C.c_void_p)]
 
 
 _lib = None
@@ -95,6 +95,11 @@ def load():
     L.ep_validate.argtypes = [C.c_void_p, C.c_size_t]
     L.ep_decode_scratch_bytes.restype = C.c_size_t
     L.ep_decode_scratch_bytes.argtypes = [C.POINTER(Info)]
+    L.ep_decode_tables_bytes.restype = C.c_size_t
+    L.ep_decode_tables_bytes.argtypes = [C.POINTER(Info)]
+    L.ep_prepare_tables.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ep_decode_tiles_per_sm.restype = C.c_uint32
+    L.ep_decode_tiles_per_sm.argtypes = []
     L.ep_decode_tensor.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
     L.ep_decode_tiles.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
@@ -133,7 +138,12 @@ def default_tile_vectors(target_bpp: float) -> int:
     return load().ep_default_tile_vectors(float(target_bpp))
 
 
-def suggest_tile_vectors(R: int, Cc: int, target_bpp: float, decode_slots: int = 148 * 32) -> int:
+def decode_tiles_per_sm() -> int:
+    """ep_decode_tiles_per_sm: tiles the decode kernel works on at a time per SM."""
+    return int(load().ep_decode_tiles_per_sm())
+
+
+def suggest_tile_vectors(R: int, Cc: int, target_bpp: float, decode_slots: int = 148 * 48) -> int:
     """ep_suggest_tile_vectors: tile size that fills whole rounds of `decode_slots` concurrent tiles."""
     return load().ep_suggest_tile_vectors(R, Cc, float(target_bpp), decode_slots)
 
@@ -237,6 +247,15 @@ def decode_scratch_bytes(info: Info) -> int:
     return load().ep_decode_scratch_bytes(C.byref(info))
 
 
+def decode_tables_bytes(info: Info) -> int:
+    return load().ep_decode_tables_bytes(C.byref(info))
+
+
+def prepare_tables(info: Info, d_stream: int, d_tables: int, tables_bytes: int, stream: int = 0) -> None:
+    """ep_prepare_tables with raw device addresses (ints)."""
+    _check(load().ep_prepare_tables(C.byref(info), d_stream, d_tables, tables_bytes, stream or None), "ep_prepare_tables")
+
+
 def decode_tensor(info: Info, d_stream: int, d_tile_index: int, d_row_scales: int, out_dtype: int, d_out: int,
                   d_scratch: int = 0, scratch_bytes: int = 0, stream: int = 0) -> None:
     """ep_decode_tensor with raw device addresses (ints)."""
@@ -286,7 +305,7 @@ def _out_torch_dtype(dt: int):
 class DeviceBlob:
     """A blob resident in device memory: one uint8 tensor plus the host-side Info."""
 
-    def __init__(self, dev, info: Info):
+    def __init__(self, dev, info: Info, prepare: bool = True):
         self.dev = dev
         self.info = info
         base = dev.data_ptr()
@@ -294,24 +313,36 @@ class DeviceBlob:
         self.d_tile_index = base + info.off_tiles
         self.d_row_scales = base + info.off_scales
         self.scratch = None
-        nb = decode_scratch_bytes(info)
-        if nb:
-            self.scratch = _torch().empty(nb, dtype=_torch().uint8, device=dev.device)
+        self.tables = None
+        torch = _torch()
+        if prepare:
+            # the lookup tables depend on the stream only: derive them once, here, not in every decode
+            self.tables = torch.empty(decode_tables_bytes(info), dtype=torch.uint8, device=dev.device)
+            with torch.cuda.device(dev.device):
+                prepare_tables(info, self.d_stream, self.tables.data_ptr(), self.tables.numel(), _stream_handle(None))
+        else:
+            nb = decode_scratch_bytes(info)
+            if nb:
+                self.scratch = torch.empty(nb, dtype=torch.uint8, device=dev.device)
 
-    def job(self, out_dtype: int, d_out: int, d_row_scales: int | None = None) -> DecodeJob:
+    def job(self, out_dtype: int, d_out: int, d_row_scales: int | None = None, tiles: range | None = None) -> DecodeJob:
         return DecodeJob(C.pointer(self.info), self.d_stream, self.d_tile_index,
                          self.d_row_scales if d_row_scales is None else d_row_scales, out_dtype, d_out,
                          self.scratch.data_ptr() if self.scratch is not None else None,
-                         self.scratch.numel() if self.scratch is not None else 0)
+                         self.scratch.numel() if self.scratch is not None else 0,
+                         tiles.start if tiles is not None else 0, len(tiles) if tiles is not None else 0,
+                         self.tables.data_ptr() if self.tables is not None else None)
 
 
-def upload(blob: Blob | np.ndarray, device="cuda", pinned=None, non_blocking=False) -> DeviceBlob:
+def upload(blob: Blob | np.ndarray, device="cuda", pinned=None, non_blocking=False, prepare: bool = True) -> DeviceBlob:
+    """Copy a blob to the device.  prepare=True also derives the decoder's lookup tables there once
+    (ep_prepare_tables); prepare=False leaves that to every decode call (scratch is allocated if the stream needs it)."""
     torch = _torch()
     data = blob.data if isinstance(blob, Blob) else np.ascontiguousarray(blob, np.uint8)
     info = blob.info if isinstance(blob, Blob) else blob_info(data)
     host = pinned if pinned is not None else torch.from_numpy(data)
     dev = host.to(device, non_blocking=non_blocking)
-    return DeviceBlob(dev, info)
+    return DeviceBlob(dev, info, prepare)
 
 
 def _stream_handle(stream) -> int:
@@ -330,9 +361,12 @@ def decode(dblob: DeviceBlob, out_dtype: int = BF16, out=None, row_scales=None, 
         else:
             out = torch.empty((I.R, I.C), dtype=_out_torch_dtype(out_dtype), device=dblob.dev.device)
     sc = dblob.d_row_scales if row_scales is None else row_scales.data_ptr()
-    decode_tensor(I, dblob.d_stream, dblob.d_tile_index, sc, out_dtype, out.data_ptr(),
-                  dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
-                  dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
+    if dblob.tables is not None:
+        decode_batch([dblob.job(out_dtype, out.data_ptr(), sc)], _stream_handle(stream))
+    else:
+        decode_tensor(I, dblob.d_stream, dblob.d_tile_index, sc, out_dtype, out.data_ptr(),
+                      dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
+                      dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
     return out
 
 
@@ -347,10 +381,13 @@ def decode_tile_range(dblob: DeviceBlob, tiles: range, out_dtype: int = BF16, ou
     if out is None:
         out = torch.empty((last - first) * 8, dtype=_out_torch_dtype(out_dtype), device=dblob.dev.device)
     assert out.numel() >= (last - first) * 8 and out.data_ptr() % 16 == 0
-    decode_tiles(I, dblob.d_stream, dblob.d_tile_index, dblob.d_row_scales, out_dtype,
-                 out.data_ptr() - first * 8 * esize, tiles.start, len(tiles),
-                 dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
-                 dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
+    if dblob.tables is not None:
+        decode_batch([dblob.job(out_dtype, out.data_ptr() - first * 8 * esize, tiles=tiles)], _stream_handle(stream))
+    else:
+        decode_tiles(I, dblob.d_stream, dblob.d_tile_index, dblob.d_row_scales, out_dtype,
+                     out.data_ptr() - first * 8 * esize, tiles.start, len(tiles),
+                     dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
+                     dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
     return out
 
 

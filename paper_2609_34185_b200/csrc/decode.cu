@@ -3,21 +3,23 @@
 // rounding to the output type (Eq. 19), written straight to the weight tensor.  No symbol tensor,
 // no codebook, no tensor cores (the path is not a contraction).
 //
-// Mapping: one warp per tile, one rANS state per lane (the paper's layout); a CTA of 32 warps
-// builds the seventeen slot->(frequency, offset, value) lookup tables once in shared memory from the
-// stream's frequency tables and then streams tiles through them.  A lookup entry is one 32-bit word
+// Mapping: one warp per tile, one rANS state per lane (the paper's layout).  A CTA of 32 warps builds (or
+// copies) the sixteen slot -> (frequency, offset, value) lookup tables of the coordinate fields once in
+// shared memory and then streams tiles through them.  A lookup entry is one word
 //     [31:21] f      [20:11] code     [10:0] u - F
 // where `code` is the symbol's coordinate relative to an even base zlo (z - zlo; 2m - zlo for the m
-// field; 32c for the coset, which makes (entry & 0x1FF800) the byte offset of coset c's tables).
-// f < 2^11 always: a table with a single symbol at b = 11 (f = 2^11) goes to the large-table path.
-// (entry & 0x1FF800) | 0x45800000 is the fp32 number 4096 + code, so one subtraction of
-// 4096 - zlo - c/2 yields the lattice coordinate p exactly, and one fp32 multiply by the row scale
-// gives the product of Eq. 19 with the same operands and rounding as the definition.
+// field).  f < 2^11 always: a coordinate table with a single symbol at b = 11 (f = 2^11) goes to the
+// large-table path.  (entry & 0x1FF800) | 0x45800000 is the fp32 number 4096 + code (| 0x400 adds the
+// half of coset 1), so one subtraction of 4096 - zlo yields the lattice coordinate p exactly, and one fp32
+// multiply by the row scale gives the product of Eq. 19 with the same operands and rounding as the
+// definition.  The coset symbol has two values only: it is decoded by comparing the slot with the
+// frequency of coset 0, without a table.
 //
-// Payload words reach the lanes through a per-warp ring in shared memory, filled 512 bytes at a
-// time by cp.async (16 bytes per lane, source clamped to the end of the payload) a few chunks ahead
-// of the read cursor; the first 640 bytes of the ring are mirrored behind its end so that the nine
-// steps of a group never have to wrap an address.
+// Payload words reach the lanes through a per-tile ring in shared memory, filled 512 bytes at a time by
+// cp.async (16 bytes per lane, source clamped to the end of the payload) ahead of the read cursor; the
+// first 512 bytes of the ring are mirrored behind its end so that the nine steps of a group never have
+// to wrap an address.  (With b <= 11 a lane takes at most seven words in nine steps: a step shortens the
+// state by at most eleven bits, a word adds sixteen.)
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -27,19 +29,56 @@
 
 namespace {
 
-constexpr int kThreads = 1024;                         // one CTA per SM: 32 warps = 32 tiles in flight
-constexpr int kWarps = kThreads / 32;
-constexpr uint32_t kLutEntries = 2048;                 // 2^11 slots per table
-constexpr uint32_t kLutStride = kLutEntries * 4;       // bytes per table in shared memory
-constexpr uint32_t kCosetTableOff = 16 * kLutStride;   // coset table sits after the 16 coordinate tables
-constexpr uint32_t kLutBytes = 17 * kLutStride;        // 139264
-constexpr uint32_t kRingBytes = 2048;                  // four 512-byte chunks per warp
-constexpr uint32_t kRingMirror = 640;                  // >= 9 steps * 32 words * 2 bytes + one lane span
-constexpr uint32_t kRingStride = kRingBytes + kRingMirror;
-constexpr uint32_t kSmemBytes = kLutBytes + kWarps * kRingStride;   // 225280
-constexpr uint32_t kCodeMask = 0x001FF800u;            // 10-bit code field
-constexpr uint32_t kExp4096 = 0x45800000u;             // fp32 bit pattern of 4096.0
-constexpr uint32_t kOwnSlots = 16;                     // table build: slots of a symbol that its own lane writes
+// Tiles a warp decodes side by side (1 to 4) and warps per CTA.  The loop below is written for any number of
+// chains per warp, their instructions interleaved line by line; measured on B200 (8192 x 8192 at 4 bpp to FP16 /
+// the 372 M-parameter layer at 3.5 bpp to BF16, Gparams/s): 32 warps x 1 chain 985 / 1171, 24 x 2 940 / 1104,
+// 16 x 3 781 / 889, 12 x 4 677 / 744.  The loop is bound by the issue slots, the ALU pipe and the shared-memory
+// pipe together (each about 70 % busy), not by the latency of one chain: what counts is the number of warps.
+#ifndef EP_CHAINS
+#define EP_CHAINS 1
+#endif
+#ifndef EP_WARPS
+#define EP_WARPS (EP_CHAINS == 1 ? 32 : 48 / EP_CHAINS)
+#endif
+constexpr uint32_t kChains = EP_CHAINS;
+constexpr int kWarps = EP_WARPS;                             // warps per CTA (one CTA per SM)
+constexpr int kThreads = kWarps * 32;
+constexpr uint32_t kTilesPerRound = kWarps * kChains;        // 48 tiles per CTA at a time
+static_assert(kTilesPerRound == ep::kDecodeTilesPerCta, "tile-size suggestions assume this many tiles per CTA");
+constexpr uint32_t kLutEntries = 2048;                       // 2^11 slots per table
+constexpr uint32_t kLutStride = kLutEntries * 4;             // bytes per table in shared memory
+constexpr uint32_t kCosetStride = 8 * kLutStride;            // the eight tables of coset 1 follow those of coset 0
+constexpr uint32_t kLutBytes = 16 * kLutStride;              // 131072
+constexpr uint32_t kChunk = 512;                             // bytes per cp.async round of a warp
+constexpr uint32_t kRingSlots = 3;
+constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536
+constexpr uint32_t kRingMirror = 512;                        // >= 7 words * 32 lanes * 2 bytes + one lane span (62)
+constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 per chain
+constexpr uint32_t kCtxBytes = 32 + 32 * kChains;            // per warp: what the rare paths of the hot loop need
+constexpr uint32_t kRingBase = kLutBytes;
+constexpr uint32_t kCtxBase = kRingBase + kWarps * kChains * kRingStride;
+constexpr uint32_t kSmemBytes = kCtxBase + kWarps * kCtxBytes;   // 231680
+static_assert(kSmemBytes <= 232448, "more shared memory than an sm_100 CTA can have");
+constexpr uint32_t kCodeMask = 0x001FF800u;                  // 10-bit code field
+constexpr uint32_t kExp4096 = 0x45800000u;                   // fp32 bit pattern of 4096.0
+constexpr uint32_t kOwnSlots = 16;                           // table build: slots of a symbol that its own lane writes
+constexpr uint32_t kEntryUnused = 1u << 21;                  // f = 1: what a slot no symbol owns holds (damaged tables)
+
+// per-warp context block (byte offsets); chain c has its part at kCtxChain + c * kCtxChainStride
+constexpr uint32_t kCtxScales = 0;         // u64 row scales
+constexpr uint32_t kCtxRowBytes = 8;       // u32 output bytes per row
+constexpr uint32_t kCtxRowMax = 12;        // u32 last row index
+constexpr uint32_t kCtxMul21 = 16;         // u32 2^21 and
+constexpr uint32_t kCtxMul11 = 20;         // u32 2^11: multipliers the hot loop must not see as constants (see EP_STEP)
+constexpr uint32_t kCtxRowRcp = 24;        // u32 ceil(2^32 / bytes per row)
+constexpr uint32_t kCtxChain = 32, kCtxChainStride = 32;
+constexpr uint32_t kCcA0 = 0;              // u64 global address of chunk 0 (first payload byte rounded down to 16)
+constexpr uint32_t kCcRoom = 8;            // u32 bytes from a0 to the end of the payload
+constexpr uint32_t kCcNext = 12;           // u32 next chunk to request
+constexpr uint32_t kCcNextSlot = 16;       // u32 the ring slot it goes to (chunk number mod 3)
+constexpr uint32_t kCcWbase = 20;          // u32 ring address of byte position 0 (cursor address minus position)
+constexpr uint32_t kCcEndo = 24;           // u32 output byte offset after the tile's last block
+constexpr uint32_t kCcRing = 28;           // u32 ring base (shared-memory address)
 
 __device__ unsigned int g_ep_status = 0;
 
@@ -48,6 +87,7 @@ struct JobParams {
     const uint32_t *tile_index;   // n_tiles records of 33 words + 1 final word
     const float *scales;
     void *out;
+    const uint32_t *lut_image;    // tables prepared by ep_prepare_tables (16 x 2048 entries), or null: build them here
     uint32_t off_freq;            // byte offset of the u16 frequency arrays inside the blob
     uint32_t off_payload;
     uint32_t total_words;
@@ -56,9 +96,12 @@ struct JobParams {
     uint32_t V, n_tiles, b;       // n_tiles: tiles of the whole tensor
     uint32_t tile0, tile_cnt;     // the tiles this launch decodes: [tile0, tile0 + tile_cnt)
     int32_t zlo;                  // even, <= -2
-    uint32_t rounds;              // ceil(tile_cnt / warps): in one round the 32 warps of a CTA take 32 consecutive tiles
+    uint32_t rounds;              // ceil(tile_cnt / 48): in one round the warps of a CTA take 48 consecutive tiles
     uint32_t round_cost;          // work of one round in groups of 32 vectors (ceil(V / 32))
     uint32_t cost_begin;          // sum of rounds * round_cost over the jobs before this one
+    uint32_t row_bytes;           // output bytes per row
+    uint32_t row_rcp;             // ceil(2^32 / row_bytes)
+    uint32_t row_max;             // index of the last row
     int16_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint16_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
@@ -78,6 +121,9 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
 }
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t addr, uint64_t v) {
+    asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, uint64_t src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
@@ -141,18 +187,19 @@ __device__ __forceinline__ uint32_t cvt_s8(float v) {
 }
 
 // ---- lookup-table construction (per CTA, from the stream's frequency tables) ---------------------
-// Warp t fills table t.  Symbols are taken 32 at a time: a warp scan gives each lane its symbol's
-// first slot, every lane writes the first sixteen slots of its own symbol, and the few symbols with more
-// slots than that are then filled by the whole warp, one after the other (that loop is serial: its length,
-// not the number of stores, is what the build time depends on).
-__device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t lut_addr, uint32_t warp, uint32_t lane) {
-  for (uint32_t t = warp; t < EP_NUM_TABLES; t += kWarps) {
+// Warp t - 1 fills coordinate table t (t = 1..16; the coset table t = 0 needs none).  Symbols are taken 32 at
+// a time: a warp scan gives each lane its symbol's first slot, every lane writes the first sixteen slots of
+// its own symbol, and the few symbols with more slots than that are then filled by the whole warp, one
+// after the other (that loop is serial: its length, not the number of stores, is what the build time
+// depends on).  `base` receives the 2048 entries: a shared-memory address here, see ep_prepare_tables_kernel
+// for the same routine writing a table image to global memory.
+template <class Store>
+__device__ __forceinline__ void build_one_table(const JobParams &J, uint32_t t, uint32_t lane, Store put) {
     const uint32_t K = J.tK[t];
-    if (K == 0) continue;
     const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_freq) + J.foff[t];
     const int32_t tmin = J.tmin[t];
-    const uint32_t base = lut_addr + (t == 0 ? kCosetTableOff : (t - 1) * kLutStride);
-    const bool is_m = (t != 0) && (((t - 1) & 7) == 7);
+    const bool is_m = ((t - 1) & 7) == 7;
+    const uint32_t slots = min(1u << J.b, kLutEntries);
     uint32_t run = 0;
     for (uint32_t j0 = 0; j0 < K; j0 += 32) {
         const uint32_t j = j0 + lane;
@@ -165,12 +212,12 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
         }
         const uint32_t first = run + incl - f;
         const int32_t v = tmin + int32_t(j);
-        const uint32_t code = t == 0 ? uint32_t(v) * 32u : uint32_t((is_m ? 2 * v : v) - J.zlo);
+        const uint32_t code = uint32_t((is_m ? 2 * v : v) - J.zlo);
         const uint32_t entry = (f << 21) | ((code & 0x3FFu) << 11);
         if (f >= kLutEntries) atomicOr(&g_ep_status, 1u);   // not a stream the launcher sends here: f does not fit its field
 #pragma unroll
         for (uint32_t u = 0; u < kOwnSlots; ++u)
-            if (u < f && first + u < kLutEntries) sts32(base + 4u * (first + u), entry | u);
+            if (u < f && first + u < slots) put(first + u, entry | u);
         uint32_t big = __ballot_sync(0xFFFFFFFFu, f > kOwnSlots);
         while (big) {
             const int i = __ffs(big) - 1;
@@ -178,65 +225,56 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
             const uint32_t fi = __shfl_sync(0xFFFFFFFFu, f, i);
             const uint32_t Fi = __shfl_sync(0xFFFFFFFFu, first, i);
             const uint32_t ei = __shfl_sync(0xFFFFFFFFu, entry, i);
-            for (uint32_t u = kOwnSlots + lane; u < fi && Fi + u < kLutEntries; u += 32) sts32(base + 4u * (Fi + u), ei | u);
+            for (uint32_t u = kOwnSlots + lane; u < fi && Fi + u < slots; u += 32) put(Fi + u, ei | u);
         }
         run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
-    // frequencies of a damaged stream may sum to less than 2^b: no slot keeps what an earlier CTA left there
-    // (the coset entry's code field is added to a shared-memory address)
-    for (uint32_t u = run + lane; u < (1u << J.b) && u < kLutEntries; u += 32) sts32(base + 4u * u, 0u);
-  }
+    // frequencies of a damaged stream may sum to less than 2^b, and a table may be empty: a slot that no symbol
+    // owns gets f = 1, never what an earlier job left there (the word bound of the ring relies on f >= 1)
+    for (uint32_t u = min(run, slots) + lane; u < slots; u += 32) put(u, kEntryUnused);
 }
 
-// ---- one rANS symbol (Eq. 18) followed by renormalisation --------------------------------------
+__device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t lut_addr, uint32_t warp, uint32_t lane) {
+    for (uint32_t t = 1 + warp; t < EP_NUM_TABLES; t += kWarps) {
+        const uint32_t base = lut_addr + (t - 1) * kLutStride;
+        build_one_table(J, t, lane, [base](uint32_t slot, uint32_t e) { sts32(base + 4u * slot, e); });
+    }
+}
+
+// the prepared image of the same sixteen tables: 128 KB copied by all threads of the CTA, 16 bytes each.  The
+// copy is only started here; whoever reads the tables first waits for it (cp.async.wait_group, then a CTA barrier).
+__device__ __forceinline__ void copy_tables_smem(const uint32_t *image, uint32_t lut_addr) {
+    const uint64_t src = reinterpret_cast<uint64_t>(image);
+    for (uint32_t o = 16u * threadIdx.x; o < kLutBytes; o += 16u * kThreads) cp_async16(lut_addr + o, src + o, 16);
+    cp_async_commit();
+}
+
+// frequencies of the two cosets as the decode uses them: u < f0 means coset 0.  A coset that never occurs
+// has frequency 0 in the stream and is never selected; it is raised to 1 here only so that a damaged stream
+// cannot produce a state that takes a word in every step.
+struct CosetFreq { uint32_t f0, f1; };
+__device__ __forceinline__ CosetFreq load_coset(const JobParams &J) {
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_freq) + J.foff[0];
+    uint32_t f0 = 0, f1 = 0;
+    if (J.tmin[0] == 0) {
+        f0 = __ldg(fq);
+        if (J.tK[0] > 1) f1 = __ldg(fq + 1);
+    } else {
+        f1 = __ldg(fq);
+    }
+    const uint32_t M = 1u << J.b;
+    CosetFreq c;
+    c.f0 = min(f0, M);                 // u < f0 <=> coset 0 (f0 = 0: never)
+    c.f1 = max(min(f1, M), 1u);
+    return c;
+}
+
+// ---- one rANS symbol (Eq. 18) followed by renormalisation: plain version --------------------------
 // x: this lane's state; wa: shared-memory byte address of the tile's word cursor (same in all lanes).
 // Lanes that need a word take them in lane order: lane l reads the word popc(ballot & lanes below l)
-// places after the cursor (every lane reads, only the needy merge); the cursor then advances by
-// popc(ballot) words.  Returns the table entry.
-template <uint32_t TABLE_OFF>
-__device__ __forceinline__ uint32_t rans_step(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &wa,
-                                              uint32_t lt) {
-    uint32_t e;
-    asm volatile(
-        "{\n\t"
-        ".reg .pred p;\n\t"
-        ".reg .b32 u, f, q, bias, bal, t, w;\n\t"
-        "and.b32 u, %1, %3;\n\t"
-        "shl.b32 u, u, 2;\n\t"
-        "add.u32 u, u, %5;\n\t"
-        "ld.shared.u32 %0, [u + %7];\n\t"
-        "shr.u32 f, %0, 21;\n\t"
-        "and.b32 bias, %0, 0x7FF;\n\t"
-        "shr.u32 q, %1, %4;\n\t"
-        "mad.lo.u32 %1, f, q, bias;\n\t"
-        "setp.lt.u32 p, %1, 32768;\n\t"
-        "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"
-        "and.b32 t, bal, %6;\n\t"
-        "popc.b32 t, t;\n\t"
-        "shl.b32 t, t, 1;\n\t"
-        "add.u32 t, t, %2;\n\t"
-        "ld.shared.u16 w, [t];\n\t"
-        "@p mad.lo.u32 %1, %1, 65536, w;\n\t"
-        "popc.b32 t, bal;\n\t"
-        "shl.b32 t, t, 1;\n\t"
-        "add.u32 %2, %2, t;\n\t"
-        "}"
-        : "=&r"(e), "+r"(x), "+r"(wa)
-        : "r"(mask), "r"(b), "r"(table_addr), "r"(lt), "n"(TABLE_OFF)
-        : "memory");
-    return e;
-}
-
-// the same for the last, partly filled group of a tile: lanes without a vector leave their state alone
-__device__ __forceinline__ uint32_t rans_step_tail(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &wa,
-                                                   uint32_t lt, bool act) {
-    uint32_t e = 0;
-    bool need = false;
-    if (act) {
-        e = lds32(table_addr + ((x & mask) << 2));
-        x = (e >> 21) * (x >> b) + (e & 0x7FFu);
-        need = x < ep::kStateLow;
-    }
+// places after the cursor; the cursor then advances by popc(ballot) words.  Lanes without a vector
+// (`act` false: the last, partly filled group of a tile) leave their state alone and take no word.
+__device__ __forceinline__ void renorm_plain(uint32_t &x, uint32_t &wa, uint32_t lt, bool need) {
     const uint32_t bal = __ballot_sync(0xFFFFFFFFu, need);
     if (need) {
         uint16_t w;
@@ -244,7 +282,32 @@ __device__ __forceinline__ uint32_t rans_step_tail(uint32_t &x, uint32_t table_a
         x = (x << 16) | w;
     }
     wa += 2u * __popc(bal);
+}
+__device__ __forceinline__ uint32_t rans_step_plain(uint32_t &x, uint32_t table_addr, uint32_t mask, uint32_t b, uint32_t &wa,
+                                                    uint32_t lt, bool act) {
+    uint32_t e = 0;
+    bool need = false;
+    if (act) {
+        e = lds32(table_addr + ((x & mask) << 2));
+        x = (e >> 21) * (x >> b) + (e & 0x7FFu);
+        need = x < ep::kStateLow;
+    }
+    renorm_plain(x, wa, lt, need);
     return e;
+}
+// the coset symbol: 0 if the slot lies below f0, else 1
+__device__ __forceinline__ uint32_t coset_step_plain(uint32_t &x, CosetFreq cf, uint32_t mask, uint32_t b, uint32_t &wa,
+                                                     uint32_t lt, bool act) {
+    uint32_t c = 0;
+    bool need = false;
+    if (act) {
+        const uint32_t u = x & mask;
+        c = u < cf.f0 ? 0u : 1u;
+        x = (c ? cf.f1 : max(cf.f0, 1u)) * (x >> b) + (c ? u - cf.f0 : u);
+        need = x < ep::kStateLow;
+    }
+    renorm_plain(x, wa, lt, need);
+    return c;
 }
 
 template <int DT>
@@ -318,48 +381,35 @@ struct BlockBytes { static constexpr uint32_t value = Out<DT>::kBlockBytes; };
 template <>
 struct BlockBytes<EP_FIELDS_I32> { static constexpr uint32_t value = 36; };
 
-// ---- one group of 32 vectors: nine symbols per lane, then Eq. 5 / Eq. 19 and the store ------------
-template <int DT, bool TAIL>
-__device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &wa, uint32_t lut_addr, uint32_t mask, uint32_t b, uint32_t lt,
-                                             bool act, uint32_t k0_bits, float sigma, int32_t zlo, void *dst) {
+// ---- one group of 32 vectors, plain version: nine symbols per lane, then Eq. 5 / Eq. 19 and the store ---
+template <int DT>
+__device__ __forceinline__ void decode_group_plain(uint32_t &x, uint32_t &wa, uint32_t lut_addr, CosetFreq cf, uint32_t mask,
+                                                   uint32_t b, uint32_t lt, bool act, uint32_t k0_bits, float sigma,
+                                                   int32_t zlo, void *dst) {
     uint32_t e[9];
-    e[0] = TAIL ? rans_step_tail(x, lut_addr + kCosetTableOff, mask, b, wa, lt, act)
-                : rans_step<kCosetTableOff>(x, lut_addr, mask, b, wa, lt);
-    // 0 or 65536: byte offset of this coset's tables (one bit only, so that a damaged table cannot point elsewhere)
-    const uint32_t coff = e[0] & 0x10000u;
-    const uint32_t tab = lut_addr + coff;
-    if (TAIL) {
+    const uint32_t c = coset_step_plain(x, cf, mask, b, wa, lt, act);
+    const uint32_t tab = lut_addr + c * kCosetStride;
 #pragma unroll
-        for (int k = 1; k <= 8; ++k) e[k] = rans_step_tail(x, tab + uint32_t(k - 1) * kLutStride, mask, b, wa, lt, act);
-    } else {
-        e[1] = rans_step<0 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[2] = rans_step<1 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[3] = rans_step<2 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[4] = rans_step<3 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[5] = rans_step<4 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[6] = rans_step<5 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[7] = rans_step<6 * kLutStride>(x, tab, mask, b, wa, lt);
-        e[8] = rans_step<7 * kLutStride>(x, tab, mask, b, wa, lt);
-    }
-    if (TAIL && !act) return;
+    for (int k = 1; k <= 8; ++k) e[k] = rans_step_plain(x, tab + uint32_t(k - 1) * kLutStride, mask, b, wa, lt, act);
+    if (!act) return;
     // parity of z1 + ... + z7 = xor of the codes' lowest bits (zlo is even); it is the lowest bit of z8
     const uint32_t par = (e[1] ^ e[2] ^ e[3] ^ e[4] ^ e[5] ^ e[6] ^ e[7]) & 0x800u;
     if constexpr (DT == EP_FIELDS_I32) {
         int32_t *f = reinterpret_cast<int32_t *>(dst);
-        f[0] = int32_t(coff >> 16);
+        f[0] = int32_t(c);
 #pragma unroll
         for (int k = 1; k <= 7; ++k) f[k] = int32_t((e[k] & kCodeMask) >> 11) + zlo;
         f[8] = (int32_t((e[8] & kCodeMask) >> 11) + zlo) >> 1;
     } else {
-        // (entry & mask) | 0x45800000 is 4096 + code as fp32; subtracting kc = 4096 - zlo - c/2 gives
-        // p = z + c/2 exactly (one ulp here is 2^-11, so c/2 is 1024 ulps of the bit pattern)
-        const uint32_t kc = k0_bits - (coff >> 6);
-        const uint64_t kk = pack64(kc, kc);
+        // (entry & mask) | 0x45800000 | c << 10 is 4096 + code + c/2 as fp32 (one ulp here is 2^-11); subtracting
+        // 4096 - zlo gives p = z + c/2 exactly
+        const uint32_t cc = kExp4096 | (c << 10);
+        const uint64_t kk = pack64(k0_bits, k0_bits);
         const uint64_t ss = pack64(__float_as_uint(sigma), __float_as_uint(sigma));
         uint32_t xb[8];
 #pragma unroll
-        for (int k = 1; k <= 7; ++k) xb[k - 1] = (e[k] & kCodeMask) | kExp4096;
-        xb[7] = (e[8] & kCodeMask) | par | kExp4096;
+        for (int k = 1; k <= 7; ++k) xb[k - 1] = (e[k] & kCodeMask) | cc;
+        xb[7] = (e[8] & kCodeMask) | par | cc;
         float w[8];
 #pragma unroll
         for (int i = 0; i < 8; i += 2) unpack64(mul2(sub2(pack64(xb[i], xb[i + 1]), kk), ss), w[i], w[i + 1]);
@@ -369,419 +419,556 @@ __device__ __forceinline__ void decode_group(uint32_t &x, uint32_t &wa, uint32_t
 
 // ---- payload ring ------------------------------------------------------------------------------------
 // chunk c of a tile = global bytes [a0 + 512c, a0 + 512c + 512), a0 = tile's first word rounded down to
-// 16 bytes; it lives in ring slot c & 3.  `room` = bytes from a0 to the end of the payload: nothing
-// beyond it is read (cp.async zero-fills the rest).
+// 16 bytes; it lives in ring slot c mod 3, and a chunk in slot 0 is written a second time behind the ring's
+// end.  `room` = bytes from a0 to the end of the payload: nothing beyond it is read (cp.async zero-fills
+// the rest).
 __device__ __forceinline__ void ring_issue(uint32_t ring, uint64_t a0, uint32_t room, uint32_t c, uint32_t lane) {
-    uint32_t o = 512u * c + 16u * lane;
+    uint32_t o = kChunk * c + 16u * lane;
     uint32_t n = 16;
     if (o + 16u > room) {
         n = o < room ? room - o : 0u;
         if (n == 0) o = 0;                       // nothing is read, but keep the address a valid one
     }
-    const uint32_t slot = c & 3u;
-    const uint32_t dst = ring + 512u * slot + 16u * lane;
+    const uint32_t slot = c % kRingSlots;
+    const uint32_t dst = ring + kChunk * slot + 16u * lane;
     cp_async16(dst, a0 + o, n);
-    if (slot == 0 || (slot == 1 && lane < 8)) cp_async16(dst + kRingBytes, a0 + o, n);   // mirror of the first 640 bytes
+    if (slot == 0) cp_async16(dst + kRingBytes, a0 + o, n);
     cp_async_commit();
 }
 
-// The cursor entered a new 512-byte chunk: request chunks up to three ahead of it and wait for all but
-// the newest.  `threshold` = start of the chunk after the cursor's at the previous service; chunks up
-// to (threshold >> 9) + 2 have been requested.  A group touches at most 576 + 62 bytes from its start,
-// i.e. chunks cur .. cur+2, which are complete after this call.
+// The cursor entered a new 512-byte chunk: request chunks up to two ahead of it and wait for all but the
+// newest.  `threshold` = start of the chunk after the cursor's at the previous service; chunks up to
+// (threshold >> 9) + 1 have been requested.  A group touches at most 448 + 62 bytes from its start,
+// i.e. chunks cur and cur + 1, which are complete after this call.
 __device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_t room, uint32_t pos, uint32_t &threshold,
                                              uint32_t lane) {
     const uint32_t cur = pos >> 9;
-    for (uint32_t c = (threshold >> 9) + 3u; c < cur + 4u; ++c) ring_issue(ring, a0, room, c, lane);
+    for (uint32_t c = (threshold >> 9) + 2u; c < cur + 3u; ++c) ring_issue(ring, a0, room, c, lane);
     cp_async_wait<1>();
     __syncwarp();
-    threshold = 512u * (cur + 1u);
+    threshold = kChunk * (cur + 1u);
 }
 
-// Plain C++ version of the tile loop, used for the field-dump mode and for tensors with fewer than 32
-// blocks per row (WIDE = false: a group may then cross several rows).
-template <int DT, bool WIDE>
-__device__ __forceinline__ void decode_tile(const JobParams &J, uint32_t tile, uint32_t lut_addr, uint32_t ring, uint32_t lane) {
+// what a chain needs to know about its tile
+struct TileSetup {
+    uint32_t x;            // this lane's state, forced into [2^15, 2^31) (a no-op for a valid stream)
+    uint32_t off, end;     // first payload word of the tile and of the next one
+    uint32_t v0, nv;       // first block and number of blocks
+    uint64_t a0;           // global address of chunk 0
+    uint32_t lead, room;   // cursor position inside chunk 0; payload bytes from a0 on
+};
+__device__ __forceinline__ TileSetup tile_setup(const JobParams &J, uint32_t tile, bool valid, uint32_t lane) {
+    TileSetup T;
     const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
-    uint32_t x = rec[lane];
-    const uint32_t off = min(rec[32], J.total_words);   // a damaged index must not move reads outside the payload
-    const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
-    const uint32_t v0 = tile * J.V;
-    const uint32_t nv = min(J.V, J.n_vec - v0);
+    T.x = max(rec[lane] & 0x7FFFFFFFu, ep::kStateLow);
+    T.off = min(rec[32], J.total_words);    // a damaged index must not move reads outside the payload
+    T.end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
+    T.v0 = tile * J.V;
+    T.nv = valid ? min(J.V, J.n_vec - T.v0) : 0u;
+    const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
+    const uint64_t first = pay + 2ull * T.off;
+    T.a0 = first & ~15ull;
+    T.lead = uint32_t(first - T.a0);
+    T.room = uint32_t(pay + 2ull * J.total_words - T.a0);     // the payload is shorter than 2 GB
+    return T;
+}
+
+// Plain C++ version of the tile loop, used for the field-dump mode, for streams with b < 11 and for tensors with
+// fewer than 32 blocks per row (a group may then cross several rows).
+template <int DT>
+__device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t tile, uint32_t lut_addr, CosetFreq cf,
+                                                  uint32_t ring, uint32_t lane) {
+    const TileSetup T = tile_setup(J, tile, true, lane);
+    uint32_t x = T.x;
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
     const uint32_t per_row = J.per_row;
-    const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
-    const uint64_t first = pay + 2ull * off;
-    const uint64_t a0 = first & ~15ull;
-    const uint32_t lead = uint32_t(first - a0);
-    const uint32_t room = uint32_t(pay + 2ull * J.total_words - a0);     // the payload is shorter than 4 GB
-    uint32_t pos = lead;          // byte position of the cursor relative to a0
+    uint32_t pos = T.lead;        // byte position of the cursor relative to a0
     uint32_t threshold;           // next chunk boundary the cursor has not yet crossed
-    for (uint32_t c = 0; c < 4; ++c) ring_issue(ring, a0, room, c, lane);
+    for (uint32_t c = 0; c < kRingSlots; ++c) ring_issue(ring, T.a0, T.room, c, lane);
     cp_async_wait<1>();
     __syncwarp();
-    threshold = 512u;
+    threshold = kChunk;
     const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
-    uint32_t v = v0 + lane;
-    uint32_t row = v / per_row, col = v - row * per_row;
-    uint8_t *dst = static_cast<uint8_t *>(J.out) + size_t(v) * BlockBytes<DT>::value;
-    const uint32_t full = nv >> 5;
-    for (uint32_t g = 0; g < full; ++g) {
-        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
-        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
+    const uint32_t row_max = J.n_vec / per_row - 1u;
+    for (uint32_t g = 0; g * 32u < T.nv; ++g) {
+        if (pos >= threshold) ring_service(ring, T.a0, T.room, pos, threshold, lane);
+        const uint32_t wa0 = ring + pos % kRingBytes;
         uint32_t wa = wa0;
-        const float sigma = (DT == EP_FIELDS_I32) ? 0.f : __ldg(J.scales + row);
-        decode_group<DT, false>(x, wa, lut_addr, mask, b, lt, true, k0_bits, sigma, J.zlo, dst);
-        pos += wa - wa0;
-        dst += 32u * BlockBytes<DT>::value;
-        col += 32;
-        if (WIDE) {
-            const bool wrap = col >= per_row;
-            col -= wrap ? per_row : 0u;
-            row += wrap ? 1u : 0u;
-        } else {
-            while (col >= per_row) { col -= per_row; ++row; }
-        }
-    }
-    if (nv & 31u) {
-        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
-        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
-        uint32_t wa = wa0;
-        const bool act = lane < (nv & 31u);
-        const float sigma = (DT == EP_FIELDS_I32 || !act) ? 0.f : __ldg(J.scales + row);
-        decode_group<DT, true>(x, wa, lut_addr, mask, b, lt, act, k0_bits, sigma, J.zlo, dst);
+        const uint32_t i = g * 32u + lane;
+        const bool act = i < T.nv;
+        const uint32_t v = T.v0 + i;
+        const float sigma = (DT == EP_FIELDS_I32) ? 0.f : __ldg(J.scales + min(v / per_row, row_max));
+        decode_group_plain<DT>(x, wa, lut_addr, cf, mask, b, lt, act, k0_bits, sigma, J.zlo,
+                               static_cast<uint8_t *>(J.out) + size_t(v) * BlockBytes<DT>::value);
         pos += wa - wa0;
     }
     cp_async_wait<0>();          // nothing may still be landing in the ring when the next tile starts
     __syncwarp();
     // integrity: the encoder started every state at 2^15 and the tile's words end where the next tile's begin
-    const bool bad = (x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end);
+    const bool bad = (x != ep::kStateLow) || (T.off + ((pos - T.lead) >> 1) != T.end);
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
 }
 
-// ---- the hot loop in PTX -------------------------------------------------------------------------------
-// All full groups of one tile.  Written as one asm statement so that every branch can be marked
-// warp-uniform (bra.uni) and the rare work - refilling the payload ring, moving to the next row, leaving
-// the loop - sits out of line behind ONE warp vote per group.  Per group: 9 x rans step, Eq. 5 / Eq. 19
-// on eight weights, one vector store.
+// ---- the hot loop in PTX: several tiles per warp ----------------------------------------------------------
+// All groups of EP_CHAINS tiles ("chains" A, B, ...), written as one asm statement so that every branch can be
+// marked warp-uniform (bra.uni), the chains' instructions can be interleaved, and the rare work - refilling a
+// payload ring, moving to the next row, a tile's end - sits out of line behind ONE warp vote per loop pass.
 //
-// Register roles (asm operands):
-//   x      rANS state                      wa    cursor (shared-memory byte address)
-//   wthr   cursor value that triggers the next ring service (next 512-byte chunk boundary)
-//   wbase  wa - (byte position of the cursor relative to a0)
-//   doff   byte offset of this lane's block in the output
-//   chg    value of doff at which this lane enters its next row;  row = row index;  sig = row scale bits
-//   lim    min(chg, endo): the fast path compares doff with this alone;  endo = doff after the last group
-//   srcp, rem, nextc  ring refill state: global address of this lane's 16 bytes of chunk nextc and
-//                     the payload bytes left from there (may be <= 0)
-#define EP_S_FQ(E)                                              \
-    "shr.u32 f, " E ", 21;\n\t"                                 \
-    "shr.u32 q, %0, %14;\n\t"
-#define EP_S_FETCH                                              \
-    "and.b32 t, bal, %12;\n\t"                                  \
-    "popc.b32 t, t;\n\t"                                        \
-    "shl.b32 t, t, 1;\n\t"                                      \
-    "add.u32 t, t, %1;\n\t"                                     \
-    "ld.shared.u16 w, [t];\n\t"                                 \
-    "@p mad.lo.u32 %0, %0, 65536, w;\n\t"                       \
-    "popc.b32 t, bal;\n\t"                                      \
-    "shl.b32 t, t, 1;\n\t"                                      \
-    "add.u32 %1, %1, t;\n\t"
-#define EP_S_STEP(E, TAB, OFF)                                  \
-    "and.b32 u, %0, %13;\n\t"                                   \
-    "shl.b32 u, u, 2;\n\t"                                      \
-    "add.u32 u, u, " TAB ";\n\t"                                \
-    "ld.shared.u32 " E ", [u+" OFF "];\n\t"                     \
-    EP_S_FQ(E)                                                  \
-    "and.b32 bias, " E ", 0x7FF;\n\t"                           \
-    "mad.lo.u32 %0, f, q, bias;\n\t"                            \
-    "setp.lt.u32 p, %0, 32768;\n\t"                             \
-    "vote.sync.ballot.b32 bal, p, 0xffffffff;\n\t"              \
-    EP_S_FETCH
+// Word addresses.  Lane l of a chain keeps its own address a_l of the word it would take in the current step.
+// With bal_k the ballot of the lanes that need a word after step k,
+//     a_l(k) = a_l(k-1) + 2 popc((bal_k & below_l) | (bal_{k-1} & ~below_l)):
+// the words taken in step k-1 by lanes l and above, plus those taken in step k by the lanes below.  The two
+// masks are disjoint, so one bit-select and ONE population count per step replace the prefix count and the
+// cursor advance (lane 0's address is the tile's word cursor before the step).
+//
+// Loop-carried per chain: x state, a word address, bal last ballot, doff byte offset of this lane's block in the
+// output; inside the asm: lim = first doff at which this lane leaves its row or the tile, wthr = ring address at
+// which the cursor leaves its 512-byte chunk (minus 2), ss = the row scale twice, act = lane has a block.
+// A chain whose tile has ended (or that never had one) runs along with all lanes inactive: states and
+// addresses stand still, nothing is stored.
+//
+// asm operands: chain c has x, a, bal, doff at %(4c) .. %(4c+3); then come the shared inputs, named here:
+#if EP_CHAINS == 1
+#define EP_LT "%4"
+#define EP_LUT0 "%5"
+#define EP_LUT1 "%6"
+#define EP_CTX "%7"
+#define EP_KK "%8"
+#define EP_OUT "%9"
+#define EP_F0 "%10"
+#define EP_F1 "%11"
+#define EP_L16 "%12"
+#elif EP_CHAINS == 2
+#define EP_LT "%8"     /* lanes below this one (mask) */
+#define EP_LUT0 "%9"   /* tables of coset 0 */
+#define EP_LUT1 "%10"  /* tables of coset 1 */
+#define EP_CTX "%11"   /* this warp's context block */
+#define EP_KK "%12"    /* {4096 - zlo, 4096 - zlo} as fp32 pair */
+#define EP_OUT "%13"   /* output base address */
+#define EP_F0 "%14"    /* frequency of coset 0 */
+#define EP_F1 "%15"    /* frequency of coset 1, at least 1 */
+#define EP_L16 "%16"   /* 16 * lane */
+#elif EP_CHAINS == 3
+#define EP_LT "%12"
+#define EP_LUT0 "%13"
+#define EP_LUT1 "%14"
+#define EP_CTX "%15"
+#define EP_KK "%16"
+#define EP_OUT "%17"
+#define EP_F0 "%18"
+#define EP_F1 "%19"
+#define EP_L16 "%20"
+#else
+#define EP_LT "%16"
+#define EP_LUT0 "%17"
+#define EP_LUT1 "%18"
+#define EP_CTX "%19"
+#define EP_KK "%20"
+#define EP_OUT "%21"
+#define EP_F0 "%22"
+#define EP_F1 "%23"
+#define EP_L16 "%24"
+#endif
+// one macro call per chain: M(S = suffix, X, AW, BAL, DOFF, CB = byte offset of the chain's context, more...)
+#define EP_CH_A(M, ...) M("A", "%0", "%1", "%2", "%3", "32", ##__VA_ARGS__)
+#define EP_CH_B(M, ...) M("B", "%4", "%5", "%6", "%7", "64", ##__VA_ARGS__)
+#define EP_CH_C(M, ...) M("C", "%8", "%9", "%10", "%11", "96", ##__VA_ARGS__)
+#define EP_CH_D(M, ...) M("D", "%12", "%13", "%14", "%15", "128", ##__VA_ARGS__)
+#if EP_CHAINS == 1
+#define EP_ALL(M, ...) EP_CH_A(M, ##__VA_ARGS__)
+#elif EP_CHAINS == 2
+#define EP_ALL(M, ...) EP_CH_A(M, ##__VA_ARGS__) EP_CH_B(M, ##__VA_ARGS__)
+#elif EP_CHAINS == 3
+#define EP_ALL(M, ...) EP_CH_A(M, ##__VA_ARGS__) EP_CH_B(M, ##__VA_ARGS__) EP_CH_C(M, ##__VA_ARGS__)
+#else
+#define EP_ALL(M, ...) EP_CH_A(M, ##__VA_ARGS__) EP_CH_B(M, ##__VA_ARGS__) EP_CH_C(M, ##__VA_ARGS__) EP_CH_D(M, ##__VA_ARGS__)
+#endif
 
-#define EP_S_PAIR(P, XA, XB, WA, WB)                            \
-    "mov.b64 " P ", {" XA ", " XB "};\n\t"                      \
-    "sub.rn.f32x2 " P ", " P ", kk;\n\t"                        \
-    "mul.rn.f32x2 " P ", " P ", ss;\n\t"                        \
-    "mov.b64 {" WA ", " WB "}, " P ";\n\t"
+#define EP_CM "0x1FF800"
+// The loop body is written line by line: every macro below emits ONE instruction for ONE chain, and EP_ALL
+// repeats it for all chains before the next line follows.  The assembler keeps this order, so a chain's next
+// dependent instruction comes only after the other chains' same instruction: that distance, not the
+// scheduler, is what hides the latencies inside a warp.
+// Common parameters of a line: S, X, AW, BAL, DOFF, CB (see EP_CH_A); then E = name of the entry register
+// (a suffix is added), OFF = byte offset of the field's table, BIN / BOUT = which register holds the previous /
+// receives the new ballot: NA, NB (temporaries) or BL (the chain's loop-carried operand).
+#define EP_B_NA(S, BAL) "na" S
+#define EP_B_NB(S, BAL) "nb" S
+#define EP_B_BL(S, BAL) BAL
+// a coordinate field: table OFF / 8192 of the lane's coset (Eq. 18)
+#ifdef EP_STEP_WIDE
+// x * 2^21 as a 64-bit product gives x >> 11 in the high word and the slot in the top bits of the low word,
+// e * 2^11 gives f in the high word: both on the multiply-add pipe instead of shifts and masks on the ALU pipe
+// (the two multipliers come from memory so that the assembler does not turn the products back into shifts)
+#define EP_L1(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "mul.wide.u32 xw" S ", " X ", m21;\n\t" "mov.b64 {u" S ", q" S "}, xw" S ";\n\t"
+#define EP_L2(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "shr.u32 u" S ", u" S ", 19;\n\t" "add.u32 u" S ", u" S ", tab" S ";\n\t"
+#define EP_L3(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "ld.shared.u32 " E S ", [u" S "+" OFF "];\n\t"
+#define EP_L4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT)
+#ifdef EP_STEP_WIDEQ
+#define EP_L5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "shr.u32 f" S ", " E S ", 21;\n\t"
+#else
+#define EP_L5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "mul.wide.u32 xw" S ", " E S ", m11;\n\t" "mov.b64 {bi" S ", f" S "}, xw" S ";\n\t"
+#endif
+#else
+#define EP_L1(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "and.b32 u" S ", " X ", 0x7FF;\n\t"
+#define EP_L2(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "mad.lo.u32 u" S ", u" S ", 4, tab" S ";\n\t"
+#define EP_L3(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "ld.shared.u32 " E S ", [u" S "+" OFF "];\n\t"
+#ifdef EP_Q_MULHI
+// x >> 11 as the high word of x * 2^21: on the multiply-add pipe, off the step's critical path
+#define EP_L4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "mul.hi.u32 q" S ", " X ", m21;\n\t"
+#else
+#define EP_L4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "shr.u32 q" S ", " X ", 11;\n\t"
+#endif
+#define EP_L5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "shr.u32 f" S ", " E S ", 21;\n\t"
+#endif
+#define EP_L6(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "and.b32 bi" S ", " E S ", 0x7FF;\n\t"
+#define EP_L7(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "@act" S " mad.lo.u32 " X ", f" S ", q" S ", bi" S ";\n\t"
+// renormalisation: lanes whose state fell below 2^15 take a word each, in lane order
+#define EP_L8(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "setp.lt.and.u32 p" S ", " X ", 32768, act" S ";\n\t"
+#define EP_L9(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "vote.sync.ballot.b32 " EP_B_##BOUT(S, BAL) ", p" S ", 0xffffffff;\n\t"
+#define EP_L10(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) \
+    "lop3.b32 t" S ", " EP_LT ", " EP_B_##BOUT(S, BAL) ", " EP_B_##BIN(S, BAL) ", 0xCA;\n\t"
+#define EP_L11(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "popc.b32 t" S ", t" S ";\n\t"
+#define EP_L12(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "mad.lo.u32 " AW ", t" S ", 2, " AW ";\n\t"
+#define EP_L13(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "ld.shared.u16 w" S ", [" AW "];\n\t"
+#define EP_L14(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT) "@p" S " mad.lo.u32 " X ", " X ", 65536, w" S ";\n\t"
+#define EP_RENORM_ALL(E, OFF, BIN, BOUT)                                                             \
+    EP_ALL(EP_L8, E, OFF, BIN, BOUT) EP_ALL(EP_L9, E, OFF, BIN, BOUT) EP_ALL(EP_L10, E, OFF, BIN, BOUT)  \
+    EP_ALL(EP_L11, E, OFF, BIN, BOUT) EP_ALL(EP_L12, E, OFF, BIN, BOUT) EP_ALL(EP_L13, E, OFF, BIN, BOUT) \
+    EP_ALL(EP_L14, E, OFF, BIN, BOUT)
+#define EP_STEP_ALL(E, OFF, BIN, BOUT)                                                               \
+    EP_ALL(EP_L1, E, OFF, BIN, BOUT) EP_ALL(EP_L2, E, OFF, BIN, BOUT) EP_ALL(EP_L3, E, OFF, BIN, BOUT)   \
+    EP_ALL(EP_L4, E, OFF, BIN, BOUT) EP_ALL(EP_L5, E, OFF, BIN, BOUT) EP_ALL(EP_L6, E, OFF, BIN, BOUT)   \
+    EP_ALL(EP_L7, E, OFF, BIN, BOUT) EP_RENORM_ALL(E, OFF, BIN, BOUT)
+// the coset: slot below f0 -> coset 0 with frequency f0, else coset 1 with frequency f1 and offset f0
+#define EP_C1(S, X, AW, BAL, DOFF, CB) "and.b32 u" S ", " X ", 0x7FF;\n\t"
+#define EP_C2(S, X, AW, BAL, DOFF, CB) "shr.u32 q" S ", " X ", 11;\n\t"
+#define EP_C3(S, X, AW, BAL, DOFF, CB) "setp.lt.u32 pc" S ", u" S ", " EP_F0 ";\n\t"
+#define EP_C4(S, X, AW, BAL, DOFF, CB) "selp.b32 f" S ", f0c, " EP_F1 ", pc" S ";\n\t"
+#define EP_C5(S, X, AW, BAL, DOFF, CB) "@!pc" S " sub.u32 u" S ", u" S ", " EP_F0 ";\n\t"
+#define EP_C6(S, X, AW, BAL, DOFF, CB) "@act" S " mad.lo.u32 " X ", f" S ", q" S ", u" S ";\n\t"
+#define EP_C7(S, X, AW, BAL, DOFF, CB) "selp.b32 tab" S ", " EP_LUT0 ", " EP_LUT1 ", pc" S ";\n\t"
+#define EP_C8(S, X, AW, BAL, DOFF, CB) "selp.b32 cc" S ", c0r, c1r, pc" S ";\n\t"
+#define EP_COSET_ALL                                                                                 \
+    EP_ALL(EP_C1) EP_ALL(EP_C2) EP_ALL(EP_C3) EP_ALL(EP_C4) EP_ALL(EP_C5) EP_ALL(EP_C6) EP_ALL(EP_C7) EP_ALL(EP_C8) \
+    EP_RENORM_ALL("", "", BL, NA)
+// Eq. 5 and the product of Eq. 19 for two neighbouring weights: 4096 + code (+ 1/2) as fp32, minus 4096 - zlo, times sigma
+#define EP_XA(S, X, AW, BAL, DOFF, CB, E) "lop3.b32 xa" S ", " E S ", " EP_CM ", cc" S ", 0xEA;\n\t"
+#define EP_XB(S, X, AW, BAL, DOFF, CB, E) "lop3.b32 xb" S ", " E S ", " EP_CM ", cc" S ", 0xEA;\n\t"
+#define EP_P1(S, X, AW, BAL, DOFF, CB) "mov.b64 pr" S ", {xa" S ", xb" S "};\n\t"
+#define EP_P2(S, X, AW, BAL, DOFF, CB) "sub.rn.f32x2 pr" S ", pr" S ", " EP_KK ";\n\t"
+#define EP_P3(S, X, AW, BAL, DOFF, CB) "mul.rn.f32x2 pr" S ", pr" S ", ss" S ";\n\t"
+#define EP_P4(S, X, AW, BAL, DOFF, CB) "mov.b64 {wl" S ", wh" S "}, pr" S ";\n\t"
+#ifdef EP_SCALAR_FP
+#undef EP_P1
+#undef EP_P2
+#undef EP_P3
+#undef EP_P4
+#define EP_P1(S, X, AW, BAL, DOFF, CB) "mov.b32 wl" S ", xa" S ";\n\t" "sub.rn.f32 wl" S ", wl" S ", k0f;\n\t"
+#define EP_P2(S, X, AW, BAL, DOFF, CB) "mov.b32 wh" S ", xb" S ";\n\t" "sub.rn.f32 wh" S ", wh" S ", k0f;\n\t"
+#define EP_P3(S, X, AW, BAL, DOFF, CB) "mul.rn.f32 wl" S ", wl" S ", sg" S ";\n\t"
+#define EP_P4(S, X, AW, BAL, DOFF, CB) "mul.rn.f32 wh" S ", wh" S ", sg" S ";\n\t"
+#endif
+#define EP_PAIR_ALL EP_ALL(EP_P1) EP_ALL(EP_P2) EP_ALL(EP_P3) EP_ALL(EP_P4)
+// parity of z1 + ... + z7 = xor of the codes' lowest bits (bit 11 of the entries; zlo is even): the lowest bit of z8
+#define EP_PAR3(S, X, AW, BAL, DOFF, CB, EA, EB, EC) "lop3.b32 par" S ", " EA S ", " EB S ", " EC S ", 0x96;\n\t"
+#define EP_PARX(S, X, AW, BAL, DOFF, CB) "lop3.b32 par" S ", par" S ", 0x800, cc" S ", 0xEA;\n\t"
+#define EP_X8(S, X, AW, BAL, DOFF, CB) "lop3.b32 xb" S ", e8" S ", " EP_CM ", par" S ", 0xEA;\n\t"
+#define EP_ADDR(S, X, AW, BAL, DOFF, CB) "mad.wide.u32 ad" S ", " DOFF ", 1, " EP_OUT ";\n\t"
 
-#define EP_S_STORE_BF16                                         \
-    "cvt.rn.bf16x2.f32 o0, w1, w0;\n\t"                         \
-    "cvt.rn.bf16x2.f32 o1, w3, w2;\n\t"                         \
-    "cvt.rn.bf16x2.f32 o2, w5, w4;\n\t"                         \
-    "cvt.rn.bf16x2.f32 o3, w7, w6;\n\t"                         \
-    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"
-#define EP_S_STORE_FP16                                         \
-    "cvt.rn.satfinite.f16x2.f32 o0, w1, w0;\n\t"                \
-    "cvt.rn.satfinite.f16x2.f32 o1, w3, w2;\n\t"                \
-    "cvt.rn.satfinite.f16x2.f32 o2, w5, w4;\n\t"                \
-    "cvt.rn.satfinite.f16x2.f32 o3, w7, w6;\n\t"                \
-    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"
-#define EP_S_STORE_E4M3                                         \
-    "cvt.rn.satfinite.e4m3x2.f32 h0, w1, w0;\n\t"               \
-    "cvt.rn.satfinite.e4m3x2.f32 h1, w3, w2;\n\t"               \
-    "cvt.rn.satfinite.e4m3x2.f32 h2, w5, w4;\n\t"               \
-    "cvt.rn.satfinite.e4m3x2.f32 h3, w7, w6;\n\t"               \
-    "mov.b32 o0, {h0, h1};\n\t"                                 \
-    "mov.b32 o1, {h2, h3};\n\t"                                 \
-    "st.global.v2.b32 [ad], {o0, o1};\n\t"
-#define EP_S_STORE_FP32                                         \
-    "mov.b32 o0, w0;\n\t"                                       \
-    "mov.b32 o1, w1;\n\t"                                       \
-    "mov.b32 o2, w2;\n\t"                                       \
-    "mov.b32 o3, w3;\n\t"                                       \
-    "st.global.v4.b32 [ad], {o0, o1, o2, o3};\n\t"              \
-    "mov.b32 o0, w4;\n\t"                                       \
-    "mov.b32 o1, w5;\n\t"                                       \
-    "mov.b32 o2, w6;\n\t"                                       \
-    "mov.b32 o3, w7;\n\t"                                       \
-    "st.global.v4.b32 [ad+16], {o0, o1, o2, o3};\n\t"
-#define EP_S_STORE_E5M2                                         \
-    "cvt.rn.satfinite.e5m2x2.f32 h0, w1, w0;\n\t"               \
-    "cvt.rn.satfinite.e5m2x2.f32 h1, w3, w2;\n\t"               \
-    "cvt.rn.satfinite.e5m2x2.f32 h2, w5, w4;\n\t"               \
-    "cvt.rn.satfinite.e5m2x2.f32 h3, w7, w6;\n\t"               \
-    "mov.b32 o0, {h0, h1};\n\t"                                 \
-    "mov.b32 o1, {h2, h3};\n\t"                                 \
-    "st.global.v2.b32 [ad], {o0, o1};\n\t"
+// per output type: CVT(S, j, lo, hi) turns weights 2j, 2j+1 into their stored form, STORE(S) writes the block
+#define EP_CVT_BF16(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.bf16x2.f32 o" J S ", wh" S ", wl" S ";\n\t"
+#define EP_CVT_FP16(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.satfinite.f16x2.f32 o" J S ", wh" S ", wl" S ";\n\t"
+#define EP_ST_16(S, X, AW, BAL, DOFF, CB) "@act" S " st.global.v4.b32 [ad" S "], {o0" S ", o1" S ", o2" S ", o3" S "};\n\t"
+#define EP_CVT_E4M3(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.satfinite.e4m3x2.f32 h" J S ", wh" S ", wl" S ";\n\t"
+#define EP_CVT_E5M2(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.satfinite.e5m2x2.f32 h" J S ", wh" S ", wl" S ";\n\t"
+#define EP_ST_F8(S, X, AW, BAL, DOFF, CB)                                                    \
+    "mov.b32 o0" S ", {h0" S ", h1" S "};\n\t"                           \
+    "mov.b32 o1" S ", {h2" S ", h3" S "};\n\t"                           \
+    "@act" S " st.global.v2.b32 [ad" S "], {o0" S ", o1" S "};\n\t"
+#define EP_CVT_FP32(S, X, AW, BAL, DOFF, CB, J) "mov.b32 ia" J S ", wl" S ";\n\t" "mov.b32 ib" J S ", wh" S ";\n\t"
+#define EP_ST_FP32(S, X, AW, BAL, DOFF, CB)                                                  \
+    "@act" S " st.global.v4.b32 [ad" S "], {ia0" S ", ib0" S ", ia1" S ", ib1" S "};\n\t" \
+    "@act" S " st.global.v4.b32 [ad" S "+16], {ia2" S ", ib2" S ", ia3" S ", ib3" S "};\n\t"
 /* one-byte integers: round to nearest even into s32 (out-of-range values end at INT_MIN / INT_MAX, NaN at 0), then
    saturate and pack four at a time: cvt.pack d, a, b, c gives (c << 16) | sat(a) << 8 | sat(b) */
-#define EP_S_STORE_UINT8                                        \
-    "cvt.rni.s32.f32 x1, w0;\n\t"                               \
-    "cvt.rni.s32.f32 x2, w1;\n\t"                               \
-    "cvt.rni.s32.f32 x3, w2;\n\t"                               \
-    "cvt.rni.s32.f32 x4, w3;\n\t"                               \
-    "cvt.rni.s32.f32 x5, w4;\n\t"                               \
-    "cvt.rni.s32.f32 x6, w5;\n\t"                               \
-    "cvt.rni.s32.f32 x7, w6;\n\t"                               \
-    "cvt.rni.s32.f32 x8, w7;\n\t"                               \
-    "cvt.pack.sat.u8.s32.b32 o2, x4, x3, 0;\n\t"                \
-    "cvt.pack.sat.u8.s32.b32 o0, x2, x1, o2;\n\t"               \
-    "cvt.pack.sat.u8.s32.b32 o3, x8, x7, 0;\n\t"                \
-    "cvt.pack.sat.u8.s32.b32 o1, x6, x5, o3;\n\t"               \
-    "st.global.v2.b32 [ad], {o0, o1};\n\t"
-#define EP_S_STORE_INT8                                         \
-    "cvt.rni.s32.f32 x1, w0;\n\t"                               \
-    "cvt.rni.s32.f32 x2, w1;\n\t"                               \
-    "cvt.rni.s32.f32 x3, w2;\n\t"                               \
-    "cvt.rni.s32.f32 x4, w3;\n\t"                               \
-    "cvt.rni.s32.f32 x5, w4;\n\t"                               \
-    "cvt.rni.s32.f32 x6, w5;\n\t"                               \
-    "cvt.rni.s32.f32 x7, w6;\n\t"                               \
-    "cvt.rni.s32.f32 x8, w7;\n\t"                               \
-    "cvt.pack.sat.s8.s32.b32 o2, x4, x3, 0;\n\t"                \
-    "cvt.pack.sat.s8.s32.b32 o0, x2, x1, o2;\n\t"               \
-    "cvt.pack.sat.s8.s32.b32 o3, x8, x7, 0;\n\t"                \
-    "cvt.pack.sat.s8.s32.b32 o1, x6, x5, o3;\n\t"               \
-    "st.global.v2.b32 [ad], {o0, o1};\n\t"
+#define EP_CVT_I8(S, X, AW, BAL, DOFF, CB, J) "cvt.rni.s32.f32 ia" J S ", wl" S ";\n\t" "cvt.rni.s32.f32 ib" J S ", wh" S ";\n\t"
+#define EP_ST_INT8(S, X, AW, BAL, DOFF, CB)                                                  \
+    "cvt.pack.sat.s8.s32.b32 o2" S ", ib1" S ", ia1" S ", 0;\n\t"        \
+    "cvt.pack.sat.s8.s32.b32 o0" S ", ib0" S ", ia0" S ", o2" S ";\n\t"  \
+    "cvt.pack.sat.s8.s32.b32 o3" S ", ib3" S ", ia3" S ", 0;\n\t"        \
+    "cvt.pack.sat.s8.s32.b32 o1" S ", ib2" S ", ia2" S ", o3" S ";\n\t"  \
+    "@act" S " st.global.v2.b32 [ad" S "], {o0" S ", o1" S "};\n\t"
+#define EP_ST_UINT8(S, X, AW, BAL, DOFF, CB)                                                 \
+    "cvt.pack.sat.u8.s32.b32 o2" S ", ib1" S ", ia1" S ", 0;\n\t"        \
+    "cvt.pack.sat.u8.s32.b32 o0" S ", ib0" S ", ia0" S ", o2" S ";\n\t"  \
+    "cvt.pack.sat.u8.s32.b32 o3" S ", ib3" S ", ia3" S ", 0;\n\t"        \
+    "cvt.pack.sat.u8.s32.b32 o1" S ", ib2" S ", ia2" S ", o3" S ";\n\t"  \
+    "@act" S " st.global.v2.b32 [ad" S "], {o0" S ", o1" S "};\n\t"
 
-#define EP_FULL_GROUPS_ASM(STORE, GROUP_BYTES)                                                                        \
+// registers of one chain
+#define EP_REGS(S, X, AW, BAL, DOFF, CB)                                                                             \
+    ".reg .pred p" S ", pc" S ", act" S ";\n\t"                                                                      \
+    ".reg .b32 u" S ", q" S ", f" S ", bi" S ", t" S ", w" S ", tab" S ", cc" S ", par" S ", na" S ", nb" S ";\n\t"  \
+    ".reg .b32 e1" S ", e2" S ", e3" S ", e4" S ", e5" S ", e6" S ", e7" S ", e8" S ", xa" S ", xb" S ";\n\t"        \
+    ".reg .b32 o0" S ", o1" S ", o2" S ", o3" S ", ia0" S ", ib0" S ", ia1" S ", ib1" S ", ia2" S ", ib2" S ", ia3" S ", ib3" S ";\n\t" \
+    ".reg .b16 h0" S ", h1" S ", h2" S ", h3" S ";\n\t"                                                              \
+    ".reg .f32 wl" S ", wh" S ", sg" S ";\n\t"                                                                       \
+    ".reg .b32 lim" S ", wthr" S ";\n\t"                                                                             \
+    ".reg .b64 pr" S ", ss" S ", ad" S ", xw" S ";\n\t"
+// before the first pass: the cursor leaves its first chunk at ring + 510; lim = 0 sends the chain through EP_ROWS
+#define EP_INIT(S, X, AW, BAL, DOFF, CB)                                 \
+    "ld.shared.u32 r0, [" EP_CTX "+" CB "+28];\n\t"                      \
+    "add.u32 wthr" S ", r0, 510;\n\t"                                    \
+    "mov.u32 lim" S ", 0;\n\t"
+
+#define EP_ADVANCE(S, X, AW, BAL, DOFF, CB, GROUP_BYTES) "add.u32 " DOFF ", " DOFF ", " GROUP_BYTES ";\n\t"
+// go on only if no lane of the chain left its chunk or reached its lim
+#define EP_CALM(S, X, AW, BAL, DOFF, CB)                                 \
+    "setp.lt.and.u32 pq, " AW ", wthr" S ", pq;\n\t"                     \
+    "setp.lt.and.u32 pq, " DOFF ", lim" S ", pq;\n\t"
+#define EP_CALM0(S, X, AW, BAL, DOFF, CB)                                \
+    "setp.lt.u32 pq, " AW ", wthr" S ";\n\t"                             \
+    "setp.lt.and.u32 pq, " DOFF ", lim" S ", pq;\n\t"
+#if EP_CHAINS == 1
+#define EP_CALM_ALL EP_CH_A(EP_CALM0)
+#elif EP_CHAINS == 2
+#define EP_CALM_ALL EP_CH_A(EP_CALM0) EP_CH_B(EP_CALM)
+#elif EP_CHAINS == 3
+#define EP_CALM_ALL EP_CH_A(EP_CALM0) EP_CH_B(EP_CALM) EP_CH_C(EP_CALM)
+#else
+#define EP_CALM_ALL EP_CH_A(EP_CALM0) EP_CH_B(EP_CALM) EP_CH_C(EP_CALM) EP_CH_D(EP_CALM)
+#endif
+
+// some lane of the chain reached its lim (also run once on entry): where is each lane now?
+// CB = byte offset of the chain's part of the context block.  row = doff / bytes per row by a multiply-high
+// with ceil(2^32 / bytes per row), which is at most one too large.
+#define EP_ROWS(S, X, AW, BAL, DOFF, CB)                                 \
+    "setp.ge.u32 pr, " DOFF ", lim" S ";\n\t"                                                                  \
+    "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                               \
+    "@!pr bra.uni EP_ROWS_END_" S ";\n\t"                                                                      \
+    "ld.shared.v2.u32 {r0, r1}, [" EP_CTX "+8];\n\t"    /* bytes per row, last row */                          \
+    "ld.shared.u32 r2, [" EP_CTX "+" CB "+24];\n\t"     /* offset after the tile's last block */               \
+    "ld.shared.u32 r5, [" EP_CTX "+24];\n\t"                                                                   \
+    "mul.hi.u32 r3, " DOFF ", r5;\n\t"                                                                         \
+    "mul.lo.u32 r4, r3, r0;\n\t"                                                                               \
+    "setp.gt.u32 pv, r4, " DOFF ";\n\t"                                                                        \
+    "@pv sub.u32 r3, r3, 1;\n\t"                                                                               \
+    "mad.lo.u32 r4, r3, r0, r0;\n\t"                    /* offset at which this lane enters the next row */    \
+    "min.u32 lim" S ", r4, r2;\n\t"                                                                            \
+    "setp.lt.u32 act" S ", " DOFF ", r2;\n\t"                                                                  \
+    "@!act" S " mov.u32 lim" S ", 0xffffffff;\n\t"      /* a lane without a block never asks again */          \
+    "min.u32 r3, r3, r1;\n\t"                                                                                  \
+    "ld.shared.u64 ra, [" EP_CTX "];\n\t"                                                                      \
+    "mul.wide.u32 rb, r3, 4;\n\t"                                                                              \
+    "add.s64 ra, ra, rb;\n\t"                                                                                  \
+    "ld.global.nc.b32 r4, [ra];\n\t"                                                                           \
+    "mov.b64 ss" S ", {r4, r4};\n\t"                                                                           \
+    "mov.b32 sg" S ", r4;\n\t"                                                                                 \
+    "EP_ROWS_END_" S ":\n\t"
+#define EP_ANY_ACT(S, X, AW, BAL, DOFF, CB) "or.pred pr, pr, act" S ";\n\t"
+
+// the chain's cursor left its chunk: request the chunks up to two ahead of it (one, as a rule), wait for all but
+// the newest, move the addresses back by the ring's length when the cursor's chunk is the one in slot 0 again.
+// The chain's context is read with two 16-byte loads up front: one shared-memory round trip, not six.
+#define EP_SERVICE(S, X, AW, BAL, DOFF, CB)                              \
+    "setp.ge.u32 pr, " AW ", wthr" S ";\n\t"                                                                   \
+    "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                               \
+    "@!pr bra.uni EP_SVC_END_" S ";\n\t"                                                                       \
+    "ld.shared.v4.u32 {r4, r5, r2, r10}, [" EP_CTX "+" CB "+16];\n\t" /* next slot, wbase, -, ring base */    \
+    "ld.shared.v4.u32 {r11, r12, r1, r9}, [" EP_CTX "+" CB "];\n\t"   /* chunk 0 address, room, next chunk */ \
+    "shfl.sync.idx.b32 r6, " AW ", 0, 31, 0xffffffff;\n\t"                                                     \
+    "popc.b32 r0, " BAL ";\n\t"                                                                                \
+    "mad.lo.u32 r6, r0, 2, r6;\n\t"                     /* the cursor's address */                             \
+    "sub.u32 r7, r6, r5;\n\t"                           /* its byte position */                                \
+    "shr.u32 r8, r7, 9;\n\t"                            /* its chunk */                                        \
+    "add.u32 r0, r8, 3;\n\t"                                                                                   \
+    "sub.s32 r0, r0, r9;\n\t"                           /* chunks the cursor has advanced: requests due */     \
+    "min.s32 r0, r0, 3;\n\t"                                                                                   \
+    "max.s32 r0, r0, 0;\n\t"                                                                                   \
+    "shl.b32 r8, r0, 9;\n\t"                            /* bytes the cursor's chunk moves on in the ring */    \
+    "setp.eq.u32 pq, r0, 0;\n\t"                                                                               \
+    "@pq bra.uni EP_SVW_" S ";\n\t"                                                                            \
+    "mov.b64 ra, {r11, r12};\n\t"                                                                              \
+    "EP_SVL_" S ":\n\t"                                                                                        \
+    "shl.b32 r2, r9, 9;\n\t"                                                                                   \
+    "add.u32 r2, r2, " EP_L16 ";\n\t"                   /* this lane's 16 bytes of the chunk */                \
+    "sub.s32 r3, r1, r2;\n\t"                                                                                  \
+    "min.s32 r3, r3, 16;\n\t"                                                                                  \
+    "max.s32 r3, r3, 0;\n\t"                            /* bytes of them inside the payload */                 \
+    "setp.gt.s32 pv, r3, 0;\n\t"                                                                               \
+    "selp.b32 r2, r2, 0, pv;\n\t"                                                                              \
+    "mad.wide.u32 rb, r2, 1, ra;\n\t"                                                                          \
+    "mad.lo.u32 r2, r4, 512, r10;\n\t"                                                                         \
+    "add.u32 r2, r2, " EP_L16 ";\n\t"                                                                          \
+    "cp.async.cg.shared.global [r2], [rb], 16, r3;\n\t"                                                        \
+    "setp.eq.u32 pv, r4, 0;\n\t"                                                                               \
+    "@pv cp.async.cg.shared.global [r2+1536], [rb], 16, r3;\n\t"                                               \
+    "cp.async.commit_group;\n\t"                                                                               \
+    "add.u32 r9, r9, 1;\n\t"                                                                                   \
+    "add.u32 r4, r4, 1;\n\t"                                                                                   \
+    "setp.eq.u32 pv, r4, 3;\n\t"                                                                               \
+    "selp.b32 r4, 0, r4, pv;\n\t"                                                                              \
+    "sub.u32 r0, r0, 1;\n\t"                                                                                   \
+    "setp.ne.u32 pq, r0, 0;\n\t"                                                                               \
+    "@pq bra.uni EP_SVL_" S ";\n\t"                                                                            \
+    "st.shared.u32 [" EP_CTX "+" CB "+12], r9;\n\t"                                                            \
+    "st.shared.u32 [" EP_CTX "+" CB "+16], r4;\n\t"                                                            \
+    "EP_SVW_" S ":\n\t"                                                                                        \
+    "cp.async.wait_group 1;\n\t"                                                                               \
+    "bar.warp.sync 0xffffffff;\n\t"                                                                            \
+    "sub.u32 r2, wthr" S ", r10;\n\t"                   /* 510 + ring offset of the cursor's old chunk */      \
+    "add.u32 r2, r2, r8;\n\t"                                                                                  \
+    "setp.ge.u32 pv, r2, 2046;\n\t"                     /* past the third slot: back to the first */           \
+    "@pv sub.u32 r2, r2, 1536;\n\t"                                                                            \
+    "add.u32 wthr" S ", r2, r10;\n\t"                                                                          \
+    "and.b32 r3, r7, 511;\n\t"                                                                                 \
+    "add.u32 r2, wthr" S ", r3;\n\t"                                                                           \
+    "sub.u32 r2, r2, 510;\n\t"                          /* the cursor's new address */                         \
+    "sub.u32 r3, r6, r2;\n\t"                                                                                  \
+    "sub.u32 " AW ", " AW ", r3;\n\t"                                                                          \
+    "sub.u32 r5, r5, r3;\n\t"                                                                                  \
+    "st.shared.u32 [" EP_CTX "+" CB "+20], r5;\n\t"                                                            \
+    "EP_SVC_END_" S ":\n\t"
+
+#if EP_CHAINS == 1
+#define EP_LOOP_OPERANDS                                                                                              \
+        : "+&r"(x[0]), "+&r"(a[0]), "+&r"(bal[0]), "+&r"(doff[0])
+#elif EP_CHAINS == 2
+#define EP_LOOP_OPERANDS                                                                                              \
+        : "+&r"(x[0]), "+&r"(a[0]), "+&r"(bal[0]), "+&r"(doff[0]), "+&r"(x[1]), "+&r"(a[1]), "+&r"(bal[1]), "+&r"(doff[1])
+#elif EP_CHAINS == 3
+#define EP_LOOP_OPERANDS                                                                                              \
+        : "+&r"(x[0]), "+&r"(a[0]), "+&r"(bal[0]), "+&r"(doff[0]), "+&r"(x[1]), "+&r"(a[1]), "+&r"(bal[1]), "+&r"(doff[1]), \
+          "+&r"(x[2]), "+&r"(a[2]), "+&r"(bal[2]), "+&r"(doff[2])
+#else
+#define EP_LOOP_OPERANDS                                                                                              \
+        : "+&r"(x[0]), "+&r"(a[0]), "+&r"(bal[0]), "+&r"(doff[0]), "+&r"(x[1]), "+&r"(a[1]), "+&r"(bal[1]), "+&r"(doff[1]), \
+          "+&r"(x[2]), "+&r"(a[2]), "+&r"(bal[2]), "+&r"(doff[2]), "+&r"(x[3]), "+&r"(a[3]), "+&r"(bal[3]), "+&r"(doff[3])
+#endif
+
+#define EP_TILES_LOOP_ASM(CVT, STORE, GROUP_BYTES)                                                                    \
     asm volatile(                                                                                                     \
         "{\n\t"                                                                                                       \
-        ".reg .pred p, ps, pw, pa, pl, pq, pr, pv, pm;\n\t"                                                           \
-        ".reg .b32 u, f, q, bias, bal, t, w, coff, tab, kc, par, pos, cur, clim, n, slot, d, mlim;\n\t"               \
-        ".reg .b32 e0, e1, e2, e3, e4, e5, e6, e7, e8, x1, x2, x3, x4, x5, x6, x7, x8, o0, o1, o2, o3;\n\t"           \
-        ".reg .b16 h0, h1, h2, h3;\n\t"                                                                               \
-        ".reg .f32 w0, w1, w2, w3, w4, w5, w6, w7;\n\t"                                                               \
-        ".reg .b64 kk, ss, p0, p1, p2, p3, ad, src;\n\t"                                                              \
-        "setp.ge.u32 pl, %7, %23;\n\t"                                                                                \
-        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"                                                                  \
-        "@pl bra.uni EP_DONE;\n\t"                                                                                    \
+        EP_ALL(EP_REGS)                                                                                               \
+        ".reg .pred pq, pv, pr;\n\t"                                                                                  \
+        ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, f0c, m21, m11;\n\t"               \
+        ".reg .b64 ra, rb;\n\t"                                                                                       \
+        ".reg .f32 k0f, k1f;\n\t"                                                                                     \
+        "mov.b64 {k0f, k1f}, " EP_KK ";\n\t"                                                                          \
+        "mov.b32 c0r, 0x45800000;\n\t"                                                                                \
+        "mov.b32 c1r, 0x45800400;\n\t"                                                                                \
+        "max.u32 f0c, " EP_F0 ", 1;\n\t"                /* frequency used for coset 0: never 0 */                     \
+        "ld.shared.v2.u32 {m21, m11}, [" EP_CTX "+16];\n\t" /* 2^21, 2^11 */                                          \
+        EP_ALL(EP_INIT)                                                                                               \
+        "bra.uni EP_RARE;\n\t"                                                                                        \
         "EP_LOOP:\n\t"                                                                                                \
-        EP_S_STEP("e0", "%15", "131072")                                                                              \
-        "and.b32 coff, e0, 0x1FF800;\n\t"                                                                              \
-        "add.u32 tab, %15, coff;\n\t"                                                                                 \
-        EP_S_STEP("e1", "tab", "0")                                                                                   \
-        EP_S_STEP("e2", "tab", "8192")                                                                                \
-        EP_S_STEP("e3", "tab", "16384")                                                                               \
-        EP_S_STEP("e4", "tab", "24576")                                                                               \
-        EP_S_STEP("e5", "tab", "32768")                                                                               \
-        EP_S_STEP("e6", "tab", "40960")                                                                               \
-        EP_S_STEP("e7", "tab", "49152")                                                                               \
-        EP_S_STEP("e8", "tab", "57344")                                                                               \
-        /* Eq. 5: 4096 + code as fp32, minus kc = 4096 - zlo - c/2 (one ulp = 2^-11, c/2 = 1024 ulps) */              \
-        "shr.u32 t, coff, 6;\n\t"                                                                                     \
-        "sub.u32 kc, %18, t;\n\t"                                                                                     \
-        "lop3.b32 x1, e1, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x2, e2, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x3, e3, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x4, e4, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x5, e5, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x6, e6, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x7, e7, 0x1FF800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 par, e1, e2, e3, 0x96;\n\t"                                                                         \
-        "lop3.b32 par, par, e4, e5, 0x96;\n\t"                                                                        \
-        "lop3.b32 par, par, e6, e7, 0x96;\n\t"                                                                        \
-        "lop3.b32 par, par, 0x800, 0x45800000, 0xEA;\n\t"                                                             \
-        "lop3.b32 x8, e8, 0x1FF800, par, 0xEA;\n\t"                                                                    \
-        "mov.b64 kk, {kc, kc};\n\t"                                                                                   \
-        "mov.b64 ss, {%6, %6};\n\t"                                                                                   \
-        EP_S_PAIR("p0", "x1", "x2", "w0", "w1")                                                                       \
-        EP_S_PAIR("p1", "x3", "x4", "w2", "w3")                                                                       \
-        EP_S_PAIR("p2", "x5", "x6", "w4", "w5")                                                                       \
-        EP_S_PAIR("p3", "x7", "x8", "w6", "w7")                                                                       \
-        "cvt.u64.u32 ad, %7;\n\t"                                                                                     \
-        "add.s64 ad, ad, %19;\n\t"                                                                                    \
-        STORE                                                                                                         \
-        "add.u32 %7, %7, " #GROUP_BYTES ";\n\t"                                                                       \
-        /* one vote for everything rare: go on only if no lane crossed a chunk boundary or reached its lim */        \
-        "setp.lt.u32 ps, %1, %2;\n\t"                                                                                 \
-        "setp.lt.and.u32 pq, %7, %8, ps;\n\t"                                                                         \
-        "vote.sync.all.pred pq, pq, 0xffffffff;\n\t"   /* a vote result is uniform to the compiler as well */         \
+        EP_COSET_ALL                                                                                                  \
+        EP_STEP_ALL("e1", "0", NA, NB)     EP_ALL(EP_XA, "e1")                                                        \
+        EP_STEP_ALL("e2", "8192", NB, NA)  EP_ALL(EP_XB, "e2") EP_PAIR_ALL EP_ALL(CVT, "0")                           \
+        EP_STEP_ALL("e3", "16384", NA, NB) EP_ALL(EP_PAR3, "e1", "e2", "e3") EP_ALL(EP_XA, "e3")                      \
+        EP_STEP_ALL("e4", "24576", NB, NA) EP_ALL(EP_XB, "e4") EP_PAIR_ALL EP_ALL(CVT, "1")                           \
+        EP_STEP_ALL("e5", "32768", NA, NB) EP_ALL(EP_PAR3, "par", "e4", "e5") EP_ALL(EP_XA, "e5")                     \
+        EP_STEP_ALL("e6", "40960", NB, NA) EP_ALL(EP_XB, "e6") EP_PAIR_ALL EP_ALL(CVT, "2")                           \
+        EP_STEP_ALL("e7", "49152", NA, NB) EP_ALL(EP_PAR3, "par", "e6", "e7") EP_ALL(EP_XA, "e7")                     \
+        EP_STEP_ALL("e8", "57344", NB, BL) EP_ALL(EP_PARX) EP_ALL(EP_X8) EP_PAIR_ALL EP_ALL(CVT, "3")                 \
+        EP_ALL(EP_ADDR) EP_ALL(STORE)                                                                                \
+        EP_ALL(EP_ADVANCE, #GROUP_BYTES)                                                                              \
+        /* one vote for everything rare */                                                                            \
+        EP_CALM_ALL                                                                                                   \
+        "vote.sync.all.pred pq, pq, 0xffffffff;\n\t"                                                                  \
         "@pq bra.uni EP_LOOP;\n\t"                                                                                    \
-        "setp.ge.u32 pr, %7, %8;\n\t"                                                                                 \
+        "EP_RARE:\n\t"                                                                                                \
+        EP_ALL(EP_ROWS)                                                                                               \
+        "setp.lt.u32 pr, " EP_LT ", 0;\n\t"          /* false */                                                                                   \
+        EP_ALL(EP_ANY_ACT)                                                                                            \
         "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                                  \
-        "@!pr bra.uni EP_SVCCHK;\n\t"                                                                                 \
-        /* ---- some lane moved to the next row (reload its scale), or the tile's full groups are done ---- */        \
-        "setp.ge.u32 pw, %7, %4;\n\t"                                                                                 \
-        "@pw add.u32 %4, %4, %17;\n\t"                                                                                \
-        "@pw add.u32 %5, %5, 1;\n\t"                                                                                  \
-        "min.u32 t, %5, %22;\n\t"                                                                                     \
-        "mul.wide.u32 ad, t, 4;\n\t"                                                                                  \
-        "add.s64 ad, ad, %20;\n\t"                                                                                    \
-        "@pw ld.global.nc.b32 %6, [ad];\n\t"                                                                          \
-        "min.u32 %8, %4, %23;\n\t"                                                                                    \
-        "setp.ge.u32 pl, %7, %23;\n\t"                                                                                \
-        "vote.sync.any.pred pl, pl, 0xffffffff;\n\t"                                                                  \
-        "@pl bra.uni EP_DONE;\n\t"                                                                                    \
-        "EP_SVCCHK:\n\t"                                                                                              \
-        "setp.ge.u32 ps, %1, %2;\n\t"                                                                                 \
-        "vote.sync.any.pred ps, ps, 0xffffffff;\n\t"                                                                  \
-        "@!ps bra.uni EP_LOOP;\n\t"                                                                                   \
-        /* ---- the cursor entered a new 512-byte chunk: request chunks up to cur+3, wait for all but the newest */   \
-        "sub.u32 pos, %1, %3;\n\t"                                                                                    \
-        "shr.u32 cur, pos, 9;\n\t"                                                                                    \
-        "add.u32 clim, cur, 4;\n\t"                                                                                   \
-        "sub.u32 t, %24, %16;\n\t"                     /* 16 * lane */                                                \
-        "setp.lt.u32 pm, t, 128;\n\t"                                                                                 \
-        "selp.u32 mlim, 2, 1, pm;\n\t"                 /* slot 0 is mirrored whole, slot 1 by lanes 0..7 */           \
-        "EP_SVC_LOOP:\n\t"                                                                                            \
-        "setp.ge.u32 pq, %11, clim;\n\t"                                                                              \
-        "vote.sync.any.pred pq, pq, 0xffffffff;\n\t"                                                                  \
-        "@pq bra.uni EP_SVC_DONE;\n\t"                                                                                \
-        "min.s32 n, %10, 16;\n\t"                                                                                     \
-        "max.s32 n, n, 0;\n\t"                                                                                        \
-        "setp.gt.s32 pv, %10, 0;\n\t"                                                                                 \
-        "selp.b64 src, %9, %21, pv;\n\t"                                                                              \
-        "and.b32 slot, %11, 3;\n\t"                                                                                   \
-        "mad.lo.u32 d, slot, 512, %24;\n\t"                                                                           \
-        "cp.async.cg.shared.global [d], [src], 16, n;\n\t"                                                            \
-        "setp.lt.u32 pm, slot, mlim;\n\t"                                                                             \
-        "@pm cp.async.cg.shared.global [d+2048], [src], 16, n;\n\t"                                                   \
-        "cp.async.commit_group;\n\t"                                                                                  \
-        "add.s64 %9, %9, 512;\n\t"                                                                                    \
-        "sub.s32 %10, %10, 512;\n\t"                                                                                  \
-        "add.u32 %11, %11, 1;\n\t"                                                                                    \
-        "bra.uni EP_SVC_LOOP;\n\t"                                                                                    \
-        "EP_SVC_DONE:\n\t"                                                                                            \
-        "cp.async.wait_group 1;\n\t"                                                                                  \
-        "bar.warp.sync 0xffffffff;\n\t"                                                                               \
-        "and.b32 t, pos, 2047;\n\t"                                                                                   \
-        "add.u32 %1, %16, t;\n\t"                                                                                     \
-        "sub.u32 %3, %1, pos;\n\t"                                                                                    \
-        "shl.b32 t, cur, 9;\n\t"                                                                                      \
-        "add.u32 t, t, 512;\n\t"                                                                                      \
-        "add.u32 %2, %3, t;\n\t"                                                                                      \
+        "@!pr bra.uni EP_DONE;\n\t"                                                                                   \
+        EP_ALL(EP_SERVICE)                                                                                            \
         "bra.uni EP_LOOP;\n\t"                                                                                        \
         "EP_DONE:\n\t"                                                                                                \
         "}"                                                                                                           \
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
-        : "+&r"(x), "+&r"(wa), "+&r"(wthr), "+&r"(wbase), "+&r"(chg), "+&r"(row), "+&r"(sig), "+&r"(doff),            \
-          "+&r"(lim), "+&l"(srcp), "+&r"(rem), "+&r"(nextc)                                                           \
-        : "r"(lt), "r"(mask), "r"(b), "r"(lut_addr), "r"(ring), "r"(row_bytes), "r"(k0_bits), "l"(out_base),         \
-          "l"(scales), "l"(a0), "r"(row_max), "r"(endo), "r"(ring_lane)                                               \
+        EP_LOOP_OPERANDS                                                                                              \
+        : "r"(lt), "r"(lut_addr), "r"(lut_addr + kCosetStride), "r"(ctx), "l"(kk), "l"(out_base), "r"(cf.f0),         \
+          "r"(cf.f1), "r"(lane16)                                                                                     \
         : "memory")
 
-// One tile of a tensor whose rows hold at least 32 blocks: the full groups in PTX, a last partial group
-// through decode_group.  `valid` is false for a warp whose slot lies past the last tile (`tile` is then
-// the last tile, only so that addresses stay inside the stream): it does no group at all.  The number of
-// groups is data here, not control flow the compiler reasons about: every branch on it is a bra.uni.
+// kChains tiles of a tensor whose rows hold at least 32 blocks and whose tables have 2^11 slots; chain c takes tile
+// `first + c`.  A chain whose slot lies past the job's last tile gets that last tile's record, only so that its
+// addresses stay inside the stream, and no block at all.  The number of groups is data here, not control flow the
+// compiler reasons about: every branch on it is a bra.uni on a warp vote.
+// `tables_pending`: the job's lookup tables are still being written (by this CTA's own stores or copies): the
+// tiles' records and first payload chunks are requested first, the CTA barrier comes after.
 template <int DT>
-__device__ __forceinline__ void decode_tile_fast(const JobParams &J, uint32_t tile, bool valid, uint32_t lut_addr,
-                                                 uint32_t ring, uint32_t lane) {
-    const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
-    uint32_t x = rec[lane];
-    const uint32_t off = min(rec[32], J.total_words);   // a damaged index must not move reads outside the payload
-    const uint32_t end = (tile + 1 < J.n_tiles) ? rec[33 + 32] : rec[33];
-    const uint32_t v0 = tile * J.V;
-    const uint32_t nv = valid ? min(J.V, J.n_vec - v0) : 0u;
-    const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
-    const uint32_t per_row = J.per_row;
-    const uint64_t pay = reinterpret_cast<uint64_t>(J.stream + J.off_payload);
-    const uint64_t first = pay + 2ull * off;
-    const uint64_t a0 = first & ~15ull;
-    const uint32_t lead = uint32_t(first - a0);
-    const uint32_t room = uint32_t(pay + 2ull * J.total_words - a0);     // the payload is shorter than 2 GB
-    const uint32_t lane16 = 16u * lane;
-    for (uint32_t c = 0; c < 4; ++c) ring_issue(ring, a0, room, c, lane);
-    cp_async_wait<1>();
-    __syncwarp();
-    uint32_t wa = ring + lead;                    // cursor
-    uint32_t wbase = ring;                        // wa - position
-    uint32_t wthr = ring + 512u;                  // next chunk boundary
-    uint64_t srcp = a0 + 2048u + lane16;          // this lane's part of chunk 4
-    uint32_t rem = room - (2048u + lane16);       // signed in the asm: may be negative
-    uint32_t nextc = 4;
-    const uint32_t ring_lane = ring + lane16;
-    const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
-    const uint32_t v = v0 + lane;
-    uint32_t row = v / per_row;
-    const float *scales = J.scales;
-    uint32_t sig = __float_as_uint(__ldg(scales + row));
-    uint32_t doff = v * Out<DT>::kBlockBytes;
-    const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
-    // The loop runs on byte offsets into the output: this lane leaves its row when doff reaches chg and the tile's
-    // full groups are done when it reaches endo.  The group count is the same in all lanes but comes from loaded
-    // data, which the compiler treats as possibly different per lane; the loop therefore branches on warp votes of
-    // these comparisons (see the asm), never on the values themselves.  nv >> 5 may be 0: the asm falls through.
-    const uint32_t row_bytes = per_row * Out<DT>::kBlockBytes;
-    uint32_t chg = (row + 1u) * row_bytes;
-    const uint32_t endo = doff + (nv >> 5) * (32u * Out<DT>::kBlockBytes);
-    uint32_t lim = min(chg, endo);
-    const uint32_t row_max = J.n_vec / per_row - 1u;   // the wrap after a tensor's last block must not read past the scales
-    if constexpr (DT == EP_BF16) EP_FULL_GROUPS_ASM(EP_S_STORE_BF16, 512);
-    else if constexpr (DT == EP_FP16) EP_FULL_GROUPS_ASM(EP_S_STORE_FP16, 512);
-    else if constexpr (DT == EP_FP8_E4M3) EP_FULL_GROUPS_ASM(EP_S_STORE_E4M3, 256);
-    else if constexpr (DT == EP_FP32) EP_FULL_GROUPS_ASM(EP_S_STORE_FP32, 1024);
-    else if constexpr (DT == EP_FP8_E5M2) EP_FULL_GROUPS_ASM(EP_S_STORE_E5M2, 256);
-    else if constexpr (DT == EP_UINT8) EP_FULL_GROUPS_ASM(EP_S_STORE_UINT8, 256);
-    else EP_FULL_GROUPS_ASM(EP_S_STORE_INT8, 256);
-    uint32_t pos = wa - wbase;
-    if (nv & 31u) {
-        uint32_t threshold = wthr - wbase;
-        // chunks up to (threshold >> 9) + 2 are requested: the same bookkeeping as ring_service expects
-        if (__any_sync(0xFFFFFFFFu, pos >= threshold)) ring_service(ring, a0, room, pos, threshold, lane);
-        const uint32_t wa0 = ring + (pos & (kRingBytes - 1u));
-        uint32_t wt = wa0;
-        const bool act = lane < (nv & 31u);
-        decode_group<DT, true>(x, wt, lut_addr, mask, b, lt, act, k0_bits, __uint_as_float(sig), J.zlo,
-                               static_cast<uint8_t *>(J.out) + doff);
-        pos += wt - wa0;
+__device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t first, uint32_t lut_addr, CosetFreq cf,
+                                                  uint32_t ring, uint32_t ctx, uint32_t lane, bool tables_pending) {
+    constexpr uint32_t BB = Out<DT>::kBlockBytes;
+    const uint32_t lt = (1u << lane) - 1u, lane16 = 16u * lane;
+    uint32_t x[kChains], a[kChains], bal[kChains], doff[kChains], off[kChains], end[kChains], lead[kChains];
+    bool valid[kChains];
+#pragma unroll
+    for (uint32_t c = 0; c < kChains; ++c) {
+        valid[c] = first + c < J.tile_cnt;
+        const uint32_t tile = J.tile0 + min(first + c, J.tile_cnt - 1u);
+        const uint32_t rg = ring + c * kRingStride, cctx = ctx + kCtxChain + c * kCtxChainStride;
+        const TileSetup T = tile_setup(J, tile, valid[c], lane);
+        for (uint32_t k = 0; k < kRingSlots; ++k) ring_issue(rg, T.a0, T.room, k, lane);
+        if (lane == 0) {
+            sts64(cctx + kCcA0, T.a0);
+            sts32(cctx + kCcRoom, T.room);
+            sts32(cctx + kCcNext, kRingSlots);
+            sts32(cctx + kCcNextSlot, 0u);
+            sts32(cctx + kCcWbase, rg);
+            sts32(cctx + kCcEndo, (T.v0 + T.nv) * BB);
+            sts32(cctx + kCcRing, rg);
+        }
+        x[c] = T.x; a[c] = rg + T.lead; bal[c] = 0; doff[c] = (T.v0 + lane) * BB;
+        off[c] = T.off; end[c] = T.end; lead[c] = T.lead;
     }
-    cp_async_wait<0>();
+    cp_async_wait<1>();           // all but the last chain's third chunk have landed (and the table image, if any)
     __syncwarp();
-    const bool bad = valid && ((x != ep::kStateLow) || (off + ((pos - lead) >> 1) != end));
+    if (tables_pending) __syncthreads();
+    const uint32_t k0 = __float_as_uint(float(4096 - J.zlo));
+    const uint64_t kk = pack64(k0, k0);
+    const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
+    if constexpr (DT == EP_BF16) EP_TILES_LOOP_ASM(EP_CVT_BF16, EP_ST_16, 512);
+    else if constexpr (DT == EP_FP16) EP_TILES_LOOP_ASM(EP_CVT_FP16, EP_ST_16, 512);
+    else if constexpr (DT == EP_FP8_E4M3) EP_TILES_LOOP_ASM(EP_CVT_E4M3, EP_ST_F8, 256);
+    else if constexpr (DT == EP_FP8_E5M2) EP_TILES_LOOP_ASM(EP_CVT_E5M2, EP_ST_F8, 256);
+    else if constexpr (DT == EP_FP32) EP_TILES_LOOP_ASM(EP_CVT_FP32, EP_ST_FP32, 1024);
+    else if constexpr (DT == EP_UINT8) EP_TILES_LOOP_ASM(EP_CVT_I8, EP_ST_UINT8, 256);
+    else EP_TILES_LOOP_ASM(EP_CVT_I8, EP_ST_INT8, 256);
+    cp_async_wait<0>();           // nothing may still be landing in the rings when the next tiles start
+    __syncwarp();
+    // integrity: the encoder started every state at 2^15 and a tile's words end where the next tile's begin
+    bool bad = false;
+#pragma unroll
+    for (uint32_t c = 0; c < kChains; ++c) {
+        const uint32_t cur = __shfl_sync(0xFFFFFFFFu, a[c], 0) + 2u * __popc(bal[c]) -
+                             lds32(ctx + kCtxChain + c * kCtxChainStride + kCcWbase);
+        bad |= valid[c] && ((x[c] != ep::kStateLow) || (off[c] + ((cur - lead[c]) >> 1) != end[c]));
+    }
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
+    __syncwarp();                 // the context block is rewritten by the next tiles
 }
 
 // One persistent CTA per SM.  The rounds of all jobs of the launch form one list (job after job); CTA k takes the
 // rounds whose cumulative cost at their start lies in [k, k + 1) * ceil(total / gridDim.x) - a contiguous stretch,
-// usually inside one job - and rebuilds the lookup tables when the stretch crosses into the next job.  Everything
+// usually inside one job - and sets the lookup tables up again when the stretch crosses into the next job.  Everything
 // that steers this (loop bounds, job changes) depends on blockIdx and kernel parameters only, so the compiler
 // sees warp-uniform control flow and puts no divergence guards around the warp votes of the hot loop; in the last
-// round of a job a warp past the job's last tile goes through the same code with zero groups to do.
-// SINGLE: the launch has one job (the common single-tensor call); its parameters then sit at fixed offsets of
-// the parameter block and the job loop disappears.
-template <int DT, bool SINGLE>
+// round of a job a chain past the job's last tile goes through the same code with no block to decode.
+template <int DT>
 __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __grid_constant__ BatchParams P) {
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
-    const uint32_t ring = lut_addr + kLutBytes + warp * kRingStride;
+    const uint32_t ring = lut_addr + kRingBase + warp * (kChains * kRingStride);
+    const uint32_t ctx = lut_addr + kCtxBase + warp * kCtxBytes;
     bool tables_in_use = false;
-    const int n_jobs = SINGLE ? 1 : P.n_jobs;
-    for (int j = 0; j < n_jobs; ++j) {
-        const JobParams &J = P.job[SINGLE ? 0 : j];
+    for (int j = 0; j < P.n_jobs; ++j) {
+        const JobParams &J = P.job[j];
         // rounds r of this job with cost_begin + r * round_cost in [lo, hi), this CTA's share of the total cost
         // (recomputed per job rather than kept in registers across the decode loops)
         const uint32_t lo = P.cost_per_cta * blockIdx.x, hi = lo + P.cost_per_cta;      // below 2^31 (see the launcher)
@@ -789,33 +976,46 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
         const uint32_t r0 = min((a + J.round_cost - 1u) / J.round_cost, J.rounds);
         const uint32_t r1 = min((b + J.round_cost - 1u) / J.round_cost, J.rounds);
         if (r0 >= r1) continue;
-        {   // while the tables are built, bring this warp's first tile record and the start of its payload into L2
-            const uint32_t t_first = J.tile0 + min(r0 * kWarps + warp, J.tile_cnt - 1u);
+        {   // while the tables are set up, bring this warp's first tile records and the start of their payload into L2
+            const uint32_t t_first = J.tile0 + min(r0 * kTilesPerRound + kChains * warp, J.tile_cnt - 1u);
             const uint32_t *rec = J.tile_index + size_t(t_first) * 33u;
-            if (lane < 2) prefetch_l2(rec + 32u * lane);                     // the record spans two 128-byte lines
+            if (lane < kChains + 1u) prefetch_l2(rec + 32u * lane);          // the warp's records span kChains + 1 lines
             const uint32_t off = min(rec[32], J.total_words);
-            const uint64_t at = 2ull * off + 128u * lane;                      // 4 KB: the ring's first fill and more
+            const uint64_t at = 2ull * off + 128u * lane;                      // 4 KB: the rings' first fill and more
             if (at < 2ull * J.total_words) prefetch_l2(J.stream + J.off_payload + at);
         }
         if (tables_in_use) __syncthreads();          // every warp is done with the previous job's tables
-        build_tables_smem(J, lut_addr, warp, lane);
-        __syncthreads();
+        if (J.lut_image) copy_tables_smem(J.lut_image, lut_addr);
+        else build_tables_smem(J, lut_addr, warp, lane);
+        const CosetFreq cf = load_coset(J);
+        bool tables_pending = true;
         tables_in_use = true;
-        const bool wide = J.per_row >= 32u;
+        const bool fast = DT != EP_FIELDS_I32 && J.per_row >= 32u && J.b == 11u && J.V < (1u << 20);
+        if (fast && lane == 0) {                     // what the hot loop's rare paths need to know about the job
+            sts64(ctx + kCtxScales, reinterpret_cast<uint64_t>(J.scales));
+            sts32(ctx + kCtxRowBytes, J.row_bytes);
+            sts32(ctx + kCtxRowMax, J.row_max);      // the step after a tensor's last block must not read past the scales
+            sts32(ctx + kCtxMul21, 1u << 21);
+            sts32(ctx + kCtxMul11, 1u << 11);
+            sts32(ctx + kCtxRowRcp, J.row_rcp);
+        }
+        __syncwarp();
         for (uint32_t r = r0; r < r1; ++r) {
-            const uint32_t base = r * kWarps;
-            const bool mine = base + warp < J.tile_cnt;
-            const uint32_t tile = J.tile0 + min(base + warp, J.tile_cnt - 1u);
+            const uint32_t base = r * kTilesPerRound + kChains * warp;
             if constexpr (DT != EP_FIELDS_I32) {
-                if (wide && J.V < (1u << 20)) {
-                    decode_tile_fast<DT>(J, tile, mine, lut_addr, ring, lane);
+                if (fast) {
+                    decode_tiles_fast<DT>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    tables_pending = false;
                     continue;
                 }
             }
-            if (mine) {
-                if (wide) decode_tile<DT, true>(J, tile, lut_addr, ring, lane);
-                else decode_tile<DT, false>(J, tile, lut_addr, ring, lane);
+            if (tables_pending) {
+                cp_async_wait<0>();
+                __syncthreads();
+                tables_pending = false;
             }
+            for (uint32_t c = 0; c < kChains; ++c)
+                if (base + c < J.tile_cnt) decode_tile_plain<DT>(J, J.tile0 + base + c, lut_addr, cf, ring, lane);
         }
     }
 }
@@ -845,6 +1045,10 @@ struct GJobParams {
     uint32_t V, n_tiles, b;
     uint32_t tile0, tile_cnt;     // the tiles this launch decodes
     uint32_t cta_begin, cta_count;
+    // table geometry from the host's ep_info, never from the device copy of the directory
+    int32_t tmin[EP_NUM_TABLES];
+    uint16_t tK[EP_NUM_TABLES];
+    uint32_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
 };
 
 struct GBatchParams {
@@ -856,19 +1060,21 @@ constexpr int kGThreads = 256;
 constexpr int kGWarps = kGThreads / 32;
 
 // one CTA per (table, job): exclusive prefix sums of the frequencies in shared memory (as u16; the last
-// entry 2^b <= 32768 still fits), then every slot finds its symbol by binary search
+// entry 2^b <= 32768 still fits), then every slot finds its symbol by binary search.  A table without symbols
+// (or whose frequencies fall short of 2^b in a damaged stream) gets index 0 with offset 0 in the slots nobody owns.
 __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_constant__ GBatchParams P) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint32_t part[1024];
     const GJobParams &J = P.job[blockIdx.y];
     const uint32_t t = blockIdx.x, tid = threadIdx.x;
-    const uint8_t *dir = J.stream + J.off_tables;
-    const uint32_t *Ks = reinterpret_cast<const uint32_t *>(dir) + EP_NUM_TABLES;
-    const uint32_t K = Ks[t];
-    if (K == 0) return;
-    uint32_t before = 0;
-    for (uint32_t i = 0; i < t; ++i) before += Ks[i];
-    const uint16_t *fq = reinterpret_cast<const uint16_t *>(dir + 8 * EP_NUM_TABLES) + before;
+    const uint32_t K = J.tK[t];
+    const uint32_t M = 1u << J.b;
+    uint32_t *lut = J.lut + (size_t(t) << J.b);
+    if (K == 0) {
+        for (uint32_t u = tid; u < M; u += blockDim.x) lut[u] = 0u;
+        return;
+    }
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_tables + 8 * EP_NUM_TABLES) + J.foff[t];
     uint16_t *F = reinterpret_cast<uint16_t *>(smem);              // K + 1 entries
     const uint32_t per = (K + blockDim.x - 1) / blockDim.x;
     const uint32_t j0 = min(tid * per, K), j1 = min(j0 + per, K);
@@ -879,33 +1085,31 @@ __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_cons
     if (tid == 0) {
         uint32_t run = 0;
         for (uint32_t i = 0; i < blockDim.x; ++i) { const uint32_t v = part[i]; part[i] = run; run += v; }
-        F[K] = uint16_t(run);                                        // = 2^b for a valid stream
+        F[K] = uint16_t(min(run, M));                                // = 2^b for a valid stream
     }
     __syncthreads();
     uint32_t run = part[tid];
-    for (uint32_t j = j0; j < j1; ++j) { F[j] = uint16_t(run); run += fq[j]; }
+    for (uint32_t j = j0; j < j1; ++j) { F[j] = uint16_t(min(run, M)); run += fq[j]; }
     __syncthreads();
-    const uint32_t M = 1u << J.b;
-    uint32_t *lut = J.lut + (size_t(t) << J.b);
     for (uint32_t u = tid; u < M; u += blockDim.x) {
-        uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u; F[K] = 2^b > u
+        uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u (F[0] = 0)
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
             if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
         }
-        lut[u] = (lo << 16) | (u - uint32_t(F[lo]));                 // K <= 65535 and u - F < 2^15
+        lut[u] = (lo << 16) | ((u - uint32_t(F[lo])) & 0xFFFFu);     // lo < K <= 65535
     }
 }
 
-// one symbol: returns its index inside table t's symbol range (0 for an idle lane)
-__device__ __forceinline__ uint32_t grans_step(uint32_t &x, const uint32_t *table, const uint16_t *freq, uint32_t mask,
-                                               uint32_t b, uint32_t &ptr, const uint16_t *pay, uint32_t lt, bool act,
-                                               uint32_t last_word) {
+// one symbol: returns its index inside table t's symbol range (0 for an idle lane); Kmax = the table's last index
+__device__ __forceinline__ uint32_t grans_step(uint32_t &x, const uint32_t *table, const uint16_t *freq, uint32_t Kmax,
+                                               uint32_t mask, uint32_t b, uint32_t &ptr, const uint16_t *pay, uint32_t lt,
+                                               bool act, uint32_t last_word) {
     uint32_t sym = 0;
     bool need = false;
     if (act) {
         const uint32_t e = __ldg(table + (x & mask));
-        sym = e >> 16;
+        sym = min(e >> 16, Kmax);                 // whatever the scratch holds, stay inside the frequency array
         x = uint32_t(__ldg(freq + sym)) * (x >> b) + (e & 0xFFFFu);
         need = x < ep::kStateLow;
     }
@@ -917,29 +1121,16 @@ __device__ __forceinline__ uint32_t grans_step(uint32_t &x, const uint32_t *tabl
 
 template <int DT>
 __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_constant__ GBatchParams P) {
-    __shared__ uint32_t s_foff[EP_NUM_TABLES];     // start of table t's frequencies, in u16 units
-    __shared__ int32_t s_tmin[EP_NUM_TABLES];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     int j = 0;
     while (j + 1 < P.n_jobs && blockIdx.x >= P.job[j + 1].cta_begin) ++j;
     const GJobParams &J = P.job[j];
-    const uint8_t *dir = J.stream + J.off_tables;
-    if (threadIdx.x == 0) {
-        const uint32_t *Ks = reinterpret_cast<const uint32_t *>(dir) + EP_NUM_TABLES;
-        uint32_t acc = 0;
-        for (int t = 0; t < EP_NUM_TABLES; ++t) {
-            s_foff[t] = acc;
-            s_tmin[t] = reinterpret_cast<const int32_t *>(dir)[t];
-            acc += Ks[t];
-        }
-    }
-    __syncthreads();
-    const uint16_t *fq = reinterpret_cast<const uint16_t *>(dir + 8 * EP_NUM_TABLES);
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_tables + 8 * EP_NUM_TABLES);
     const uint32_t b = J.b, mask = (1u << b) - 1u, lt = (1u << lane) - 1u;
     const uint16_t *pay = reinterpret_cast<const uint16_t *>(J.stream + J.off_payload);
     const uint32_t last_word = J.total_words ? J.total_words - 1u : 0u;
     const uint32_t cta = blockIdx.x - J.cta_begin;
-    const uint32_t foff0 = s_foff[0];
+    const uint32_t K0max = J.tK[0] ? J.tK[0] - 1u : 0u;
     for (uint32_t local = cta * kGWarps + warp; local < J.tile_cnt; local += J.cta_count * kGWarps) {
         const uint32_t tile = J.tile0 + local;
         const uint32_t *rec = J.tile_index + size_t(tile) * 33u;
@@ -952,12 +1143,15 @@ __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_
             const uint32_t i = g * 32u + lane;
             const bool act = i < nv;
             int32_t fld[9];
-            fld[0] = int32_t(grans_step(x, J.lut, fq + foff0, mask, b, ptr, pay, lt, act, last_word)) + s_tmin[0];
+            fld[0] = int32_t(grans_step(x, J.lut, fq + J.foff[0], K0max, mask, b, ptr, pay, lt, act, last_word)) + J.tmin[0];
             const uint32_t t0 = 1u + 8u * uint32_t(fld[0] & 1);          // first coordinate table of this coset
 #pragma unroll
-            for (uint32_t k = 0; k < 8; ++k)
-                fld[k + 1] = int32_t(grans_step(x, J.lut + (size_t(t0 + k) << b), fq + s_foff[t0 + k], mask, b, ptr, pay, lt,
-                                                act, last_word)) + s_tmin[t0 + k];
+            for (uint32_t k = 0; k < 8; ++k) {
+                const uint32_t t = t0 + k;
+                const uint32_t Kt = J.tK[t];
+                fld[k + 1] = int32_t(grans_step(x, J.lut + (size_t(t) << b), fq + J.foff[t], Kt ? Kt - 1u : 0u, mask, b, ptr, pay,
+                                                lt, act && Kt != 0u, last_word)) + J.tmin[t];
+            }
             if (!act) continue;
             const uint32_t v = v0 + i;
             if constexpr (DT == EP_FIELDS_I32) {
@@ -983,22 +1177,33 @@ __global__ void __launch_bounds__(kGThreads) ep_decode_glut_kernel(const __grid_
     }
 }
 
+// a prepared image of the sixteen shared-memory tables in global memory (ep_prepare_tables): warp w of the
+// job's CTA builds table w + 1 with the routine the decode kernel uses on shared memory
+__global__ void __launch_bounds__(512) ep_prepare_tables_kernel(const __grid_constant__ JobParams J, uint32_t *image) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t t = 1u + warp;
+    if (t >= EP_NUM_TABLES) return;
+    uint32_t *dst = image + (t - 1u) * kLutEntries;
+    build_one_table(J, t, lane, [dst](uint32_t slot, uint32_t e) { dst[slot] = e; });
+    // b < 11: the slots above 2^b are never read, but the image is copied whole
+    for (uint32_t u = (1u << J.b) + lane; u < kLutEntries; u += 32) dst[u] = kEntryUnused;
+}
+
 // ---- host side -----------------------------------------------------------------------------------
 
 // the tiles a job asks for: its range, or the whole tensor when both range fields are 0
 inline uint32_t job_tile0(const ep_decode_job &jb) { return jb.tile_count ? jb.tile_begin : 0u; }
 inline uint32_t job_tiles(const ep_decode_job &jb) { return jb.tile_count ? jb.tile_count : jb.info->n_tiles; }
 
-int g_num_sms = 0;
+int g_num_sms[64] = {};
 
 int num_sms() {
-    if (g_num_sms == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        g_num_sms = n;
-    }
-    return g_num_sms;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64 && g_num_sms[dev]) return g_num_sms[dev];
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (dev >= 0 && dev < 64) g_num_sms[dev] = n;
+    return n;
 }
 
 struct Range { int64_t lo, hi; bool any; };
@@ -1029,12 +1234,26 @@ bool fits_smem_tables(const ep_info &I) {
     const Range r = coord_range(I);
     const int64_t zlo = even_base(r);
     if (r.any && r.hi - zlo > 1023) return false;     // 10-bit code field
-    if (zlo < -1024) return false;                    // 4096 - zlo - c/2 stays below 8192: same fp32 exponent as 4096 + code
-    for (int t = 0; t < EP_NUM_TABLES; ++t) {
+    if (zlo < -1024) return false;                    // 4096 - zlo stays below 8192: same fp32 exponent as 4096 + code
+    for (int t = 1; t < EP_NUM_TABLES; ++t) {         // (the coset table is decoded by comparison: any frequency goes)
         if (I.table_K[t] > kLutEntries) return false;
         if (I.b == 11 && I.table_K[t] == 1) return false;   // a lone symbol has f = 2^11: one bit more than the f field
     }
     return true;
+}
+
+// table geometry of a job whose tables fit shared memory
+void fill_table_params(JobParams &J, const ep_info &I) {
+    J.off_freq = I.off_tables + 8u * EP_NUM_TABLES;
+    J.b = I.b;
+    J.zlo = int32_t(even_base(coord_range(I)));
+    uint32_t acc = 0;
+    for (int t = 0; t < EP_NUM_TABLES; ++t) {
+        J.tmin[t] = int16_t(I.table_min[t]);
+        J.tK[t] = uint16_t(I.table_K[t]);
+        J.foff[t] = uint16_t(acc);
+        acc += I.table_K[t];
+    }
 }
 
 template <int DT>
@@ -1044,14 +1263,54 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
+        e = cudaFuncSetAttribute(ep_decode_smem_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kSmemBytes));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    if (P.n_jobs == 1) ep_decode_smem_kernel<DT, true><<<grid, kThreads, kSmemBytes, st>>>(P);
-    else ep_decode_smem_kernel<DT, false><<<grid, kThreads, kSmemBytes, st>>>(P);
+    ep_decode_smem_kernel<DT><<<grid, kThreads, kSmemBytes, st>>>(P);
+    return cudaGetLastError();
+}
+
+size_t large_table_bytes(const ep_info &I) { return size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 4u; }
+
+// the host-side parameters of a large-table job (geometry from `info` only); `lut` = where its tables are or go
+int fill_large_job(GJobParams &J, const ep_decode_job &jb, uint32_t *lut) {
+    const ep_info &I = *jb.info;
+    uint32_t acc = 0;
+    for (int t = 0; t < EP_NUM_TABLES; ++t) {
+        if (I.table_K[t] > 65535u) return EP_ERR_UNSUPPORTED;
+        J.tmin[t] = I.table_min[t];
+        J.tK[t] = uint16_t(I.table_K[t]);
+        J.foff[t] = acc;
+        acc += I.table_K[t];
+    }
+    J.stream = static_cast<const uint8_t *>(jb.d_stream);
+    J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
+    J.scales = jb.d_row_scales;
+    J.out = jb.d_out;
+    J.lut = lut;
+    J.off_tables = I.off_tables;
+    J.off_payload = I.off_payload;
+    J.total_words = uint32_t(I.total_words);
+    J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
+    J.per_row = I.C / 8;
+    J.V = I.V;
+    J.n_tiles = I.n_tiles;
+    J.b = I.b;
+    return EP_OK;
+}
+
+cudaError_t launch_build(const GBatchParams &P, int n_jobs, cudaStream_t st) {
+    uint32_t max_K = 1;
+    for (int i = 0; i < n_jobs; ++i)
+        for (int t = 0; t < EP_NUM_TABLES; ++t)
+            if (P.job[i].tK[t] > max_K) max_K = P.job[i].tK[t];
+    const size_t smem = 2u * (size_t(max_K) + 1u);
+    if (smem > 48u * 1024u) {
+        const cudaError_t e = cudaFuncSetAttribute(ep_build_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+    }
+    ep_build_tables_kernel<<<dim3(EP_NUM_TABLES, n_jobs), 1024, smem, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -1060,7 +1319,40 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
 extern "C" size_t ep_decode_scratch_bytes(const ep_info *info) {
     if (!info) return 0;
     if (fits_smem_tables(*info)) return 0;
-    return size_t(EP_NUM_TABLES) * (size_t(1) << info->b) * 4u;
+    return large_table_bytes(*info);
+}
+
+extern "C" size_t ep_decode_tables_bytes(const ep_info *info) {
+    if (!info) return 0;
+    return fits_smem_tables(*info) ? size_t(kLutBytes) : large_table_bytes(*info);
+}
+
+extern "C" uint32_t ep_decode_tiles_per_sm(void) { return kTilesPerRound; }
+
+extern "C" int ep_prepare_tables(const ep_info *info, const void *d_stream, void *d_tables, size_t tables_bytes, void *stream) {
+    if (!info || !d_stream || !d_tables) return EP_ERR_BAD_ARG;
+    const ep_info &I = *info;
+    if (I.b < 9 || I.b > 15 || (reinterpret_cast<uintptr_t>(d_stream) & 3)) return EP_ERR_BAD_ARG;
+    if (tables_bytes < ep_decode_tables_bytes(info) || (reinterpret_cast<uintptr_t>(d_tables) & 255)) return EP_ERR_SCRATCH;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (fits_smem_tables(I)) {
+        JobParams J;
+        std::memset(&J, 0, sizeof(J));
+        J.stream = static_cast<const uint8_t *>(d_stream);
+        fill_table_params(J, I);
+        ep_prepare_tables_kernel<<<1, 512, 0, st>>>(J, static_cast<uint32_t *>(d_tables));
+        return cudaGetLastError() == cudaSuccess ? EP_OK : EP_ERR_CUDA;
+    }
+    GBatchParams P;
+    std::memset(&P, 0, sizeof(P));
+    P.n_jobs = 1;
+    ep_decode_job jb;
+    std::memset(&jb, 0, sizeof(jb));
+    jb.info = info;
+    jb.d_stream = d_stream;
+    const int rc = fill_large_job(P.job[0], jb, static_cast<uint32_t *>(d_tables));
+    if (rc) return rc;
+    return launch_build(P, 1, st) == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
 namespace {
@@ -1071,35 +1363,30 @@ cudaError_t launch_glut(const GBatchParams &P, uint32_t grid, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-// jobs whose tables do not fit shared memory: build the tables into scratch, then decode from them
+// jobs whose tables do not fit shared memory: decode from tables in global memory - the caller's prepared
+// ones, or tables built into the caller's scratch by one extra launch first
 int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt, int sms, cudaStream_t st) {
-    GBatchParams P;
+    GBatchParams P, B;      // B: the jobs whose tables have to be built
     std::memset(&P, 0, sizeof(P));
+    std::memset(&B, 0, sizeof(B));
     P.n_jobs = n_jobs;
-    uint32_t next = 0, max_K = 1;
+    uint32_t next = 0;
+    int n_build = 0;
     for (int i = 0; i < n_jobs; ++i) {
         const ep_decode_job &jb = *jobs[i];
         const ep_info &I = *jb.info;
-        const size_t need = size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 4u;
-        if (!jb.d_scratch || jb.scratch_bytes < need || (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255)) return EP_ERR_SCRATCH;
-        for (int t = 0; t < EP_NUM_TABLES; ++t) {
-            if (I.table_K[t] > 65535u) return EP_ERR_UNSUPPORTED;
-            if (I.table_K[t] > max_K) max_K = I.table_K[t];
+        const size_t need = large_table_bytes(I);
+        uint32_t *lut;
+        if (jb.d_tables) {
+            if (reinterpret_cast<uintptr_t>(jb.d_tables) & 255) return EP_ERR_SCRATCH;
+            lut = static_cast<uint32_t *>(const_cast<void *>(jb.d_tables));
+        } else {
+            if (!jb.d_scratch || jb.scratch_bytes < need || (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255)) return EP_ERR_SCRATCH;
+            lut = static_cast<uint32_t *>(jb.d_scratch);
         }
         GJobParams &J = P.job[i];
-        J.stream = static_cast<const uint8_t *>(jb.d_stream);
-        J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
-        J.scales = jb.d_row_scales;
-        J.out = jb.d_out;
-        J.lut = static_cast<uint32_t *>(jb.d_scratch);
-        J.off_tables = I.off_tables;
-        J.off_payload = I.off_payload;
-        J.total_words = uint32_t(I.total_words);
-        J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
-        J.per_row = I.C / 8;
-        J.V = I.V;
-        J.n_tiles = I.n_tiles;
-        J.b = I.b;
+        const int rc = fill_large_job(J, jb, lut);
+        if (rc) return rc;
         J.tile0 = job_tile0(jb);
         J.tile_cnt = job_tiles(jb);
         const uint64_t want = (uint64_t(J.tile_cnt) + kGWarps - 1) / kGWarps;
@@ -1107,16 +1394,12 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
         J.cta_begin = next;
         J.cta_count = uint32_t(want < cap ? want : cap);
         next += J.cta_count;
+        if (!jb.d_tables) B.job[n_build++] = J;
     }
-    const size_t smem = 2u * (size_t(max_K) + 1u);
-    if (smem > 48u * 1024u) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
-        if (cudaFuncSetAttribute(ep_build_tables_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-            return EP_ERR_CUDA;
+    if (n_build) {
+        B.n_jobs = n_build;
+        if (launch_build(B, n_build, st) != cudaSuccess) return EP_ERR_CUDA;
     }
-    ep_build_tables_kernel<<<dim3(EP_NUM_TABLES, n_jobs), 1024, smem, st>>>(P);
-    if (cudaGetLastError() != cudaSuccess) return EP_ERR_CUDA;
     cudaError_t e;
     switch (dt) {
     case EP_BF16: e = launch_glut<EP_BF16>(P, next, st); break;
@@ -1183,11 +1466,12 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         const ep_info &I = *jb.info;
         JobParams &J = P.job[i];
         const uint32_t my_tiles = job_tiles(jb);
+        if (jb.d_tables && (reinterpret_cast<uintptr_t>(jb.d_tables) & 255)) return EP_ERR_SCRATCH;
         J.stream = static_cast<const uint8_t *>(jb.d_stream);
         J.tile_index = static_cast<const uint32_t *>(jb.d_tile_index);
         J.scales = jb.d_row_scales;
         J.out = jb.d_out;
-        J.off_freq = I.off_tables + 8u * EP_NUM_TABLES;
+        J.lut_image = static_cast<const uint32_t *>(jb.d_tables);
         J.off_payload = I.off_payload;
         J.total_words = uint32_t(I.total_words);
         J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
@@ -1196,20 +1480,16 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.n_tiles = I.n_tiles;
         J.tile0 = job_tile0(jb);
         J.tile_cnt = my_tiles;
-        J.b = I.b;
-        J.zlo = int32_t(even_base(coord_range(I)));
-        J.rounds = (my_tiles + uint32_t(kWarps) - 1u) / uint32_t(kWarps);
+        fill_table_params(J, I);
+        const uint32_t block_bytes = dt == EP_FIELDS_I32 ? 36u : dt == EP_FP32 ? 32u : (dt == EP_BF16 || dt == EP_FP16) ? 16u : 8u;
+        J.row_bytes = J.per_row * block_bytes;
+        J.row_rcp = uint32_t(0xFFFFFFFFu / J.row_bytes + 1u);
+        J.row_max = I.R - 1u;
+        J.rounds = (my_tiles + kTilesPerRound - 1u) / kTilesPerRound;
         J.round_cost = (I.V + 31u) / 32u;
         J.cost_begin = uint32_t(cost);
         cost += uint64_t(J.rounds) * J.round_cost;
         rounds_total += J.rounds;
-        uint32_t acc = 0;
-        for (int t = 0; t < EP_NUM_TABLES; ++t) {
-            J.tmin[t] = int16_t(I.table_min[t]);
-            J.tK[t] = uint16_t(I.table_K[t]);
-            J.foff[t] = uint16_t(acc);
-            acc += I.table_K[t];
-        }
     }
     const uint32_t next = uint32_t(rounds_total < uint64_t(sms) ? rounds_total : uint64_t(sms));   // grid size
     // a tensor has under 2^27 blocks, so sixteen of them cost under 2^26 groups: 32-bit arithmetic in the kernel
@@ -1230,11 +1510,11 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     return e == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
-extern "C" int ep_decode_tiles(const ep_info *info, const void *d_stream, const void *d_tile_index,
-                               const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
-                               size_t scratch_bytes, uint32_t tile_begin, uint32_t tile_count, void *stream) {
-    if (tile_count == 0) return EP_ERR_BAD_ARG;
+namespace {
+ep_decode_job one_job(const ep_info *info, const void *d_stream, const void *d_tile_index, const float *d_row_scales,
+                      int32_t out_dtype, void *d_out, void *d_scratch, size_t scratch_bytes) {
     ep_decode_job jb;
+    std::memset(&jb, 0, sizeof(jb));
     jb.info = info;
     jb.d_stream = d_stream;
     jb.d_tile_index = d_tile_index;
@@ -1243,6 +1523,15 @@ extern "C" int ep_decode_tiles(const ep_info *info, const void *d_stream, const 
     jb.d_out = d_out;
     jb.d_scratch = d_scratch;
     jb.scratch_bytes = scratch_bytes;
+    return jb;
+}
+}  // namespace
+
+extern "C" int ep_decode_tiles(const ep_info *info, const void *d_stream, const void *d_tile_index,
+                               const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
+                               size_t scratch_bytes, uint32_t tile_begin, uint32_t tile_count, void *stream) {
+    if (tile_count == 0) return EP_ERR_BAD_ARG;
+    ep_decode_job jb = one_job(info, d_stream, d_tile_index, d_row_scales, out_dtype, d_out, d_scratch, scratch_bytes);
     jb.tile_begin = tile_begin;
     jb.tile_count = tile_count;
     return ep_decode_batch(&jb, 1, stream);
@@ -1251,17 +1540,7 @@ extern "C" int ep_decode_tiles(const ep_info *info, const void *d_stream, const 
 extern "C" int ep_decode_tensor(const ep_info *info, const void *d_stream, const void *d_tile_index,
                                 const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
                                 size_t scratch_bytes, void *stream) {
-    ep_decode_job jb;
-    jb.info = info;
-    jb.d_stream = d_stream;
-    jb.d_tile_index = d_tile_index;
-    jb.d_row_scales = d_row_scales;
-    jb.out_dtype = out_dtype;
-    jb.d_out = d_out;
-    jb.d_scratch = d_scratch;
-    jb.scratch_bytes = scratch_bytes;
-    jb.tile_begin = 0;
-    jb.tile_count = 0;
+    const ep_decode_job jb = one_job(info, d_stream, d_tile_index, d_row_scales, out_dtype, d_out, d_scratch, scratch_bytes);
     return ep_decode_batch(&jb, 1, stream);
 }
 

@@ -104,7 +104,6 @@ extern "C" const char *ep_strerror(int status) {
     case EP_ERR_BAD_STREAM: return "malformed or inconsistent compressed stream";
     case EP_ERR_UNSUPPORTED: return "unsupported request";
     case EP_ERR_CUDA: return "CUDA runtime error";
-    case EP_ERR_TIMEOUT: return "device-side wait timed out";
     case EP_ERR_NOMEM: return "out of host memory";
     case EP_ERR_SCRATCH: return "scratch buffer missing, misaligned or too small";
     case EP_ERR_STATIC_LIMIT: return "stream needs lookup tables larger than the built-in area (b above EP_STATIC_MAX_B)";
@@ -142,7 +141,7 @@ extern "C" uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint3
                                                   uint32_t decode_ctas) {
     const uint32_t vmax = ep_default_tile_vectors(target_bpp);
     if (!R || !C || n == 0 || decode_ctas == 0) return vmax;
-    // One launch decodes all n tensors: a CTA takes 32 tiles per round, the rounds of all tensors are split evenly
+    // One launch decodes all n tensors: a CTA takes 48 tiles per round, the rounds of all tensors are split evenly
     // over the CTAs, so the launch lasts ceil(rounds / CTAs) rounds of ceil(V / 32) groups each (plus a small
     // fixed cost per round: tile set-up and the last, partly idle steps).  Take the multiple of 32 that makes this
     // shortest; on ties the larger tile (less metadata).  Never below a quarter of the paper's default.
@@ -154,7 +153,7 @@ extern "C" uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint3
         for (uint32_t i = 0; i < n; ++i) {
             const uint64_t nvec = uint64_t(R[i]) * (C[i] / 8u);
             const uint64_t tiles = (nvec + V - 1u) / V;
-            rounds += (tiles + 31u) / 32u;
+            rounds += (tiles + ep::kDecodeTilesPerCta - 1u) / ep::kDecodeTilesPerCta;
         }
         const uint64_t cost = ((rounds + decode_ctas - 1u) / decode_ctas) * (V / 32u + 2u);
         if (cost <= best_cost) { best_cost = cost; best_v = V; }

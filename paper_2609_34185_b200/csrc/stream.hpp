@@ -13,6 +13,10 @@ constexpr uint32_t kHeaderBytes = 64;
 constexpr uint32_t kStates = 32;          // J
 constexpr uint32_t kTileRecordBytes = 4 * kStates + 4;
 constexpr uint32_t kStateLow = 1u << 15;  // states live in [2^15, 2^31)
+#ifndef EP_TILES_PER_CTA
+#define EP_TILES_PER_CTA 32
+#endif
+constexpr uint32_t kDecodeTilesPerCta = EP_TILES_PER_CTA;  // tiles one CTA of the decode kernel works on at a time (one per warp)
 
 template <class T>
 inline T load_le(const uint8_t *p) {

@@ -26,19 +26,19 @@ def _bits(t: torch.Tensor) -> np.ndarray:
 
 
 def _check_all_types(blob_bytes, scales=None):
-    d = ep.upload(blob_bytes)
     sc_dev = None if scales is None else torch.from_numpy(scales).cuda()
-    ref_fields = None
-    for dt, odt in ORACLE_DT.items():
-        got = ep.decode(d, dt, row_scales=sc_dev)
-        ref, ref_fields = oracle.decode(blob_bytes, odt, scales=scales, want_fields=True)
-        torch.cuda.synchronize()
-        if dt == ep.FP32:
-            ref = ref.view(np.uint32)
-        assert np.array_equal(_bits(got), ref), f"dtype {dt}"
-    f = ep.decode(d, ep.FIELDS_I32)
-    assert np.array_equal(f.cpu().numpy(), ref_fields)
-    assert ep.last_device_status() == 0
+    ref = {odt: oracle.decode(blob_bytes, odt, scales=scales, want_fields=True) for odt in ORACLE_DT.values()}
+    # lookup tables prepared once at upload (ep_prepare_tables), and derived inside every decode call
+    for prepare in (True, False):
+        d = ep.upload(blob_bytes, prepare=prepare)
+        for dt, odt in ORACLE_DT.items():
+            got = ep.decode(d, dt, row_scales=sc_dev)
+            torch.cuda.synchronize()
+            want = ref[odt][0].view(np.uint32) if dt == ep.FP32 else ref[odt][0]
+            assert np.array_equal(_bits(got), want), f"dtype {dt}, prepared tables {prepare}"
+        f = ep.decode(d, ep.FIELDS_I32)
+        assert np.array_equal(f.cpu().numpy(), ref[oracle.BF16][1]), f"fields, prepared tables {prepare}"
+        assert ep.last_device_status() == 0
 
 
 def test_config1_all_types_both_directions():
@@ -215,16 +215,27 @@ def test_coordinate_range_up_to_1024_stays_on_the_shared_memory_path():
     _check_all_types(blob.data)
 
 
-def test_single_symbol_table_at_b11_takes_the_large_table_path():
-    # a lone symbol has frequency 2^11, one bit more than the shared-memory entry's frequency field
+def test_single_symbol_tables_at_b11():
     rng = np.random.default_rng(5)
     n = 4 * 64
     fields = np.zeros((n, 9), np.int32)                      # coset always 0: the coset table has one symbol
     fields[:, 1:] = np.rint(rng.standard_normal((n, 8)) * 3).astype(np.int32)
+    # the coset is decoded by comparing the slot with the frequency of coset 0: a lone coset (f = 2^11) needs no table
     blob = ep.pack_fields(fields, 4, 512, 11, 40, np.full(4, 0.02, np.float32))
-    assert blob.info.table_K[0] == 1 and ep.decode_scratch_bytes(blob.info) > 0
+    assert blob.info.table_K[0] == 1 and ep.decode_scratch_bytes(blob.info) == 0
     _check_all_types(blob.data)
-    blob10 = ep.pack_fields(fields, 4, 512, 10, 40, np.full(4, 0.02, np.float32))
+    only1 = fields.copy()
+    only1[:, 0] = 1                                          # coset always 1
+    blob = ep.pack_fields(only1, 4, 512, 11, 40, np.full(4, 0.02, np.float32))
+    assert blob.info.table_K[0] == 1 and blob.info.table_min[0] == 1 and ep.decode_scratch_bytes(blob.info) == 0
+    _check_all_types(blob.data)
+    # a lone coordinate symbol has frequency 2^11, one bit more than the shared-memory entry's frequency field
+    lone = fields.copy()
+    lone[:, 3] = 2
+    blob = ep.pack_fields(lone, 4, 512, 11, 40, np.full(4, 0.02, np.float32))
+    assert blob.info.table_K[3] == 1 and ep.decode_scratch_bytes(blob.info) > 0
+    _check_all_types(blob.data)
+    blob10 = ep.pack_fields(lone, 4, 512, 10, 40, np.full(4, 0.02, np.float32))
     assert ep.decode_scratch_bytes(blob10.info) == 0        # f = 2^10 fits
     _check_all_types(blob10.data)
 
@@ -286,7 +297,7 @@ def test_config3_one_wide_tensor_fp8_and_int8_containers():
 
 
 def test_config4_with_the_tile_size_the_bench_uses():
-    V = ep.suggest_tile_vectors(8192, 8192, 4.0, 32 * torch.cuda.get_device_properties(0).multi_processor_count)
+    V = ep.suggest_tile_vectors(8192, 8192, 4.0, ep.decode_tiles_per_sm() * torch.cuda.get_device_properties(0).multi_processor_count)
     blob = _full_compare(synth.config4(), 4.0, ep.FP16, V)
     assert blob.info.V == V
 
@@ -349,7 +360,9 @@ def test_tile_ranges_tile_the_tensor_and_write_nothing_else():
                 assert np.array_equal(got, part[first * 8 * es:last * 8 * es])
                 pieces.append(got)
             assert np.array_equal(np.concatenate(pieces), ref)
-        # in place in a full-size buffer: bytes outside the range keep their fill value
+        # in place in a full-size buffer: bytes outside the range keep their fill value (the plain call: tables
+        # derived inside the decode, caller scratch where the stream needs it)
+        d = ep.upload(blob, prepare=False)
         full = torch.full((I.R * I.C * es,), 0xA5, dtype=torch.uint8, device="cuda")
         t0, cnt = I.n_tiles // 3, max(1, I.n_tiles // 3)
         ep.decode_tiles(I, d.d_stream, d.d_tile_index, d.d_row_scales, dt, full.data_ptr(), t0, cnt,

@@ -129,7 +129,7 @@ def test_validate_rejects_damaged_structure():
 
 
 def test_suggested_tile_size_fills_whole_rounds_of_slots():
-    slots = 148 * 32
+    slots = 148 * ep.decode_tiles_per_sm()
     for R, C, bpp in ((8192, 8192, 4.0), (8192, 8192, 2.0), (8192, 8192, 6.0), (10240, 3840, 4.0), (5120, 17408, 3.5)):
         V = ep.suggest_tile_vectors(R, C, bpp, slots)
         assert V <= ep.default_tile_vectors(bpp) and V % 32 == 0
@@ -144,7 +144,7 @@ def test_suggested_tile_size_for_a_batch_minimises_the_number_of_group_steps():
     ctas = 148
 
     def steps(shapes, V):                     # rounds per CTA times groups per round (plus the fixed cost per round)
-        rounds = sum(-(-(-(-(R * (C // 8)) // V)) // 32) for R, C in shapes)
+        rounds = sum(-(-(-(-(R * (C // 8)) // V)) // ep.decode_tiles_per_sm()) for R, C in shapes)
         return -(-rounds // ctas) * (V // 32 + 2)
 
     for shapes, bpp in ((synth.BLOCK_SHAPES, 3.5), (synth.BLOCK_SHAPES, 2.5), ([(8192, 8192)], 4.0),
