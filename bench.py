@@ -11,7 +11,14 @@ two the roofline target is stated on); the other one, the 8192x8192 Laplace tens
   python bench.py --impl reference       # the CPU oracle on the same workload (bounded sample per step)
 
 Prints ONE JSON line (rank 0).  Timing: CUDA events on the launching stream around each step, an
-L2 flush (512 MB write) between steps outside the events, max over ranks.
+L2 flush (512 MB write) between steps outside the events, max over ranks.  After the headline measurement (and
+outside its timed region) the default run also measures the other stated configurations and puts them in the
+same line under "records": the 8192x8192 tensor at 4.0 bpp with its own roofline block, its rate sweep 2.0 .. 6.0,
+the block bundle decoded to FP8-E4M3 and to INT8, the paper's default tile size, and one GPU-encoder call
+(--no-extras skips them).
+
+--gpus N > 1 without a launcher starts N ranks itself (torch.distributed.run on 127.0.0.1): independent replicas,
+NCCL only for the barrier and the max-reduction of the times.
 """
 from __future__ import annotations
 
@@ -34,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEA
 
 # dram bytes (read + write) per launch measured with ncu for the default workload, filled in from
 # profiles/ after a capture; None = not captured for this workload
-NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 41855744 + 76059904,      # dram read + write of one launch
+NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 39866880 + 76230144,      # dram read + write of one launch
                      ("c5", 3.5, "bf16"): 212336128 + 687062272}
 
 
@@ -59,6 +66,8 @@ def parse_args():
                     help="also time decode-then-GEMM against a GEMM on resident BF16 weights (10240x3840 layer, 4 bpp)")
     ap.add_argument("--graph", action="store_true",
                     help="record the step's launches once in a CUDA graph and replay it in the timed region")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="headline workload only: skip the records of the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -66,38 +75,81 @@ def parse_args():
 
 # ---- workloads ---------------------------------------------------------------------------------------
 
-def make_workload(args):
-    """Returns (name, dtype_name, target_bpp, list of layers; a layer is a list of fp32 matrices)."""
+def make_workload(args, rows=None):
+    """Returns (name, dtype_name, target_bpp, list of layers, full shapes of one layer); a layer is a list of fp32
+    matrices.  rows: draw only that many rows of every tensor (same distribution and width; the CPU arm's sample)."""
     from paper_2609_34185_b200 import synth
     w = args.workload
+    cut = (lambda R: R) if rows is None else (lambda R: min(R, rows))
     if w == "c4":
-        return "config4: 8192x8192 Laplace rows", args.dtype or "fp16", args.bpp or 4.0, [[synth.config4()]]
+        return ("config4: 8192x8192 Laplace rows", args.dtype or "fp16", args.bpp or 4.0, [[synth.config4(R=cut(8192))]],
+                [(8192, 8192)])
     if w == "c1":
         if args.tile_vectors < 0:
             args.tile_vectors = 4096            # the configuration fixes one tile per 64 rows
-        return "config1: 512x512 Gaussian rows, one tile per 64 rows", args.dtype or "bf16", args.bpp or 4.0, [[synth.config1()]]
+        return ("config1: 512x512 Gaussian rows, one tile per 64 rows", args.dtype or "bf16", args.bpp or 4.0,
+                [[synth.config1()]], [(512, 512)])
     if w == "c2":
-        return "config2: 4096x4096 Student-t rows", args.dtype or "bf16", args.bpp or 3.0, [[synth.config2()]]
+        return ("config2: 4096x4096 Student-t rows", args.dtype or "bf16", args.bpp or 3.0, [[synth.config2(R=cut(4096))]],
+                [(4096, 4096)])
     if w == "c3":
         kind = args.dtype or "fp8"
-        mats = []
-        for i in range(7):
-            W = synth.config3_tensor(i)
-            if kind in ("fp8", "int8"):
-                import torch
-                a, Wc = synth.to_container(W, kind)
-                if kind == "fp8":
-                    Wc = torch.from_numpy(Wc).to(torch.float8_e4m3fn).float().numpy()
-                else:
-                    Wc = np.clip(np.rint(Wc), -128, 127).astype(np.float32)
-                W = Wc
-            mats.append(W)
-        return "config3: block bundle 4x5120^2 + 3x5120x17408, 0.1% outliers", kind, args.bpp or 2.5, [mats]
+        mats = [container_values(synth.config3_tensor(i, shape=(cut(R), C)), kind)[1] if kind in ("fp8", "int8")
+                else synth.config3_tensor(i, shape=(cut(R), C)) for i, (R, C) in enumerate(synth.BLOCK_SHAPES)]
+        return ("config3: block bundle 4x5120^2 + 3x5120x17408, 0.1% outliers", kind, args.bpp or 2.5, [mats],
+                list(synth.BLOCK_SHAPES))
     if w == "c5":
-        layers = [[synth.config5_tensor(l, i) for i in range(7)] for l in range(args.distinct_layers)]
+        layers = [[synth.config5_tensor(l, i, shape=(cut(R), C)) for i, (R, C) in enumerate(synth.BLOCK_SHAPES)]
+                  for l in range(args.distinct_layers if rows is None else 1)]
         return (f"config5: {args.layers}-layer stack of block bundles ({args.distinct_layers} distinct layers "
-                f"encoded, cycled)"), args.dtype or "bf16", args.bpp or 3.5, layers
+                f"encoded, cycled)"), args.dtype or "bf16", args.bpp or 3.5, layers, list(synth.BLOCK_SHAPES)
     raise ValueError(w)
+
+
+def container_values(W, kind):
+    """The FP8 / INT8 route (Sec. "FP8 and INT8 computation"): weights scaled row by row into the container and
+    rounded to its grid; these values are what gets compressed.  Returns (per-row output scale, container values)."""
+    from paper_2609_34185_b200 import synth
+    a, Wc = synth.to_container(W, kind)
+    if kind == "fp8":
+        import torch
+        return a, torch.from_numpy(Wc).to(torch.float8_e4m3fn).float().numpy()
+    return a, np.clip(np.rint(Wc), -128, 127).astype(np.float32)
+
+
+# tile-size suggestions in plain Python, for the CPU arm (which must not load the CUDA library): the same rules as
+# ep_suggest_tile_vectors / ep_suggest_tile_vectors_batch with 32 tiles per SM (tests compare the two)
+TILES_PER_SM = 32
+
+
+def suggest_v_py(R, C, vmax, slots):
+    nvec = R * (C // 8)
+    if slots == 0 or nvec == 0:
+        return vmax
+    floor_v = max(32, vmax // 4 // 32 * 32)
+    rounds = 1
+    while True:
+        tiles = rounds * slots
+        V = -(-nvec // tiles)
+        if V <= vmax:
+            V32 = (V + 31) // 32 * 32
+            if V32 <= vmax:
+                V = V32
+            return max(V, floor_v)
+        rounds += 1
+
+
+def suggest_v_batch_py(shapes, vmax, ctas):
+    if not shapes or ctas == 0:
+        return vmax
+    lo = max(32, vmax // 4 // 32 * 32)
+    best_v, best_cost = vmax, None
+    for V in range(lo, vmax + 1, 32):
+        rounds = sum(-(-(-(-(R * (C // 8)) // V)) // TILES_PER_SM) for R, C in shapes)
+        cost = -(-rounds // ctas) * (V // 32 + 2)
+        if best_cost is None or cost <= best_cost:
+            best_cost, best_v = cost, V
+    return best_v
 
 
 def pick_tile_vectors(V, shape, bpp, slots, batch_shapes=None):
@@ -226,32 +278,58 @@ def oracle_time(blob, dtype_name, tiles, reps):
 
 
 def run_reference(args):
-    """The reference arm: the CPU oracle's decoder on this workload's first stream, a bounded tile
-    range per step.  Rank 0 only."""
+    """The reference arm: the CPU oracle alone (encoder and decoder; the CUDA library is never loaded).  A step
+    decodes a bounded sample of the workload: the first rows of every tensor of its first layer, compressed by
+    the oracle's encoder at the workload's target rate and the GPU arm's tile size.  Rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import oracle
-    name, dtype_name, bpp, layers = make_workload(args)
-    V = args.tile_vectors
-    import paper_2609_34185_b200 as ep
-    blob = ep.encode(layers[0][0], bpp, tile_vectors=pick_tile_vectors(V, layers[0][0].shape, bpp, 148 * 48,
-                                                                       [W.shape for W in layers[0]]))
-    I = blob.info
-    # each step decodes a leading tile range (repeated if short) sized so that the whole run stays near a minute
-    params, tiles, reps, threads = oracle_sample(blob, dtype_name, min(0.5, 60.0 / max(1, args.steps + args.warmup)))
+    probe_rows = 64
+    name, dtype_name, bpp, layers, shapes = make_workload(args, rows=probe_rows)
+    vmax = oracle.default_tile_vectors(bpp)
+    if args.tile_vectors >= 0:
+        V = args.tile_vectors
+    elif len(shapes) > 1:
+        V = suggest_v_batch_py(shapes, vmax, 148)
+    else:
+        V = suggest_v_py(shapes[0][0], shapes[0][1], vmax, 148 * TILES_PER_SM)
+    odt = ORACLE_DT[dtype_name]
+
+    def encode_all(mats):
+        return [oracle.encode(W, bpp, oracle.default_opts(tile_vectors=V))[0] for W in mats]
+
+    def decode_all(blobs):
+        t0 = time.perf_counter()
+        for b in blobs:
+            oracle.decode(b, odt)
+        return time.perf_counter() - t0
+
+    # size the sample: rows per tensor such that one step takes about the budget (whole run: about a minute)
+    blobs = encode_all(layers[0])
+    decode_all(blobs)
+    dt = max(decode_all(blobs), 1e-4)
+    budget = min(0.5, 60.0 / max(1, args.steps + args.warmup))
+    rows = int(max(8, min(max(R for R, _ in shapes), probe_rows * budget / dt)))
+    if rows != probe_rows:
+        name, dtype_name, bpp, layers, shapes = make_workload(args, rows=rows)
+        blobs = encode_all(layers[0])
+    params = sum(W.size for W in layers[0])
+    stored = 8.0 * sum(len(b) for b in blobs) / params
     times = []
     for i in range(args.warmup + args.steps):
-        dt = oracle_time(blob, dtype_name, tiles, reps)
+        dt = decode_all(blobs)
         if i >= args.warmup:
             times.append(dt)
-    params *= reps
     total = sum(times)
     value = params * len(times) / total / 1e9
-    sample = f"oracle decoder, tiles 0..{tiles} of {I.n_tiles} of the first tensor x{reps} ({params} params) per step"
+    threads = oracle.num_threads()
+    sample = (f"oracle decoder on oracle-encoded streams of the first {rows} rows of each of the {len(blobs)} tensors of "
+              f"the workload's first layer ({params} params per step)")
     line = {"impl": "reference", "metric": "decoded Gparams/s", "value": value, "unit": "Gparams/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
-            "config": {"workload": name, "target_bpp": bpp, "stored_bpp": blob.stored_bpp, "tile_vectors": I.V},
+            "config": {"workload": name, "target_bpp": bpp, "stored_bpp": stored, "tile_vectors": V,
+                       "out_dtype": dtype_name, "params_per_step": params},
             "cpu_baseline": {"value": value, "unit": "Gparams/s", "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "Gparams/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -268,7 +346,7 @@ def decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms):
     from paper_2609_34185_b200 import synth
     R, C, bpp = 10240, 3840, 4.0
     W = synth.gaussian_rows(R, C, 77)
-    V = pick_tile_vectors(-1, W.shape, bpp, 32 * n_sms)
+    V = pick_tile_vectors(-1, W.shape, bpp, ep.decode_tiles_per_sm() * n_sms)
     blob = ep.encode(W, bpp, tile_vectors=V)
     d = ep.upload(blob, device=dev)
     Wd = torch.empty(R, C, dtype=torch.bfloat16, device=dev)
@@ -310,8 +388,116 @@ def decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms):
             "rows": rows}
 
 
+
+def peak_info():
+    """(HBM GB/s the roofline fractions refer to, where the number comes from)"""
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak, skip):
+    """The stated configurations other than the headline one, each timed as the paper times its codec (CUDA events
+    around the call, three warm-ups, fifteen runs; here with an L2 flush before every run and the median reported).
+    Streams come from the library's GPU encoder (byte-identical to the host encoder's).  Returns a dict of records."""
+    from paper_2609_34185_b200 import synth
+
+    def timed(fn, reps=15, warm=3):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(reps):
+            flush.fill_(0)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return min(ts), statistics.median(ts)
+
+    def record(params, nbytes_in, esize, ms, **more):
+        alg = nbytes_in + params * esize
+        gbs = alg / (ms * 1e-3) / 1e9
+        return dict(Gparams_per_s=params / (ms * 1e-3) / 1e9, median_ms=ms, effective_GBps=gbs,
+                    roofline={"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                              "bytes_per_launch": alg, "ms_per_launch": ms, "kernel": "ep_decode_smem_kernel"}, **more)
+
+    out = {}
+    # ---- config 4: 8192 x 8192 Laplace rows to FP16, 4.0 bpp and the sweep 2.0 .. 6.0 ----
+    W4 = torch.from_numpy(synth.config4()).to(dev)
+    buf = torch.empty((8192, 8192), dtype=torch.float16, device=dev)
+    sweep = []
+    for r in (2.0, 2.5, 3.0, 3.5, 4.0, 4.5, 5.0, 5.5, 6.0):
+        V = ep.suggest_tile_vectors(8192, 8192, r, slots)
+        bl = ep.encode_device(W4, r, tile_vectors=V)
+        dd = ep.upload(bl, device=dev)
+        mn, med = timed(lambda: ep.decode(dd, ep.FP16, out=buf, stream=stream))
+        rec = record(W4.numel(), len(bl), 2, med, target_bpp=r, stored_bpp=bl.stored_bpp, tile_vectors=bl.info.V,
+                     b=bl.info.b, min_ms=mn)
+        sweep.append(rec)
+        if r == 4.0:
+            out["config4_fp16_4.0bpp"] = dict(rec, traffic=NCU_TRAFFIC_BYTES.get(("c4", 4.0, "fp16")))
+            # the paper's default tile size for this rate (not a multiple of 32: the last group of every tile is
+            # partly filled) against the suggested one
+            blp = ep.encode_device(W4, r, tile_vectors=ep.default_tile_vectors(r))
+            dp = ep.upload(blp, device=dev)
+            mnp, medp = timed(lambda: ep.decode(dp, ep.FP16, out=buf, stream=stream))
+            out["config4_fp16_4.0bpp_paper_tile_size"] = record(W4.numel(), len(blp), 2, medp, target_bpp=r,
+                                                                stored_bpp=blp.stored_bpp, tile_vectors=blp.info.V, min_ms=mnp)
+            del dp
+        del dd
+    out["config4_sweep_fp16"] = [{k: v for k, v in rec.items() if k != "roofline"} | {"frac": rec["roofline"]["frac"]}
+                                 for rec in sweep]
+    # one call of the GPU encoder on the same tensor (wall time of the call, buffers warm)
+    ws = None
+    for _ in range(2):
+        t0 = time.perf_counter()
+        bl = ep.encode_device(W4, 4.0, tile_vectors=ep.suggest_tile_vectors(8192, 8192, 4.0, slots))
+        enc_ms = 1e3 * (time.perf_counter() - t0)
+    out["encode_device_8192x8192_4.0bpp"] = {"ms": enc_ms, "stored_bpp": bl.stored_bpp,
+                                             "what": "ep_encode_device call to finished host blob, second call"}
+    del W4, buf
+    # ---- config 3: the block bundle in its FP8-E4M3 and INT8 containers, 2.5 bpp, one batched launch ----
+    if skip != "c3":
+        V = ep.suggest_tile_vectors_batch(synth.BLOCK_SHAPES, 2.5, n_sms)
+        src = [synth.config3_tensor(i) for i in range(7)]
+        for kind, DT, tdt in (("fp8", ep.FP8_E4M3, torch.float8_e4m3fn), ("int8", ep.INT8, torch.int8)):
+            blobs = [ep.encode_device(torch.from_numpy(container_values(W, kind)[1]).to(dev), 2.5, tile_vectors=V) for W in src]
+            total = sum(b.info.R * b.info.C for b in blobs)
+            obuf = torch.empty(total, dtype=tdt, device=dev)
+            outs, at = [], 0
+            for b in blobs:
+                n = b.info.R * b.info.C
+                outs.append(obuf[at:at + n].view(b.info.R, b.info.C))
+                at += n
+            ds = [ep.upload(b, device=dev) for b in blobs]
+            mn, med = timed(lambda: ep.decode_many(ds, DT, outs, stream=stream))
+            nin = sum(len(b) for b in blobs)
+            out[f"config3_{kind}_2.5bpp"] = record(total, nin, 1, med, target_bpp=2.5, stored_bpp=8.0 * nin / total,
+                                                   tile_vectors=V, min_ms=mn, launches=1)
+            del ds, obuf, outs, blobs
+    if ep.last_device_status() != 0:
+        raise RuntimeError("decoder reported an inconsistent stream in the extra records")
+    return out
+
+
 def main():
     args = parse_args()
+    env_world = os.environ.get("WORLD_SIZE")
+    if args.gpus > 1 and env_world is None:
+        # no launcher: start the N ranks ourselves, one process per GPU, rendezvous on the loopback address
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if env_world is not None and int(env_world) != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {env_world} ranks", file=sys.stderr)
+        sys.exit(2)
     if args.impl == "reference":
         run_reference(args)
         return
@@ -329,7 +515,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    name, dtype_name, bpp, layers = make_workload(args)
+    name, dtype_name, bpp, layers, _shapes = make_workload(args)
     DT = {"bf16": ep.BF16, "fp16": ep.FP16, "fp8": ep.FP8_E4M3, "int8": ep.INT8}[dtype_name]
     tdt = {"bf16": torch.bfloat16, "fp16": torch.float16, "fp8": torch.float8_e4m3fn, "int8": torch.int8}[dtype_name]
     esize = ep.DTYPE_BYTES[DT]
@@ -447,7 +633,8 @@ def main():
         slot_in = [[torch.empty(len(b), dtype=torch.uint8, device=dev) for b in blobs[l0]] for _ in range(n_slots)]
         slot_dev_out = [torch.empty(layer_params[l0], dtype=tdt, device=dev) for _ in range(n_slots)]
         slot_host_out = [torch.empty(layer_params[l0], dtype=tdt).pin_memory() for _ in range(n_slots)]
-        slot_scratch = [[ep.DeviceBlob(d, b.info) for d, b in zip(slot_in[k], blobs[l0])] for k in range(n_slots)]
+        # (the stream arrives anew in every step: its lookup tables are derived inside the decode, not prepared ahead)
+        slot_scratch = [[ep.DeviceBlob(d, b.info, prepare=False) for d, b in zip(slot_in[k], blobs[l0])] for k in range(n_slots)]
         slot_outs = []
         for k in range(n_slots):
             outs, at = [], 0
@@ -547,16 +734,17 @@ def main():
     if args.gemm_curve and rank == 0:
         gemm_curve = decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms)
 
+
+    records = None
+    if not args.no_extras and rank == 0:
+        records = extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak_info()[0], skip=args.workload)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    peak, peak_src = peak_info()
     # dominant (only) kernel: the fused decode; algorithmic bytes per launch = compressed bytes + weight bytes
     launch_bytes = alg_bytes_step / launches_per_step
     launch_ms = ms_per_step / launches_per_step
@@ -594,7 +782,7 @@ def main():
                        "warm_ms_per_step_no_flush": warm_ms, "rel_l2_first_tensor": rel_l2_first},
             "effective_GBps": eff_gbs, "pct_of_measured_hbm": 100.0 * eff_gbs / peak, "pct_of_8TBps": 100.0 * eff_gbs / 8000.0,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "per_layer_ms": per_layer_ms, "sweep": sweep, "decode_then_gemm": gemm_curve,
+            "per_layer_ms": per_layer_ms, "sweep": sweep, "decode_then_gemm": gemm_curve, "records": records,
             "clocks": clocks}
     print(json.dumps(line), flush=True)
     if world > 1:

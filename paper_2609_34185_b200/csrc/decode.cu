@@ -213,8 +213,10 @@ __device__ __forceinline__ void build_one_table(const JobParams &J, uint32_t t, 
         const uint32_t first = run + incl - f;
         const int32_t v = tmin + int32_t(j);
         const uint32_t code = uint32_t((is_m ? 2 * v : v) - J.zlo);
-        const uint32_t entry = (f << 21) | ((code & 0x3FFu) << 11);
-        if (f >= kLutEntries) atomicOr(&g_ep_status, 1u);   // not a stream the launcher sends here: f does not fit its field
+        // (a frequency of 2^11 or more is not a stream the launcher sends here: it does not fit its field; whatever the
+        // device copy holds, an entry's frequency stays in 1 .. 2047, which the word bound of the ring relies on)
+        const uint32_t entry = (min(f, kLutEntries - 1u) << 21) | ((code & 0x3FFu) << 11);
+        if (f >= kLutEntries) atomicOr(&g_ep_status, 1u);
 #pragma unroll
         for (uint32_t u = 0; u < kOwnSlots; ++u)
             if (u < f && first + u < slots) put(first + u, entry | u);

@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the GPU box)")
+    config.addinivalue_line("markers", "timeout(seconds): upper bound enforced by pytest-timeout where it is installed")
 
 
 def pytest_collection_modifyitems(config, items):

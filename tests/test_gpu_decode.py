@@ -283,6 +283,66 @@ def test_config4_full_size_three_rates():
     _full_compare(W, 6.0, ep.FP16)
 
 
+def test_config4_every_rate_of_the_sweep_at_the_tile_size_the_bench_uses():
+    # the whole sweep 2.0, 2.5 .. 6.0 bpp as `bench.py` times it: streams from the GPU encoder, tile size from
+    # ep_suggest_tile_vectors, FP16 output; every weight against the oracle and the stored rate within 1 %
+    slots = ep.decode_tiles_per_sm() * torch.cuda.get_device_properties(0).multi_processor_count
+    Wd = torch.from_numpy(synth.config4()).cuda()
+    out = torch.empty((8192, 8192), dtype=torch.float16, device="cuda")
+    for bpp in (2.0, 2.5, 3.0, 3.5, 4.0, 4.5, 5.0, 5.5, 6.0):
+        blob = ep.encode_device(Wd, bpp, tile_vectors=ep.suggest_tile_vectors(8192, 8192, bpp, slots))
+        assert abs(blob.stored_bpp - bpp) < 0.01 * bpp, (bpp, blob.stored_bpp)
+        ep.decode(ep.upload(blob), ep.FP16, out=out)
+        ref, _ = oracle.decode(blob.data, oracle.FP16)
+        torch.cuda.synchronize()
+        assert np.array_equal(_bits(out), ref), bpp
+    assert ep.last_device_status() == 0
+
+
+def _container(W, kind):
+    """Row-scaled FP8 / INT8 container values of W as fp32 (the low-precision route compresses these)."""
+    a, Wc = synth.to_container(W, kind)
+    if kind == "fp8":
+        return a, torch.from_numpy(Wc).to(torch.float8_e4m3fn).float().numpy()
+    return a, np.clip(np.rint(Wc), -128, 127).astype(np.float32)
+
+
+@pytest.mark.parametrize("kind,dt,odt", [("fp8", ep.FP8_E4M3, oracle.E4M3), ("int8", ep.INT8, oracle.INT8)])
+def test_config3_whole_bundle_in_one_batched_launch(kind, dt, odt):
+    # the seven tensors of the block bundle at full size (372 M weights), each first scaled row by row into the
+    # FP8 / INT8 container, compressed at 2.5 bpp and decoded into that container by ONE ep_decode_batch launch:
+    # every byte against the oracle; the per-row output scale a_r then brings the weights back (error vs the source)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    V = ep.suggest_tile_vectors_batch(synth.BLOCK_SHAPES, 2.5, sms)
+    blobs, scales, sources = [], [], []
+    for i in range(7):
+        W = synth.config3_tensor(i)
+        a, Wc = _container(W, kind)
+        blobs.append(ep.encode_device(torch.from_numpy(Wc).cuda(), 2.5, tile_vectors=V))
+        scales.append(a)
+        if i in (0, 4):
+            sources.append((i, W))
+        del W, Wc
+    total = sum(b.info.R * b.info.C for b in blobs)
+    assert abs(8.0 * sum(len(b) for b in blobs) / total - 2.5) < 0.025
+    tdt = torch.float8_e4m3fn if kind == "fp8" else torch.int8
+    buf = torch.empty(total, dtype=tdt, device="cuda")
+    outs, at = [], 0
+    for b in blobs:
+        n = b.info.R * b.info.C
+        outs.append(buf[at:at + n].view(b.info.R, b.info.C))
+        at += n
+    ep.decode_many([ep.upload(b) for b in blobs], dt, outs)
+    torch.cuda.synchronize()
+    assert ep.last_device_status() == 0
+    for b, o in zip(blobs, outs):
+        ref, _ = oracle.decode(b.data, odt)
+        assert np.array_equal(_bits(o).view(ref.dtype), ref), (kind, b.info.R, b.info.C)
+    for i, W in sources:                                        # container value times its row's output scale
+        back = outs[i].float().cpu().numpy() * scales[i][:, None]
+        assert oracle.rel_l2(W, back) < 0.25                   # 2.5 bpp: about 20 % on these rows
+
+
 def test_config3_one_wide_tensor_fp8_and_int8_containers():
     # MLP-shaped tensor of the block bundle, pre-scaled to the FP8 / INT8 container as in the paper's
     # low-precision route; decoded values must equal the oracle's in that container

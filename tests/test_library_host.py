@@ -157,3 +157,18 @@ def test_suggested_tile_size_for_a_batch_minimises_the_number_of_group_steps():
         assert steps(shapes, V) == best
         assert all(steps(shapes, v) > best for v in range(V + 32, vmax + 1, 32))      # the largest of the best
     assert ep.suggest_tile_vectors_batch([(8192, 8192)], 4.0, 0) == ep.default_tile_vectors(4.0)
+
+
+def test_bench_tile_size_rules_mirror_the_library():
+    # the CPU arm of bench.py must not load the CUDA library, so it carries the two tile-size rules in Python
+    import bench
+    assert bench.TILES_PER_SM == ep.decode_tiles_per_sm()
+    for bpp in (2.0, 3.5, 4.0, 6.0, 8.0):
+        vmax = ep.default_tile_vectors(bpp)
+        assert oracle.default_tile_vectors(bpp) == vmax
+        for R, C in ((8192, 8192), (512, 512), (4096, 4096), (10240, 3840), (5120, 17408), (64, 256)):
+            for slots in (148 * 32, 132 * 32, 0):
+                assert bench.suggest_v_py(R, C, vmax, slots) == ep.suggest_tile_vectors(R, C, bpp, slots), (R, C, bpp)
+        for shapes in (synth.BLOCK_SHAPES, [(8192, 8192)], [(4096, 4096), (4096, 11008), (11008, 4096)]):
+            for ctas in (148, 132, 0):
+                assert bench.suggest_v_batch_py(shapes, vmax, ctas) == ep.suggest_tile_vectors_batch(shapes, bpp, ctas)

@@ -227,7 +227,27 @@ def test_relative_error_follows_second_moment_law():
     assert abs(e - ref) < 1e-12
 
 
+def test_papers_printed_error_levels_are_those_of_the_high_resolution_law():
+    # the dtype table's BF16 rows (real weights): the relative error printed there at each stored rate lies within
+    # 30 % of sqrt(929/12960) * s with s from Eq. 9 for unit-variance Gaussian rows at the payload rate (stored
+    # rate minus the tile metadata share of the tile-overhead table), and the oracle on Gaussian rows sits in
+    # the same band.  Context for the pins above, not a target.
+    rows = [tuple(float(v) for v in ln.split()) for ln in open(os.path.join(GOLDEN, "dtype_table_rates.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert [r[0] for r in rows] == [4.0, 8.0]
+    share = {4.0: 0.0180, 8.0: 0.0360}                      # tile metadata share of the stored bytes at these targets
+    for target, stored, rel_pct in rows:
+        payload = stored * (1.0 - share[target])
+        law = 100.0 * 0.26774 * 2.0 ** (2.047 - payload)
+        assert 0.7 < rel_pct / law < 1.3, (target, rel_pct, law)
+    W = synth.gaussian_rows(256, 1024, 31)
+    blob, rep = oracle.encode(W, 4.0)
+    e = 100.0 * oracle.rel_l2(W, oracle.decode(blob, oracle.FP32)[0])
+    assert 0.8 < e / rows[0][2] < 1.2                         # paper: 7.19 % at 4.02 bpp
+
+
 def test_sample_rows_are_complete_sorted_and_fixed():
+    # (the paper fixes nothing about the draw beyond "complete rows, shape-dependent seed": parity unpinned)
     r1 = oracle.sample_rows(4096, 4096)
     assert len(r1) == 512 and np.all(np.diff(r1.astype(np.int64)) > 0) and r1.max() < 4096
     assert np.array_equal(r1, oracle.sample_rows(4096, 4096))

@@ -1,14 +1,16 @@
-"""The allocation-free entry point against the regular one.
+"""The allocation-free entry point against the regular one and against the oracle.
 
 ep_decode_tensor_static serves callers that cannot allocate device memory at decode time (they run under a
 framework that owns the allocator and hands them only input and output buffers, or in a serving loop where
 an allocation would stall the device): streams that need large lookup tables get them built in a fixed
-area inside the library instead of in caller scratch.  Its output must equal ep_decode_tensor's bit for
-bit, also on a second call that reuses the area with different tables.  Collected last on purpose."""
+area inside the library instead of in caller scratch.  Its output must equal ep_decode_tensor's and the CPU
+oracle's bit for bit, also on a second call that reuses the area with different tables, and the call must leave
+the amount of free device memory as it found it.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2609_34185_b200 as ep
 from paper_2609_34185_b200 import synth
 
@@ -28,13 +30,20 @@ def test_static_area_decode_equals_scratch_decode_twice_in_a_row():
     small = ep.encode(Wa, 4.0)                                # tables fit shared memory: no scratch at all
     assert ep.decode_scratch_bytes(a.info) > 0 and ep.decode_scratch_bytes(b.info) > 0
     assert ep.decode_scratch_bytes(small.info) == 0
-    for dt, tdt in ((ep.BF16, torch.bfloat16), (ep.INT8, torch.int8)):
+    for dt, tdt, odt in ((ep.BF16, torch.bfloat16, oracle.BF16), (ep.INT8, torch.int8, oracle.INT8)):
         for blob in (a, b, a, small):                          # back to back, the area is reused and overwritten
-            d = ep.upload(blob)
+            d = ep.upload(blob, prepare=False)
             ref = ep.decode(d, dt)                             # existing entry point, scratch from the caller
-            got = _static(d, dt, torch.empty((blob.info.R, blob.info.C), dtype=tdt, device="cuda"))
+            out = torch.empty((blob.info.R, blob.info.C), dtype=tdt, device="cuda")
+            _static(d, dt, out)                                # first use: looks up the area's address
             torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
+            got = _static(d, dt, out)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before  # the call took no device memory
             assert torch.equal(got.view(torch.uint8), ref.view(torch.uint8))
+            want, _ = oracle.decode(blob.data, odt)             # and the independent CPU decoder agrees
+            assert np.array_equal(got.view(torch.uint8).cpu().numpy().reshape(-1), want.reshape(-1).view(np.uint8))
     assert ep.last_device_status() == 0
 
 
@@ -42,7 +51,7 @@ def test_static_area_decode_equals_scratch_decode_twice_in_a_row():
 def test_static_area_refuses_tables_it_cannot_hold():
     W = synth.gaussian_rows(32, 512, 303)
     big = ep.encode(W, 4.0, b_start=14)
-    d = ep.upload(big)
+    d = ep.upload(big, prepare=False)
     out = torch.empty((32, 512), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(ep.EntroPackError) as ei:
         _static(d, ep.BF16, out)
