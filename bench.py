@@ -448,6 +448,14 @@ def extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak, skip):
                                                                 stored_bpp=blp.stored_bpp, tile_vectors=blp.info.V, min_ms=mnp)
             del dp
         del dd
+    # the paper's other headline rate: 8 bpp (b = 12, two-level lookup tables)
+    V8 = ep.suggest_tile_vectors(8192, 8192, 8.0, slots)
+    bl8 = ep.encode_device(W4, 8.0, tile_vectors=V8)
+    d8 = ep.upload(bl8, device=dev)
+    mn8, med8 = timed(lambda: ep.decode(d8, ep.FP16, out=buf, stream=stream))
+    out["config4_fp16_8.0bpp"] = record(W4.numel(), len(bl8), 2, med8, target_bpp=8.0, stored_bpp=bl8.stored_bpp,
+                                        tile_vectors=bl8.info.V, b=bl8.info.b, min_ms=mn8)
+    del d8
     out["config4_sweep_fp16"] = [{k: v for k, v in rec.items() if k != "roofline"} | {"frac": rec["roofline"]["frac"]}
                                  for rec in sweep]
     # one call of the GPU encoder on the same tensor (wall time of the call, buffers warm)

@@ -182,11 +182,14 @@ size_t ep_blob_bytes(const ep_blob *blob);       /* B_stored of Eq. 1 */
 int ep_blob_report(const ep_blob *blob, ep_encode_report *out);
 void ep_blob_free(ep_blob *blob);
 
-/* Parse header and table directory of a host copy of a blob (n bytes). */
+/* Parse header and table directory of a host copy of a blob (n bytes): the "tensor layout" and "frequency tables,
+ * alphabet offsets" parts of the stored representation (Sec. 3.6, paragraph on the stored representation;
+ * App. "Tile layout and storage").  EP_ERR_BAD_STREAM if the bytes are not a blob of this format. */
 int ep_blob_info(const void *blob, size_t n, ep_info *out);
 
-/* Full structural check of a host copy of a blob: sizes and offsets consistent and monotone,
- * frequencies of every used table sum to 2^b, states inside [2^15, 2^31).  A blob that passes can
+/* Full structural check of a host copy of a blob against what the stored representation must satisfy (Sec. 3.6;
+ * App. "Tile layout and storage", "State normalisation"): sizes and offsets consistent and monotone,
+ * frequencies of every used table sum to 2^b (Sec. 3.3), states inside [2^15, 2^31).  A blob that passes can
  * be given to the decoder without risk of out-of-range accesses. */
 int ep_validate(const void *blob, size_t n);
 
@@ -234,8 +237,10 @@ int ep_decode_tiles(const ep_info *info, const void *d_stream, const void *d_til
                     const float *d_row_scales, int32_t out_dtype, void *d_out, void *d_scratch,
                     size_t scratch_bytes, uint32_t tile_begin, uint32_t tile_count, void *stream);
 
-/* The same for up to EP_MAX_BATCH tensors in one kernel launch (independent tiles of all tensors
- * share the grid).  Jobs needing scratch get their lookup tables built by one extra launch first. */
+/* The same decode (Sec. 3.7) for up to EP_MAX_BATCH tensors in one kernel launch: tiles are independently
+ * decodable (Sec. 3.6), so the tiles of all tensors share one grid - the way the paper's per-layer use decodes the
+ * weights of a block before its matrix products (Sec. "Reconstruction cost and tile overhead").  All jobs of a call
+ * have the same out_dtype.  Jobs needing scratch get their lookup tables built by one extra launch first. */
 int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
 
 /* Largest probability precision b served by ep_decode_tensor_static: its built-in table area holds
@@ -260,9 +265,12 @@ int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
 int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const void *d_tile_index,
                             const float *d_row_scales, int32_t out_dtype, void *d_out, void *stream);
 
-/* Device-side integrity word.  The kernel ORs in a flag when a tile does not end with every state
- * at 2^15 and its word pointer at the next tile's offset (a damaged stream).  This call
- * synchronises `stream`, returns EP_OK or EP_ERR_BAD_STREAM / EP_ERR_CUDA, and clears the word.
+/* Device-side integrity word (no counterpart in the paper; it uses the fact that the encoder of Eq. 17 starts
+ * every state at 2^15, so a correct decode of Eq. 18 must end there).  The kernel ORs in a flag when a tile does
+ * not end with every state at 2^15 and its word pointer at the next tile's offset (a damaged stream).  There is ONE
+ * such word per device and process, shared by all streams and callers: the `stream` argument only says which
+ * stream to wait for.  This call synchronises `stream`, returns EP_OK or EP_ERR_BAD_STREAM / EP_ERR_CUDA, and
+ * clears the word.
  * For tests and debugging; not needed on the hot path.  The decode kernels take every address bound
  * from `info` (sizes, counts, offsets), never from the stream's contents: damaged tables, tile records
  * or payload give wrong weights and this flag, not an access outside the buffers `info` describes.
@@ -270,7 +278,7 @@ int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const voi
 int ep_last_device_status(void *stream);
 
 /* ---- misc --------------------------------------------------------------------------------- */
-const char *ep_strerror(int status);
+const char *ep_strerror(int status);                  /* text of an ep_status value (library convention, not the paper's) */
 uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile-size defaults */
 
 /* Tile size for a decoder with `decode_slots` concurrent tile slots (ep_decode_tiles_per_sm() = 48 per SM for this library: 7104 on

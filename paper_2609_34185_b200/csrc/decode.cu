@@ -57,7 +57,15 @@ constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 per chain
 constexpr uint32_t kCtxBytes = 32 + 32 * kChains;            // per warp: what the rare paths of the hot loop need
 constexpr uint32_t kRingBase = kLutBytes;
 constexpr uint32_t kCtxBase = kRingBase + kWarps * kChains * kRingStride;
-constexpr uint32_t kSmemBytes = kCtxBase + kWarps * kCtxBytes;   // 231680
+// 2^12-slot streams: the symbols within kHotSpan of each table's most frequent one have their entry of the symbol
+// array in shared memory (the rest is read from global memory); this fills what the tables, rings and context
+// blocks of the 32-warp build leave of the 227 KB
+constexpr uint32_t kHotSpan = 264;
+constexpr uint32_t kHotEntries = 16 * kHotSpan;              // 4224: image values below this are hot indices
+constexpr uint32_t kHotBytes = kHotEntries * 8;              // 33792
+constexpr uint32_t kHotBase = kCtxBase + kWarps * kCtxBytes;
+constexpr bool kTwoLevelInLoop = EP_CHAINS == 1 && kHotBase + kHotBytes <= 232448;
+constexpr uint32_t kSmemBytes = kHotBase + (kTwoLevelInLoop ? kHotBytes : 0);   // 232448 in the default build
 static_assert(kSmemBytes <= 232448, "more shared memory than an sm_100 CTA can have");
 constexpr uint32_t kCodeMask = 0x001FF800u;                  // 10-bit code field
 constexpr uint32_t kExp4096 = 0x45800000u;                   // fp32 bit pattern of 4096.0
@@ -87,7 +95,10 @@ struct JobParams {
     const uint32_t *tile_index;   // n_tiles records of 33 words + 1 final word
     const float *scales;
     void *out;
-    const uint32_t *lut_image;    // tables prepared by ep_prepare_tables (16 x 2048 entries), or null: build them here
+    const uint32_t *lut_image;    // 128 KB table image from ep_prepare_tables / the table-build launch, or null: build the
+                                  // tables here (b <= 11 only)
+    const uint2 *l2;              // b = 12: the symbol array behind the image's 16-bit indices, and
+    uint32_t l2max;               //         its last index
     uint32_t off_freq;            // byte offset of the u16 frequency arrays inside the blob
     uint32_t off_payload;
     uint32_t total_words;
@@ -245,9 +256,12 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
 
 // the prepared image of the same sixteen tables: 128 KB copied by all threads of the CTA, 16 bytes each.  The
 // copy is only started here; whoever reads the tables first waits for it (cp.async.wait_group, then a CTA barrier).
-__device__ __forceinline__ void copy_tables_smem(const uint32_t *image, uint32_t lut_addr) {
+__device__ __forceinline__ void copy_tables_smem(const uint32_t *image, uint32_t lut_addr, bool two_level) {
     const uint64_t src = reinterpret_cast<uint64_t>(image);
     for (uint32_t o = 16u * threadIdx.x; o < kLutBytes; o += 16u * kThreads) cp_async16(lut_addr + o, src + o, 16);
+    if (kTwoLevelInLoop && two_level)        // the hot part of the symbol array follows the image
+        for (uint32_t o = 16u * threadIdx.x; o < kHotBytes; o += 16u * kThreads)
+            cp_async16(lut_addr + kHotBase + o, src + kLutBytes + o, 16);
     cp_async_commit();
 }
 
@@ -540,6 +554,9 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F0 "%10"
 #define EP_F1 "%11"
 #define EP_L16 "%12"
+#define EP_L2B "%13"
+#define EP_KMAX "%14"
+#define EP_HOTOFF "%15"
 #elif EP_CHAINS == 2
 #define EP_LT "%8"     /* lanes below this one (mask) */
 #define EP_LUT0 "%9"   /* tables of coset 0 */
@@ -549,7 +566,10 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_OUT "%13"   /* output base address */
 #define EP_F0 "%14"    /* frequency of coset 0 */
 #define EP_F1 "%15"    /* frequency of coset 1, at least 1 */
-#define EP_L16 "%16"   /* 16 * lane */
+#define EP_L16 "%16"
+#define EP_L2B "%17"   /* level-2 table of the 2^12-slot streams (global) */
+#define EP_KMAX "%18"
+#define EP_HOTOFF "%19"  /* its last index */   /* 16 * lane */
 #elif EP_CHAINS == 3
 #define EP_LT "%12"
 #define EP_LUT0 "%13"
@@ -560,6 +580,9 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F0 "%18"
 #define EP_F1 "%19"
 #define EP_L16 "%20"
+#define EP_L2B "%21"
+#define EP_KMAX "%22"
+#define EP_HOTOFF "%23"
 #else
 #define EP_LT "%16"
 #define EP_LUT0 "%17"
@@ -570,6 +593,9 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F0 "%22"
 #define EP_F1 "%23"
 #define EP_L16 "%24"
+#define EP_L2B "%25"
+#define EP_KMAX "%26"
+#define EP_HOTOFF "%27"
 #endif
 // one macro call per chain: M(S = suffix, X, AW, BAL, DOFF, CB = byte offset of the chain's context, more...)
 #define EP_CH_A(M, ...) M("A", "%0", "%1", "%2", "%3", "32", ##__VA_ARGS__)
@@ -677,6 +703,69 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_PARX(S, X, AW, BAL, DOFF, CB) "lop3.b32 par" S ", par" S ", 0x800, cc" S ", 0xEA;\n\t"
 #define EP_X8(S, X, AW, BAL, DOFF, CB) "lop3.b32 xb" S ", e8" S ", " EP_CM ", par" S ", 0xEA;\n\t"
 #define EP_ADDR(S, X, AW, BAL, DOFF, CB) "mad.wide.u32 ad" S ", " DOFF ", 1, " EP_OUT ";\n\t"
+
+// ---- streams with 2^12 slots per table (b = 12: the paper's setting for 8 bpp targets) ------------------------
+// Sixteen tables of 4096 four-byte entries would not fit shared memory, so the lookup has two levels: shared
+// memory holds, per slot, the 16-bit index of the slot's symbol in ONE array of all symbols of all tables (the
+// same 128 KB as the one-level tables of b = 11, same strides), and that array - its most frequent part in
+// shared memory too, all of it in global memory - holds per symbol
+//     word 0: [12:0] f   [15] lowest bit of the coordinate   [31:16] F        word 1: the lattice coordinate
+// z + c/2 (2m + c/2 for the m field) as fp32, so that Eq. 19 is one multiply.  XD = register that receives word 1.
+#define EP_M1(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "and.b32 u" S ", " X ", 0xFFF;\n\t"
+#define EP_M2(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "mad.lo.u32 t" S ", u" S ", 2, tab" S ";\n\t"
+#define EP_M3(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "ld.shared.u16 w" S ", [t" S "+" OFF "];\n\t"
+/* an index below 4224 is an entry of the hot part in shared memory, any other one (minus 4224) of the whole array */
+#define EP_M4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "setp.lt.u32 pc" S ", w" S ", 4224;\n\t"
+#define EP_M5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "mad.lo.u32 t" S ", w" S ", 8, hotb;\n\t"
+#define EP_M6(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) \
+    "sub.u32 w" S ", w" S ", 4224;\n\t" "min.u32 w" S ", w" S ", " EP_KMAX ";\n\t" "mad.wide.u32 ad" S ", w" S ", 8, " EP_L2B ";\n\t"
+#define EP_M7(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) \
+    "@pc" S " ld.shared.v2.u32 {" E S ", " XD S "}, [t" S "];\n\t" "@!pc" S " ld.global.nc.v2.u32 {" E S ", " XD S "}, [ad" S "];\n\t"
+#define EP_M8(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "shr.u32 q" S ", " X ", 12;\n\t" "and.b32 f" S ", " E S ", 0x1FFF;\n\t"
+#define EP_M9(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "shr.u32 bi" S ", " E S ", 16;\n\t"
+#define EP_M10(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "sub.u32 bi" S ", u" S ", bi" S ";\n\t"
+#define EP_M11(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "@act" S " mad.lo.u32 " X ", f" S ", q" S ", bi" S ";\n\t"
+#define EP_STEP12_ALL(E, OFF, BIN, BOUT, XD)                                                                     \
+    EP_ALL(EP_M1, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M2, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M3, E, OFF, BIN, BOUT, XD)   \
+    EP_ALL(EP_M4, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M5, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M6, E, OFF, BIN, BOUT, XD)   \
+    EP_ALL(EP_M7, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M8, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M9, E, OFF, BIN, BOUT, XD)   \
+    EP_ALL(EP_M10, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M11, E, OFF, BIN, BOUT, XD) EP_RENORM_ALL(E, OFF, BIN, BOUT)
+#define EP_C1_12(S, X, AW, BAL, DOFF, CB) "and.b32 u" S ", " X ", 0xFFF;\n\t"
+#define EP_C2_12(S, X, AW, BAL, DOFF, CB) "shr.u32 q" S ", " X ", 12;\n\t"
+#define EP_COSET12_ALL                                                                               \
+    EP_ALL(EP_C1_12) EP_ALL(EP_C2_12) EP_ALL(EP_C3) EP_ALL(EP_C4) EP_ALL(EP_C5) EP_ALL(EP_C6) EP_ALL(EP_C7)  \
+    EP_RENORM_ALL("", "", BL, NA)
+#define EP_Q1(S, X, AW, BAL, DOFF, CB) "mov.b64 pr" S ", {xa" S ", xb" S "};\n\t"
+#define EP_Q2(S, X, AW, BAL, DOFF, CB) "mul.rn.f32x2 pr" S ", pr" S ", ss" S ";\n\t"
+#define EP_Q3(S, X, AW, BAL, DOFF, CB) "mov.b64 {wl" S ", wh" S "}, pr" S ";\n\t"
+#define EP_PAIR12_ALL EP_ALL(EP_Q1) EP_ALL(EP_Q2) EP_ALL(EP_Q3)
+// z8 = 2m + parity of (z1 + ... + z7): bit 15 of the xor of the first words, added to the m field's coordinate as 1.0
+#define EP_PAR12(S, X, AW, BAL, DOFF, CB)                                \
+    "and.b32 par" S ", par" S ", 0x8000;\n\t"                            \
+    "setp.ne.u32 pc" S ", par" S ", 0;\n\t"                              \
+    "selp.b32 par" S ", 0x3F800000, 0, pc" S ";\n\t"                     \
+    "add.rn.f32 xb" S ", xb" S ", par" S ";\n\t"
+// the nine steps and the arithmetic of one group, 2^11-slot and 2^12-slot streams
+#define EP_BODY11(CVT)                                                                                                \
+        EP_COSET_ALL                                                                                                  \
+        EP_STEP_ALL("e1", "0", NA, NB)     EP_ALL(EP_XA, "e1")                                                        \
+        EP_STEP_ALL("e2", "8192", NB, NA)  EP_ALL(EP_XB, "e2") EP_PAIR_ALL EP_ALL(CVT, "0")                           \
+        EP_STEP_ALL("e3", "16384", NA, NB) EP_ALL(EP_PAR3, "e1", "e2", "e3") EP_ALL(EP_XA, "e3")                      \
+        EP_STEP_ALL("e4", "24576", NB, NA) EP_ALL(EP_XB, "e4") EP_PAIR_ALL EP_ALL(CVT, "1")                           \
+        EP_STEP_ALL("e5", "32768", NA, NB) EP_ALL(EP_PAR3, "par", "e4", "e5") EP_ALL(EP_XA, "e5")                     \
+        EP_STEP_ALL("e6", "40960", NB, NA) EP_ALL(EP_XB, "e6") EP_PAIR_ALL EP_ALL(CVT, "2")                           \
+        EP_STEP_ALL("e7", "49152", NA, NB) EP_ALL(EP_PAR3, "par", "e6", "e7") EP_ALL(EP_XA, "e7")                     \
+        EP_STEP_ALL("e8", "57344", NB, BL) EP_ALL(EP_PARX) EP_ALL(EP_X8) EP_PAIR_ALL EP_ALL(CVT, "3")
+#define EP_BODY12(CVT)                                                                                                \
+        EP_COSET12_ALL                                                                                                \
+        EP_STEP12_ALL("e1", "0", NA, NB, "xa")                                                                        \
+        EP_STEP12_ALL("e2", "8192", NB, NA, "xb")  EP_PAIR12_ALL EP_ALL(CVT, "0")                                     \
+        EP_STEP12_ALL("e3", "16384", NA, NB, "xa") EP_ALL(EP_PAR3, "e1", "e2", "e3")                                  \
+        EP_STEP12_ALL("e4", "24576", NB, NA, "xb") EP_PAIR12_ALL EP_ALL(CVT, "1")                                     \
+        EP_STEP12_ALL("e5", "32768", NA, NB, "xa") EP_ALL(EP_PAR3, "par", "e4", "e5")                                 \
+        EP_STEP12_ALL("e6", "40960", NB, NA, "xb") EP_PAIR12_ALL EP_ALL(CVT, "2")                                     \
+        EP_STEP12_ALL("e7", "49152", NA, NB, "xa") EP_ALL(EP_PAR3, "par", "e6", "e7")                                 \
+        EP_STEP12_ALL("e8", "57344", NB, BL, "xb") EP_ALL(EP_PAR12) EP_PAIR12_ALL EP_ALL(CVT, "3")
 
 // per output type: CVT(S, j, lo, hi) turns weights 2j, 2j+1 into their stored form, STORE(S) writes the block
 #define EP_CVT_BF16(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.bf16x2.f32 o" J S ", wh" S ", wl" S ";\n\t"
@@ -849,31 +938,24 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
           "+&r"(x[2]), "+&r"(a[2]), "+&r"(bal[2]), "+&r"(doff[2]), "+&r"(x[3]), "+&r"(a[3]), "+&r"(bal[3]), "+&r"(doff[3])
 #endif
 
-#define EP_TILES_LOOP_ASM(CVT, STORE, GROUP_BYTES)                                                                    \
+#define EP_TILES_LOOP_ASM(BODY, CVT, STORE, GROUP_BYTES)                                                                    \
     asm volatile(                                                                                                     \
         "{\n\t"                                                                                                       \
         EP_ALL(EP_REGS)                                                                                               \
         ".reg .pred pq, pv, pr;\n\t"                                                                                  \
-        ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, f0c, m21, m11;\n\t"               \
+        ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, f0c, m21, m11, hotb;\n\t"         \
         ".reg .b64 ra, rb;\n\t"                                                                                       \
         ".reg .f32 k0f, k1f;\n\t"                                                                                     \
         "mov.b64 {k0f, k1f}, " EP_KK ";\n\t"                                                                          \
         "mov.b32 c0r, 0x45800000;\n\t"                                                                                \
         "mov.b32 c1r, 0x45800400;\n\t"                                                                                \
         "max.u32 f0c, " EP_F0 ", 1;\n\t"                /* frequency used for coset 0: never 0 */                     \
+        "add.u32 hotb, " EP_LUT0 ", " EP_HOTOFF ";\n\t"           /* hot part of the symbol array (2^12-slot streams) */         \
         "ld.shared.v2.u32 {m21, m11}, [" EP_CTX "+16];\n\t" /* 2^21, 2^11 */                                          \
         EP_ALL(EP_INIT)                                                                                               \
         "bra.uni EP_RARE;\n\t"                                                                                        \
         "EP_LOOP:\n\t"                                                                                                \
-        EP_COSET_ALL                                                                                                  \
-        EP_STEP_ALL("e1", "0", NA, NB)     EP_ALL(EP_XA, "e1")                                                        \
-        EP_STEP_ALL("e2", "8192", NB, NA)  EP_ALL(EP_XB, "e2") EP_PAIR_ALL EP_ALL(CVT, "0")                           \
-        EP_STEP_ALL("e3", "16384", NA, NB) EP_ALL(EP_PAR3, "e1", "e2", "e3") EP_ALL(EP_XA, "e3")                      \
-        EP_STEP_ALL("e4", "24576", NB, NA) EP_ALL(EP_XB, "e4") EP_PAIR_ALL EP_ALL(CVT, "1")                           \
-        EP_STEP_ALL("e5", "32768", NA, NB) EP_ALL(EP_PAR3, "par", "e4", "e5") EP_ALL(EP_XA, "e5")                     \
-        EP_STEP_ALL("e6", "40960", NB, NA) EP_ALL(EP_XB, "e6") EP_PAIR_ALL EP_ALL(CVT, "2")                           \
-        EP_STEP_ALL("e7", "49152", NA, NB) EP_ALL(EP_PAR3, "par", "e6", "e7") EP_ALL(EP_XA, "e7")                     \
-        EP_STEP_ALL("e8", "57344", NB, BL) EP_ALL(EP_PARX) EP_ALL(EP_X8) EP_PAIR_ALL EP_ALL(CVT, "3")                 \
+        BODY(CVT)                                                                                                     \
         EP_ALL(EP_ADDR) EP_ALL(STORE)                                                                                \
         EP_ALL(EP_ADVANCE, #GROUP_BYTES)                                                                              \
         /* one vote for everything rare */                                                                            \
@@ -893,16 +975,17 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
         EP_LOOP_OPERANDS                                                                                              \
         : "r"(lt), "r"(lut_addr), "r"(lut_addr + kCosetStride), "r"(ctx), "l"(kk), "l"(out_base), "r"(cf.f0),         \
-          "r"(cf.f1), "r"(lane16)                                                                                     \
+          "r"(cf.f1), "r"(lane16), "l"(l2base), "r"(l2max), "n"(kHotBase)                                             \
         : "memory")
 
-// kChains tiles of a tensor whose rows hold at least 32 blocks and whose tables have 2^11 slots; chain c takes tile
+// kChains tiles of a tensor whose rows hold at least 32 blocks and whose tables have 2^B slots (B = 11: one-level
+// tables; B = 12: two levels, see EP_M1); chain c takes tile
 // `first + c`.  A chain whose slot lies past the job's last tile gets that last tile's record, only so that its
 // addresses stay inside the stream, and no block at all.  The number of groups is data here, not control flow the
 // compiler reasons about: every branch on it is a bra.uni on a warp vote.
 // `tables_pending`: the job's lookup tables are still being written (by this CTA's own stores or copies): the
 // tiles' records and first payload chunks are requested first, the CTA barrier comes after.
-template <int DT>
+template <int DT, int B>
 __device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t first, uint32_t lut_addr, CosetFreq cf,
                                                   uint32_t ring, uint32_t ctx, uint32_t lane, bool tables_pending) {
     constexpr uint32_t BB = Out<DT>::kBlockBytes;
@@ -934,13 +1017,25 @@ __device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t f
     const uint32_t k0 = __float_as_uint(float(4096 - J.zlo));
     const uint64_t kk = pack64(k0, k0);
     const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
-    if constexpr (DT == EP_BF16) EP_TILES_LOOP_ASM(EP_CVT_BF16, EP_ST_16, 512);
-    else if constexpr (DT == EP_FP16) EP_TILES_LOOP_ASM(EP_CVT_FP16, EP_ST_16, 512);
-    else if constexpr (DT == EP_FP8_E4M3) EP_TILES_LOOP_ASM(EP_CVT_E4M3, EP_ST_F8, 256);
-    else if constexpr (DT == EP_FP8_E5M2) EP_TILES_LOOP_ASM(EP_CVT_E5M2, EP_ST_F8, 256);
-    else if constexpr (DT == EP_FP32) EP_TILES_LOOP_ASM(EP_CVT_FP32, EP_ST_FP32, 1024);
-    else if constexpr (DT == EP_UINT8) EP_TILES_LOOP_ASM(EP_CVT_I8, EP_ST_UINT8, 256);
-    else EP_TILES_LOOP_ASM(EP_CVT_I8, EP_ST_INT8, 256);
+    const uint64_t l2base = reinterpret_cast<uint64_t>(J.l2);
+    const uint32_t l2max = J.l2max;
+    if constexpr (B == 11) {
+        if constexpr (DT == EP_BF16) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_BF16, EP_ST_16, 512);
+        else if constexpr (DT == EP_FP16) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_FP16, EP_ST_16, 512);
+        else if constexpr (DT == EP_FP8_E4M3) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_E4M3, EP_ST_F8, 256);
+        else if constexpr (DT == EP_FP8_E5M2) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_E5M2, EP_ST_F8, 256);
+        else if constexpr (DT == EP_FP32) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_FP32, EP_ST_FP32, 1024);
+        else if constexpr (DT == EP_UINT8) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_I8, EP_ST_UINT8, 256);
+        else EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_I8, EP_ST_INT8, 256);
+    } else {
+        if constexpr (DT == EP_BF16) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_BF16, EP_ST_16, 512);
+        else if constexpr (DT == EP_FP16) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_FP16, EP_ST_16, 512);
+        else if constexpr (DT == EP_FP8_E4M3) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_E4M3, EP_ST_F8, 256);
+        else if constexpr (DT == EP_FP8_E5M2) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_E5M2, EP_ST_F8, 256);
+        else if constexpr (DT == EP_FP32) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_FP32, EP_ST_FP32, 1024);
+        else if constexpr (DT == EP_UINT8) EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_I8, EP_ST_UINT8, 256);
+        else EP_TILES_LOOP_ASM(EP_BODY12, EP_CVT_I8, EP_ST_INT8, 256);
+    }
     cp_async_wait<0>();           // nothing may still be landing in the rings when the next tiles start
     __syncwarp();
     // integrity: the encoder started every state at 2^15 and a tile's words end where the next tile's begin
@@ -987,12 +1082,13 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
             if (at < 2ull * J.total_words) prefetch_l2(J.stream + J.off_payload + at);
         }
         if (tables_in_use) __syncthreads();          // every warp is done with the previous job's tables
-        if (J.lut_image) copy_tables_smem(J.lut_image, lut_addr);
+        if (J.lut_image) copy_tables_smem(J.lut_image, lut_addr, J.b == 12u);
         else build_tables_smem(J, lut_addr, warp, lane);
         const CosetFreq cf = load_coset(J);
         bool tables_pending = true;
         tables_in_use = true;
-        const bool fast = DT != EP_FIELDS_I32 && J.per_row >= 32u && J.b == 11u && J.V < (1u << 20);
+        // (a stream with 2^12 slots reaches this kernel only in the configuration of the hot loop: see the launcher)
+        const bool fast = DT != EP_FIELDS_I32 && J.per_row >= 32u && (J.b == 11u || J.b == 12u) && J.V < (1u << 20);
         if (fast && lane == 0) {                     // what the hot loop's rare paths need to know about the job
             sts64(ctx + kCtxScales, reinterpret_cast<uint64_t>(J.scales));
             sts32(ctx + kCtxRowBytes, J.row_bytes);
@@ -1006,7 +1102,8 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
             const uint32_t base = r * kTilesPerRound + kChains * warp;
             if constexpr (DT != EP_FIELDS_I32) {
                 if (fast) {
-                    decode_tiles_fast<DT>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    if (J.b == 12u) decode_tiles_fast<DT, 12>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    else decode_tiles_fast<DT, 11>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
                     tables_pending = false;
                     continue;
                 }
@@ -1051,6 +1148,11 @@ struct GJobParams {
     int32_t tmin[EP_NUM_TABLES];
     uint16_t tK[EP_NUM_TABLES];
     uint32_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
+    // two-level tables of a 2^12-slot stream (ep_build_tables12_kernel only)
+    uint16_t *image;              // 16 x 4096 symbol indices
+    uint2 *hot;                   // 16 x kHotSpan entries: the hot part
+    uint2 *l2;                    // all symbols of the sixteen coordinate tables
+    uint32_t symoff[EP_NUM_TABLES];   // first index of table t's symbols in l2
 };
 
 struct GBatchParams {
@@ -1100,6 +1202,78 @@ __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_cons
             if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
         }
         lut[u] = (lo << 16) | ((u - uint32_t(F[lo])) & 0xFFFFu);     // lo < K <= 65535
+    }
+}
+
+// Two-level tables of a 2^12-slot stream (see EP_M1): one CTA per (coordinate table, job).  Prefix sums of the
+// frequencies as above; every symbol writes its entry of the symbol array - and, if it lies within the window of
+// kHotSpan symbols around the table's most frequent one, of the hot part that the decode kernel keeps in shared
+// memory -, every slot finds its symbol by binary search and stores the symbol's index: below kHotEntries an index
+// into the hot part, else kHotEntries plus the index into the whole array.  A frequency is stored as at least 1
+// (a symbol that never occurs owns no slot; the floor only keeps a damaged stream from producing states that take
+// a word in every step).
+__global__ void __launch_bounds__(1024) ep_build_tables12_kernel(const __grid_constant__ GBatchParams P) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    __shared__ uint32_t part[1024];
+    __shared__ uint32_t best[1024];
+    __shared__ uint32_t s_lo;
+    const GJobParams &J = P.job[blockIdx.y];
+    const uint32_t t = blockIdx.x + 1u, tid = threadIdx.x;
+    const uint32_t K = J.tK[t];
+    constexpr uint32_t M = 4096;
+    uint16_t *image = J.image + size_t(t - 1u) * M;
+    uint2 *hot = J.hot + (t - 1u) * kHotSpan;
+    const uint2 unused = make_uint2(1u, 0u);                               // f = 1, F = 0, coordinate 0
+    for (uint32_t k = K + tid; k < kHotSpan; k += blockDim.x) hot[k] = unused;   // the part of the window no symbol fills
+    if (K == 0) {
+        for (uint32_t u = tid; u < M; u += blockDim.x) image[u] = uint16_t((t - 1u) * kHotSpan);   // never looked up in a valid stream
+        return;
+    }
+    const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_tables + 8 * EP_NUM_TABLES) + J.foff[t];
+    uint16_t *F = reinterpret_cast<uint16_t *>(smem);              // K + 1 entries
+    const uint32_t per = (K + blockDim.x - 1) / blockDim.x;
+    const uint32_t j0 = min(tid * per, K), j1 = min(j0 + per, K);
+    uint32_t sum = 0, top = 0;                                     // top: (frequency << 16) | (65535 - index): first maximum wins
+    for (uint32_t j = j0; j < j1; ++j) {
+        const uint32_t f = fq[j];
+        sum += f;
+        top = max(top, (f << 16) | (65535u - j));
+    }
+    part[tid] = sum;
+    best[tid] = top;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t run = 0, b = 0;
+        for (uint32_t i = 0; i < blockDim.x; ++i) { const uint32_t v = part[i]; part[i] = run; run += v; b = max(b, best[i]); }
+        F[K] = uint16_t(min(run, M));
+        const uint32_t mode = 65535u - (b & 0xFFFFu);
+        const uint32_t last = K > kHotSpan ? K - kHotSpan : 0u;   // the window lies inside the table
+        s_lo = min(mode > kHotSpan / 2 ? mode - kHotSpan / 2 : 0u, last);
+    }
+    __syncthreads();
+    const uint32_t lo_hot = s_lo;
+    const uint32_t coset = (t - 1u) >> 3, field = (t - 1u) & 7u;          // field 7 is m: its coordinate is 2m (+ parity)
+    uint2 *l2 = J.l2 + J.symoff[t];
+    uint32_t run = part[tid];
+    for (uint32_t j = j0; j < j1; ++j) {
+        const uint32_t f = fq[j], Fj = min(run, M - 1u);
+        F[j] = uint16_t(min(run, M));
+        run += f;
+        const int32_t v = J.tmin[t] + int32_t(j);
+        const float coord = float(field == 7u ? 2 * v : v) + 0.5f * float(coset);
+        const uint32_t par = field == 7u ? 0u : uint32_t(v) & 1u;
+        const uint2 e = make_uint2(min(max(f, 1u), 8191u) | (par << 15) | (Fj << 16), __float_as_uint(coord));
+        l2[j] = e;
+        if (j - lo_hot < kHotSpan) hot[j - lo_hot] = e;           // (unsigned: j below the window wraps to a large number)
+    }
+    __syncthreads();
+    for (uint32_t u = tid; u < M; u += blockDim.x) {
+        uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u (F[0] = 0)
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
+        }
+        image[u] = uint16_t(lo - lo_hot < kHotSpan ? (t - 1u) * kHotSpan + (lo - lo_hot) : kHotEntries + J.symoff[t] + lo);
     }
 }
 
@@ -1275,6 +1449,22 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
 
 size_t large_table_bytes(const ep_info &I) { return size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 4u; }
 
+// 2^12-slot streams whose symbols can be numbered with 16 bits decode from two-level tables in the hot loop
+uint32_t coord_symbols(const ep_info &I) {
+    uint64_t k = 0;
+    for (int t = 1; t < EP_NUM_TABLES; ++t) k += I.table_K[t];
+    return uint32_t(k < 0xFFFFFFFFull ? k : 0xFFFFFFFFull);
+}
+bool fits_two_level(const ep_info &I) {
+    return kTwoLevelInLoop && I.b == 12 && coord_symbols(I) >= 1 && coord_symbols(I) <= 65535u - kHotEntries;
+}
+// image, hot part, symbol array, rounded to 256 bytes; the flat tables of the large-table kernel follow at this offset
+size_t two_level_bytes(const ep_info &I) {
+    return (size_t(kLutBytes) + kHotBytes + 8u * size_t(coord_symbols(I)) + 255u) & ~size_t(255);
+}
+// can the hot loop serve this request?  (the field dump and narrow tensors take the plain kernels)
+bool hot_loop_shape(const ep_info &I, int32_t dt) { return dt != EP_FIELDS_I32 && I.C / 8 >= 32u && I.V < (1u << 20); }
+
 // the host-side parameters of a large-table job (geometry from `info` only); `lut` = where its tables are or go
 int fill_large_job(GJobParams &J, const ep_decode_job &jb, uint32_t *lut) {
     const ep_info &I = *jb.info;
@@ -1302,6 +1492,29 @@ int fill_large_job(GJobParams &J, const ep_decode_job &jb, uint32_t *lut) {
     return EP_OK;
 }
 
+// where the two-level tables of a job live inside its table buffer
+void set_two_level(GJobParams &J, const ep_info &I, void *base) {
+    J.image = static_cast<uint16_t *>(base);
+    J.hot = reinterpret_cast<uint2 *>(static_cast<uint8_t *>(base) + kLutBytes);
+    J.l2 = reinterpret_cast<uint2 *>(static_cast<uint8_t *>(base) + kLutBytes + kHotBytes);
+    uint32_t acc = 0;
+    for (int t = 1; t < EP_NUM_TABLES; ++t) { J.symoff[t] = acc; acc += I.table_K[t]; }
+}
+
+cudaError_t launch_build12(const GBatchParams &P, int n_jobs, cudaStream_t st) {
+    uint32_t max_K = 1;
+    for (int i = 0; i < n_jobs; ++i)
+        for (int t = 1; t < EP_NUM_TABLES; ++t)
+            if (P.job[i].tK[t] > max_K) max_K = P.job[i].tK[t];
+    const size_t smem = 2u * (size_t(max_K) + 1u);
+    if (smem > 48u * 1024u) {
+        const cudaError_t e = cudaFuncSetAttribute(ep_build_tables12_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+    }
+    ep_build_tables12_kernel<<<dim3(EP_NUM_TABLES - 1, n_jobs), 1024, smem, st>>>(P);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_build(const GBatchParams &P, int n_jobs, cudaStream_t st) {
     uint32_t max_K = 1;
     for (int i = 0; i < n_jobs; ++i)
@@ -1321,12 +1534,12 @@ cudaError_t launch_build(const GBatchParams &P, int n_jobs, cudaStream_t st) {
 extern "C" size_t ep_decode_scratch_bytes(const ep_info *info) {
     if (!info) return 0;
     if (fits_smem_tables(*info)) return 0;
-    return large_table_bytes(*info);
+    return (fits_two_level(*info) ? two_level_bytes(*info) : 0) + large_table_bytes(*info);
 }
 
 extern "C" size_t ep_decode_tables_bytes(const ep_info *info) {
     if (!info) return 0;
-    return fits_smem_tables(*info) ? size_t(kLutBytes) : large_table_bytes(*info);
+    return fits_smem_tables(*info) ? size_t(kLutBytes) : ep_decode_scratch_bytes(info);
 }
 
 extern "C" uint32_t ep_decode_tiles_per_sm(void) { return kTilesPerRound; }
@@ -1352,8 +1565,16 @@ extern "C" int ep_prepare_tables(const ep_info *info, const void *d_stream, void
     std::memset(&jb, 0, sizeof(jb));
     jb.info = info;
     jb.d_stream = d_stream;
-    const int rc = fill_large_job(P.job[0], jb, static_cast<uint32_t *>(d_tables));
+    // a 2^12-slot stream gets the two-level tables of the hot loop first, then the flat tables the plain kernel
+    // uses for the field dump and for narrow tensors
+    uint8_t *base = static_cast<uint8_t *>(d_tables);
+    const bool two = fits_two_level(I);
+    const int rc = fill_large_job(P.job[0], jb, reinterpret_cast<uint32_t *>(base + (two ? two_level_bytes(I) : 0)));
     if (rc) return rc;
+    if (two) {
+        set_two_level(P.job[0], I, base);
+        if (launch_build12(P, 1, st) != cudaSuccess) return EP_ERR_CUDA;
+    }
     return launch_build(P, 1, st) == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
@@ -1377,14 +1598,16 @@ int decode_large_tables(const ep_decode_job *const *jobs, int n_jobs, int32_t dt
     for (int i = 0; i < n_jobs; ++i) {
         const ep_decode_job &jb = *jobs[i];
         const ep_info &I = *jb.info;
-        const size_t need = large_table_bytes(I);
+        // the flat tables follow the two-level ones where the buffer has both (prepared tables always, scratch
+        // if it is large enough); a scratch buffer of the flat tables' size alone holds just them
+        const size_t need = large_table_bytes(I), before = fits_two_level(I) ? two_level_bytes(I) : 0;
         uint32_t *lut;
         if (jb.d_tables) {
             if (reinterpret_cast<uintptr_t>(jb.d_tables) & 255) return EP_ERR_SCRATCH;
-            lut = static_cast<uint32_t *>(const_cast<void *>(jb.d_tables));
+            lut = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(const_cast<void *>(jb.d_tables)) + before);
         } else {
             if (!jb.d_scratch || jb.scratch_bytes < need || (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255)) return EP_ERR_SCRATCH;
-            lut = static_cast<uint32_t *>(jb.d_scratch);
+            lut = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(jb.d_scratch) + (jb.scratch_bytes >= before + need ? before : 0));
         }
         GJobParams &J = P.job[i];
         const int rc = fill_large_job(J, jb, lut);
@@ -1450,6 +1673,8 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
             if (jb.tile_count == 0 || jb.tile_begin >= I.n_tiles || jb.tile_count > I.n_tiles - jb.tile_begin) return EP_ERR_BAD_ARG;
         }
         if (fits_smem_tables(I)) { fast[n_jobs++] = &jb; }
+        else if (fits_two_level(I) && hot_loop_shape(I, dt) &&
+                 (jb.d_tables || (jb.d_scratch && jb.scratch_bytes >= two_level_bytes(I)))) { fast[n_jobs++] = &jb; }
         else large[n_large++] = &jb;
     }
     if (n_large) {
@@ -1460,6 +1685,9 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
     BatchParams P;
     std::memset(&P, 0, sizeof(P));
     P.n_jobs = n_jobs;
+    GBatchParams B12;               // two-level tables that have to be built into scratch first
+    std::memset(&B12, 0, sizeof(B12));
+    int n_build12 = 0;
     // persistent CTAs, one per SM (fewer if the launch has fewer rounds than SMs); the kernel splits the
     // cost-weighted list of all rounds evenly over them
     uint64_t rounds_total = 0, cost = 0;
@@ -1474,6 +1702,20 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.scales = jb.d_row_scales;
         J.out = jb.d_out;
         J.lut_image = static_cast<const uint32_t *>(jb.d_tables);
+        if (I.b == 12) {            // two-level tables: prepared, or built into the caller's scratch by a launch before this one
+            void *base = const_cast<void *>(jb.d_tables);
+            if (!base) {
+                if (reinterpret_cast<uintptr_t>(jb.d_scratch) & 255) return EP_ERR_SCRATCH;
+                base = jb.d_scratch;
+                GJobParams &G = B12.job[n_build12++];
+                const int rc = fill_large_job(G, jb, nullptr);
+                if (rc) return rc;
+                set_two_level(G, I, base);
+            }
+            J.lut_image = static_cast<const uint32_t *>(base);
+            J.l2 = reinterpret_cast<const uint2 *>(static_cast<const uint8_t *>(base) + kLutBytes + kHotBytes);
+            J.l2max = coord_symbols(I) - 1u;
+        }
         J.off_payload = I.off_payload;
         J.total_words = uint32_t(I.total_words);
         J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
@@ -1492,6 +1734,10 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
         J.cost_begin = uint32_t(cost);
         cost += uint64_t(J.rounds) * J.round_cost;
         rounds_total += J.rounds;
+    }
+    if (n_build12) {
+        B12.n_jobs = n_build12;
+        if (launch_build12(B12, n_build12, st) != cudaSuccess) return EP_ERR_CUDA;
     }
     const uint32_t next = uint32_t(rounds_total < uint64_t(sms) ? rounds_total : uint64_t(sms));   // grid size
     // a tensor has under 2^27 blocks, so sixteen of them cost under 2^26 groups: 32-bit arithmetic in the kernel
