@@ -41,8 +41,8 @@ FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEA
 
 # dram bytes (read + write) per launch measured with ncu for the default workload, filled in from
 # profiles/ after a capture; None = not captured for this workload
-NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 39866880 + 76230144,      # dram read + write of one launch
-                     ("c5", 3.5, "bf16"): 212336128 + 687062272}
+NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 39859712 + 76110848,      # dram read + write of one launch
+                     ("c5", 3.5, "bf16"): 205188352 + 687194112}
 
 
 def parse_args():
