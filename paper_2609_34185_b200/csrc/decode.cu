@@ -49,11 +49,36 @@ constexpr uint32_t kLutEntries = 2048;                       // 2^11 slots per t
 constexpr uint32_t kLutStride = kLutEntries * 4;             // bytes per table in shared memory
 constexpr uint32_t kCosetStride = 8 * kLutStride;            // the eight tables of coset 1 follow those of coset 0
 constexpr uint32_t kLutBytes = 16 * kLutStride;              // 131072
-constexpr uint32_t kChunk = 512;                             // bytes per cp.async round of a warp
-constexpr uint32_t kRingSlots = 3;
-constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536
+// Payload ring of a chain: kRingSlots chunks of kChunk bytes plus a mirror of its first 512 bytes.  A chunk is one
+// cp.async round of a warp (16 bytes per lane: all 32 lanes for 512 bytes, the first 16 for 256).  With one tile
+// per warp the ring has three 512-byte chunks; two tiles per warp and 32 warps (64 rings in what the tables leave of
+// the shared memory) get four 256-byte chunks each, refilled twice as often.
+#if EP_CHAINS * EP_WARPS > 48
+#define EP_SMALL_RINGS 1
+constexpr uint32_t kChunk = 256, kRingSlots = 4, kMirrorSlots = 2;
+#define EP_CSH "8"          /* log2 of the chunk size */
+#define EP_CMASK "255"      /* chunk size - 1 */
+#define EP_COFF "254"       /* chunk size - 2: the cursor is about to leave its chunk at chunk start + this */
+#define EP_CBYTES "256"
+#define EP_RBYTES "1024"    /* ring size */
+#define EP_RWRAP "1278"     /* ring size + chunk size - 2 */
+#define EP_NSLOT "4"
+#define EP_MSLOT "2"        /* chunks whose slot is below this are written to the mirror too */
+#else
+constexpr uint32_t kChunk = 512, kRingSlots = 3, kMirrorSlots = 1;
+#define EP_CSH "9"
+#define EP_CMASK "511"
+#define EP_COFF "510"
+#define EP_CBYTES "512"
+#define EP_RBYTES "1536"
+#define EP_RWRAP "2046"
+#define EP_NSLOT "3"
+#define EP_MSLOT "1"
+#endif
+constexpr uint32_t kChunkLanes = kChunk / 16;                // lanes that take part in a chunk's copy
+constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536 or 1024
 constexpr uint32_t kRingMirror = 512;                        // >= 7 words * 32 lanes * 2 bytes + one lane span (62)
-constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 per chain
+constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 or 1536 per chain
 constexpr uint32_t kCtxBytes = 32 + 32 * kChains;            // per warp: what the rare paths of the hot loop need
 constexpr uint32_t kRingBase = kLutBytes;
 constexpr uint32_t kCtxBase = kRingBase + kWarps * kChains * kRingStride;
@@ -439,27 +464,29 @@ __device__ __forceinline__ void decode_group_plain(uint32_t &x, uint32_t &wa, ui
 // end.  `room` = bytes from a0 to the end of the payload: nothing beyond it is read (cp.async zero-fills
 // the rest).
 __device__ __forceinline__ void ring_issue(uint32_t ring, uint64_t a0, uint32_t room, uint32_t c, uint32_t lane) {
-    uint32_t o = kChunk * c + 16u * lane;
-    uint32_t n = 16;
-    if (o + 16u > room) {
-        n = o < room ? room - o : 0u;
-        if (n == 0) o = 0;                       // nothing is read, but keep the address a valid one
+    if (lane < kChunkLanes) {
+        uint32_t o = kChunk * c + 16u * lane;
+        uint32_t n = 16;
+        if (o + 16u > room) {
+            n = o < room ? room - o : 0u;
+            if (n == 0) o = 0;                   // nothing is read, but keep the address a valid one
+        }
+        const uint32_t slot = c % kRingSlots;
+        const uint32_t dst = ring + kChunk * slot + 16u * lane;
+        cp_async16(dst, a0 + o, n);
+        if (slot < kMirrorSlots) cp_async16(dst + kRingBytes, a0 + o, n);
     }
-    const uint32_t slot = c % kRingSlots;
-    const uint32_t dst = ring + kChunk * slot + 16u * lane;
-    cp_async16(dst, a0 + o, n);
-    if (slot == 0) cp_async16(dst + kRingBytes, a0 + o, n);
     cp_async_commit();
 }
 
-// The cursor entered a new 512-byte chunk: request chunks up to two ahead of it and wait for all but the
+// The cursor entered a new chunk: request chunks up to kRingSlots - 1 ahead of it and wait for all but the
 // newest.  `threshold` = start of the chunk after the cursor's at the previous service; chunks up to
-// (threshold >> 9) + 1 have been requested.  A group touches at most 448 + 62 bytes from its start,
-// i.e. chunks cur and cur + 1, which are complete after this call.
+// threshold / kChunk + kRingSlots - 2 have been requested.  A group touches at most 448 + 62 bytes from its start,
+// which the chunks complete after this call cover (1024 bytes from the cursor's chunk on, or 768).
 __device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_t room, uint32_t pos, uint32_t &threshold,
                                              uint32_t lane) {
-    const uint32_t cur = pos >> 9;
-    for (uint32_t c = (threshold >> 9) + 2u; c < cur + 3u; ++c) ring_issue(ring, a0, room, c, lane);
+    const uint32_t cur = pos / kChunk;
+    for (uint32_t c = threshold / kChunk + kRingSlots - 1u; c < cur + kRingSlots; ++c) ring_issue(ring, a0, room, c, lane);
     cp_async_wait<1>();
     __syncwarp();
     threshold = kChunk * (cur + 1u);
@@ -807,10 +834,10 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     ".reg .f32 wl" S ", wh" S ", sg" S ";\n\t"                                                                       \
     ".reg .b32 lim" S ", wthr" S ";\n\t"                                                                             \
     ".reg .b64 pr" S ", ss" S ", ad" S ", xw" S ";\n\t"
-// before the first pass: the cursor leaves its first chunk at ring + 510; lim = 0 sends the chain through EP_ROWS
+// before the first pass: the cursor leaves its first chunk at ring + chunk size - 2; lim = 0 sends the chain through EP_ROWS
 #define EP_INIT(S, X, AW, BAL, DOFF, CB)                                 \
     "ld.shared.u32 r0, [" EP_CTX "+" CB "+28];\n\t"                      \
-    "add.u32 wthr" S ", r0, 510;\n\t"                                    \
+    "add.u32 wthr" S ", r0, " EP_COFF ";\n\t"                            \
     "mov.u32 lim" S ", 0;\n\t"
 
 #define EP_ADVANCE(S, X, AW, BAL, DOFF, CB, GROUP_BYTES) "add.u32 " DOFF ", " DOFF ", " GROUP_BYTES ";\n\t"
@@ -859,8 +886,8 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     "EP_ROWS_END_" S ":\n\t"
 #define EP_ANY_ACT(S, X, AW, BAL, DOFF, CB) "or.pred pr, pr, act" S ";\n\t"
 
-// the chain's cursor left its chunk: request the chunks up to two ahead of it (one, as a rule), wait for all but
-// the newest, move the addresses back by the ring's length when the cursor's chunk is the one in slot 0 again.
+// the chain's cursor left its chunk: request the chunks up to (slots - 1) ahead of it (one, as a rule), wait for all
+// but the newest, move the addresses back by the ring's length when the cursor's chunk is the one in slot 0 again.
 // The chain's context is read with two 16-byte loads up front: one shared-memory round trip, not six.
 #define EP_SERVICE(S, X, AW, BAL, DOFF, CB)                              \
     "setp.ge.u32 pr, " AW ", wthr" S ";\n\t"                                                                   \
@@ -872,17 +899,18 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     "popc.b32 r0, " BAL ";\n\t"                                                                                \
     "mad.lo.u32 r6, r0, 2, r6;\n\t"                     /* the cursor's address */                             \
     "sub.u32 r7, r6, r5;\n\t"                           /* its byte position */                                \
-    "shr.u32 r8, r7, 9;\n\t"                            /* its chunk */                                        \
-    "add.u32 r0, r8, 3;\n\t"                                                                                   \
+    "shr.u32 r8, r7, " EP_CSH ";\n\t"                   /* its chunk */                                        \
+    "add.u32 r0, r8, " EP_NSLOT ";\n\t"                                                                        \
     "sub.s32 r0, r0, r9;\n\t"                           /* chunks the cursor has advanced: requests due */     \
-    "min.s32 r0, r0, 3;\n\t"                                                                                   \
+    "min.s32 r0, r0, " EP_NSLOT ";\n\t"                                                                        \
     "max.s32 r0, r0, 0;\n\t"                                                                                   \
-    "shl.b32 r8, r0, 9;\n\t"                            /* bytes the cursor's chunk moves on in the ring */    \
+    "shl.b32 r8, r0, " EP_CSH ";\n\t"                   /* bytes the cursor's chunk moves on in the ring */    \
     "setp.eq.u32 pq, r0, 0;\n\t"                                                                               \
     "@pq bra.uni EP_SVW_" S ";\n\t"                                                                            \
     "mov.b64 ra, {r11, r12};\n\t"                                                                              \
+    "setp.lt.u32 pl, " EP_L16 ", " EP_CBYTES ";\n\t"    /* lanes that copy 16 bytes of a chunk */              \
     "EP_SVL_" S ":\n\t"                                                                                        \
-    "shl.b32 r2, r9, 9;\n\t"                                                                                   \
+    "shl.b32 r2, r9, " EP_CSH ";\n\t"                                                                          \
     "add.u32 r2, r2, " EP_L16 ";\n\t"                   /* this lane's 16 bytes of the chunk */                \
     "sub.s32 r3, r1, r2;\n\t"                                                                                  \
     "min.s32 r3, r3, 16;\n\t"                                                                                  \
@@ -890,15 +918,15 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     "setp.gt.s32 pv, r3, 0;\n\t"                                                                               \
     "selp.b32 r2, r2, 0, pv;\n\t"                                                                              \
     "mad.wide.u32 rb, r2, 1, ra;\n\t"                                                                          \
-    "mad.lo.u32 r2, r4, 512, r10;\n\t"                                                                         \
+    "mad.lo.u32 r2, r4, " EP_CBYTES ", r10;\n\t"                                                               \
     "add.u32 r2, r2, " EP_L16 ";\n\t"                                                                          \
-    "cp.async.cg.shared.global [r2], [rb], 16, r3;\n\t"                                                        \
-    "setp.eq.u32 pv, r4, 0;\n\t"                                                                               \
-    "@pv cp.async.cg.shared.global [r2+1536], [rb], 16, r3;\n\t"                                               \
+    "@pl cp.async.cg.shared.global [r2], [rb], 16, r3;\n\t"                                                    \
+    "setp.lt.and.u32 pv, r4, " EP_MSLOT ", pl;\n\t"                                                            \
+    "@pv cp.async.cg.shared.global [r2+" EP_RBYTES "], [rb], 16, r3;\n\t"                                      \
     "cp.async.commit_group;\n\t"                                                                               \
     "add.u32 r9, r9, 1;\n\t"                                                                                   \
     "add.u32 r4, r4, 1;\n\t"                                                                                   \
-    "setp.eq.u32 pv, r4, 3;\n\t"                                                                               \
+    "setp.eq.u32 pv, r4, " EP_NSLOT ";\n\t"                                                                    \
     "selp.b32 r4, 0, r4, pv;\n\t"                                                                              \
     "sub.u32 r0, r0, 1;\n\t"                                                                                   \
     "setp.ne.u32 pq, r0, 0;\n\t"                                                                               \
@@ -908,14 +936,14 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     "EP_SVW_" S ":\n\t"                                                                                        \
     "cp.async.wait_group 1;\n\t"                                                                               \
     "bar.warp.sync 0xffffffff;\n\t"                                                                            \
-    "sub.u32 r2, wthr" S ", r10;\n\t"                   /* 510 + ring offset of the cursor's old chunk */      \
+    "sub.u32 r2, wthr" S ", r10;\n\t"                   /* chunk size - 2 + ring offset of the cursor's old chunk */ \
     "add.u32 r2, r2, r8;\n\t"                                                                                  \
-    "setp.ge.u32 pv, r2, 2046;\n\t"                     /* past the third slot: back to the first */           \
-    "@pv sub.u32 r2, r2, 1536;\n\t"                                                                            \
+    "setp.ge.u32 pv, r2, " EP_RWRAP ";\n\t"             /* past the last slot: back to the first */            \
+    "@pv sub.u32 r2, r2, " EP_RBYTES ";\n\t"                                                                   \
     "add.u32 wthr" S ", r2, r10;\n\t"                                                                          \
-    "and.b32 r3, r7, 511;\n\t"                                                                                 \
+    "and.b32 r3, r7, " EP_CMASK ";\n\t"                                                                        \
     "add.u32 r2, wthr" S ", r3;\n\t"                                                                           \
-    "sub.u32 r2, r2, 510;\n\t"                          /* the cursor's new address */                         \
+    "sub.u32 r2, r2, " EP_COFF ";\n\t"                  /* the cursor's new address */                         \
     "sub.u32 r3, r6, r2;\n\t"                                                                                  \
     "sub.u32 " AW ", " AW ", r3;\n\t"                                                                          \
     "sub.u32 r5, r5, r3;\n\t"                                                                                  \
@@ -942,7 +970,7 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     asm volatile(                                                                                                     \
         "{\n\t"                                                                                                       \
         EP_ALL(EP_REGS)                                                                                               \
-        ".reg .pred pq, pv, pr;\n\t"                                                                                  \
+        ".reg .pred pq, pv, pr, pl;\n\t"                                                                                  \
         ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, f0c, m21, m11, hotb;\n\t"         \
         ".reg .b64 ra, rb;\n\t"                                                                                       \
         ".reg .f32 k0f, k1f;\n\t"                                                                                     \
@@ -1102,8 +1130,11 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
             const uint32_t base = r * kTilesPerRound + kChains * warp;
             if constexpr (DT != EP_FIELDS_I32) {
                 if (fast) {
-                    if (J.b == 12u) decode_tiles_fast<DT, 12>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
-                    else decode_tiles_fast<DT, 11>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    if (kTwoLevelInLoop && J.b == 12u) {
+                        if constexpr (kTwoLevelInLoop) decode_tiles_fast<DT, 12>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    } else {
+                        decode_tiles_fast<DT, 11>(J, base, lut_addr, cf, ring, ctx, lane, tables_pending);
+                    }
                     tables_pending = false;
                     continue;
                 }
