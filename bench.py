@@ -284,6 +284,9 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import oracle
+    if os.environ.get("WORLD_SIZE") is not None:
+        # a launcher pins OMP_NUM_THREADS to 1 for its ranks; this arm runs on rank 0 alone, so give it the host's cores
+        oracle.set_threads(os.cpu_count() or 1)
     probe_rows = 64
     name, dtype_name, bpp, layers, shapes = make_workload(args, rows=probe_rows)
     vmax = oracle.default_tile_vectors(bpp)
