@@ -49,45 +49,23 @@ constexpr uint32_t kLutEntries = 2048;                       // 2^11 slots per t
 constexpr uint32_t kLutStride = kLutEntries * 4;             // bytes per table in shared memory
 constexpr uint32_t kCosetStride = 8 * kLutStride;            // the eight tables of coset 1 follow those of coset 0
 constexpr uint32_t kLutBytes = 16 * kLutStride;              // 131072
-// Payload ring of a chain: kRingSlots chunks of kChunk bytes plus a mirror of its first 512 bytes.  A chunk is one
-// cp.async round of a warp (16 bytes per lane: all 32 lanes for 512 bytes, the first 16 for 256).  With one tile
-// per warp the ring has three 512-byte chunks; two tiles per warp and 32 warps (64 rings in what the tables leave of
-// the shared memory) get four 256-byte chunks each, refilled twice as often.
-#if EP_CHAINS * EP_WARPS > 48
-#define EP_SMALL_RINGS 1
-constexpr uint32_t kChunk = 256, kRingSlots = 4, kMirrorSlots = 2;
-#define EP_CSH "8"          /* log2 of the chunk size */
-#define EP_CMASK "255"      /* chunk size - 1 */
-#define EP_COFF "254"       /* chunk size - 2: the cursor is about to leave its chunk at chunk start + this */
-#define EP_CBYTES "256"
-#define EP_RBYTES "1024"    /* ring size */
-#define EP_RWRAP "1278"     /* ring size + chunk size - 2 */
-#define EP_NSLOT "4"
-#define EP_MSLOT "2"        /* chunks whose slot is below this are written to the mirror too */
-#else
+// Payload ring of a chain: three chunks of 512 bytes (one cp.async round of a warp, 16 bytes per lane) plus a mirror
+// of its first 512 bytes.  (Measured and dropped: 64 rings of four 256-byte chunks for two tiles per warp at 32 warps.)
 constexpr uint32_t kChunk = 512, kRingSlots = 3, kMirrorSlots = 1;
-#define EP_CSH "9"
-#define EP_CMASK "511"
-#define EP_COFF "510"
-#define EP_CBYTES "512"
-#define EP_RBYTES "1536"
-#define EP_RWRAP "2046"
-#define EP_NSLOT "3"
-#define EP_MSLOT "1"
-#endif
 constexpr uint32_t kChunkLanes = kChunk / 16;                // lanes that take part in a chunk's copy
-constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536 or 1024
+constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536
 constexpr uint32_t kRingMirror = 512;                        // >= 7 words * 32 lanes * 2 bytes + one lane span (62)
-constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 or 1536 per chain
+constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 per chain
 constexpr uint32_t kCtxBytes = 32 + 32 * kChains;            // per warp: what the rare paths of the hot loop need
 constexpr uint32_t kRingBase = kLutBytes;
 constexpr uint32_t kCtxBase = kRingBase + kWarps * kChains * kRingStride;
-// 2^12-slot streams: the symbols within kHotSpan of each table's most frequent one have their entry of the symbol
-// array in shared memory (the rest is read from global memory); this fills what the tables, rings and context
-// blocks of the 32-warp build leave of the 227 KB
-constexpr uint32_t kHotSpan = 264;
-constexpr uint32_t kHotEntries = 16 * kHotSpan;              // 4224: image values below this are hot indices
-constexpr uint32_t kHotBytes = kHotEntries * 8;              // 33792
+// 2^12-slot streams: per table, the entries of the kHotSpan coordinate values around zero are kept in shared memory
+// (the rest is read from global memory); this fills what the tables, rings and context blocks of the 32-warp build
+// leave of the 227 KB
+constexpr uint32_t kHotSpan = 528;                           // coordinate codes per table in the hot window
+constexpr uint32_t kHotBytes = 16 * kHotSpan * 4;            // 33792
+constexpr uint32_t kColdCodes = 4096;                        // codes per table in the complete entry array (global memory)
+constexpr uint32_t kColdBytes = 16 * kColdCodes * 4;         // 262144
 constexpr uint32_t kHotBase = kCtxBase + kWarps * kCtxBytes;
 constexpr bool kTwoLevelInLoop = EP_CHAINS == 1 && kHotBase + kHotBytes <= 232448;
 constexpr uint32_t kSmemBytes = kHotBase + (kTwoLevelInLoop ? kHotBytes : 0);   // 232448 in the default build
@@ -105,13 +83,12 @@ constexpr uint32_t kCtxMul21 = 16;         // u32 2^21 and
 constexpr uint32_t kCtxMul11 = 20;         // u32 2^11: multipliers the hot loop must not see as constants (see EP_STEP)
 constexpr uint32_t kCtxRowRcp = 24;        // u32 ceil(2^32 / bytes per row)
 constexpr uint32_t kCtxChain = 32, kCtxChainStride = 32;
-constexpr uint32_t kCcA0 = 0;              // u64 global address of chunk 0 (first payload byte rounded down to 16)
-constexpr uint32_t kCcRoom = 8;            // u32 bytes from a0 to the end of the payload
-constexpr uint32_t kCcNext = 12;           // u32 next chunk to request
-constexpr uint32_t kCcNextSlot = 16;       // u32 the ring slot it goes to (chunk number mod 3)
+constexpr uint32_t kCcSrc = 0;             // u64 global address of lane 0's 16 bytes of the next chunk to request
+constexpr uint32_t kCcRem = 8;             // s32 payload bytes from there to the end of the payload (may be <= 0)
+constexpr uint32_t kCcDst = 12;            // u32 ring address of lane 0's 16 bytes of that chunk's slot
+constexpr uint32_t kCcRing = 16;           // u32 ring base (shared-memory address)
 constexpr uint32_t kCcWbase = 20;          // u32 ring address of byte position 0 (cursor address minus position)
 constexpr uint32_t kCcEndo = 24;           // u32 output byte offset after the tile's last block
-constexpr uint32_t kCcRing = 28;           // u32 ring base (shared-memory address)
 
 __device__ unsigned int g_ep_status = 0;
 
@@ -122,8 +99,8 @@ struct JobParams {
     void *out;
     const uint32_t *lut_image;    // 128 KB table image from ep_prepare_tables / the table-build launch, or null: build the
                                   // tables here (b <= 11 only)
-    const uint2 *l2;              // b = 12: the symbol array behind the image's 16-bit indices, and
-    uint32_t l2max;               //         its last index
+    const uint32_t *cold;         // b = 12: entries of all codes of the sixteen coordinate tables, and
+    uint32_t hs2;                 //         twice the first code of the hot window
     uint32_t off_freq;            // byte offset of the u16 frequency arrays inside the blob
     uint32_t off_payload;
     uint32_t total_words;
@@ -284,7 +261,7 @@ __device__ __forceinline__ void build_tables_smem(const JobParams &J, uint32_t l
 __device__ __forceinline__ void copy_tables_smem(const uint32_t *image, uint32_t lut_addr, bool two_level) {
     const uint64_t src = reinterpret_cast<uint64_t>(image);
     for (uint32_t o = 16u * threadIdx.x; o < kLutBytes; o += 16u * kThreads) cp_async16(lut_addr + o, src + o, 16);
-    if (kTwoLevelInLoop && two_level)        // the hot part of the symbol array follows the image
+    if (kTwoLevelInLoop && two_level)        // the hot part of the second level follows the image
         for (uint32_t o = 16u * threadIdx.x; o < kHotBytes; o += 16u * kThreads)
             cp_async16(lut_addr + kHotBase + o, src + kLutBytes + o, 16);
     cp_async_commit();
@@ -582,7 +559,7 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F1 "%11"
 #define EP_L16 "%12"
 #define EP_L2B "%13"
-#define EP_KMAX "%14"
+#define EP_HS2 "%14"
 #define EP_HOTOFF "%15"
 #elif EP_CHAINS == 2
 #define EP_LT "%8"     /* lanes below this one (mask) */
@@ -593,10 +570,10 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_OUT "%13"   /* output base address */
 #define EP_F0 "%14"    /* frequency of coset 0 */
 #define EP_F1 "%15"    /* frequency of coset 1, at least 1 */
-#define EP_L16 "%16"
-#define EP_L2B "%17"   /* level-2 table of the 2^12-slot streams (global) */
-#define EP_KMAX "%18"
-#define EP_HOTOFF "%19"  /* its last index */   /* 16 * lane */
+#define EP_L16 "%16"   /* 16 * lane */
+#define EP_L2B "%17"   /* 2^12-slot streams: the complete second-level array (global memory), */
+#define EP_HS2 "%18"   /* twice the first code of the hot window, */
+#define EP_HOTOFF "%19"  /* offset of the hot part in shared memory */
 #elif EP_CHAINS == 3
 #define EP_LT "%12"
 #define EP_LUT0 "%13"
@@ -608,7 +585,7 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F1 "%19"
 #define EP_L16 "%20"
 #define EP_L2B "%21"
-#define EP_KMAX "%22"
+#define EP_HS2 "%22"
 #define EP_HOTOFF "%23"
 #else
 #define EP_LT "%16"
@@ -621,7 +598,7 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_F1 "%23"
 #define EP_L16 "%24"
 #define EP_L2B "%25"
-#define EP_KMAX "%26"
+#define EP_HS2 "%26"
 #define EP_HOTOFF "%27"
 #endif
 // one macro call per chain: M(S = suffix, X, AW, BAL, DOFF, CB = byte offset of the chain's context, more...)
@@ -732,46 +709,50 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
 #define EP_ADDR(S, X, AW, BAL, DOFF, CB) "mad.wide.u32 ad" S ", " DOFF ", 1, " EP_OUT ";\n\t"
 
 // ---- streams with 2^12 slots per table (b = 12: the paper's setting for 8 bpp targets) ------------------------
-// Sixteen tables of 4096 four-byte entries would not fit shared memory, so the lookup has two levels: shared
-// memory holds, per slot, the 16-bit index of the slot's symbol in ONE array of all symbols of all tables (the
-// same 128 KB as the one-level tables of b = 11, same strides), and that array - its most frequent part in
-// shared memory too, all of it in global memory - holds per symbol
-//     word 0: [12:0] f   [15] lowest bit of the coordinate   [31:16] F        word 1: the lattice coordinate
-// z + c/2 (2m + c/2 for the m field) as fp32, so that Eq. 19 is one multiply.  XD = register that receives word 1.
-#define EP_M1(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "and.b32 u" S ", " X ", 0xFFF;\n\t"
-#define EP_M2(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "mad.lo.u32 t" S ", u" S ", 2, tab" S ";\n\t"
-#define EP_M3(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "ld.shared.u16 w" S ", [t" S "+" OFF "];\n\t"
-/* an index below 4224 is an entry of the hot part in shared memory, any other one (minus 4224) of the whole array */
-#define EP_M4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "setp.lt.u32 pc" S ", w" S ", 4224;\n\t"
-#define EP_M5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "mad.lo.u32 t" S ", w" S ", 8, hotb;\n\t"
-#define EP_M6(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) \
-    "sub.u32 w" S ", w" S ", 4224;\n\t" "min.u32 w" S ", w" S ", " EP_KMAX ";\n\t" "mad.wide.u32 ad" S ", w" S ", 8, " EP_L2B ";\n\t"
-#define EP_M7(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) \
-    "@pc" S " ld.shared.v2.u32 {" E S ", " XD S "}, [t" S "];\n\t" "@!pc" S " ld.global.nc.v2.u32 {" E S ", " XD S "}, [ad" S "];\n\t"
-#define EP_M8(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "shr.u32 q" S ", " X ", 12;\n\t" "and.b32 f" S ", " E S ", 0x1FFF;\n\t"
-#define EP_M9(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "shr.u32 bi" S ", " E S ", 16;\n\t"
-#define EP_M10(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "sub.u32 bi" S ", u" S ", bi" S ";\n\t"
-#define EP_M11(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, XD) "@act" S " mad.lo.u32 " X ", f" S ", q" S ", bi" S ";\n\t"
-#define EP_STEP12_ALL(E, OFF, BIN, BOUT, XD)                                                                     \
-    EP_ALL(EP_M1, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M2, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M3, E, OFF, BIN, BOUT, XD)   \
-    EP_ALL(EP_M4, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M5, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M6, E, OFF, BIN, BOUT, XD)   \
-    EP_ALL(EP_M7, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M8, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M9, E, OFF, BIN, BOUT, XD)   \
-    EP_ALL(EP_M10, E, OFF, BIN, BOUT, XD) EP_ALL(EP_M11, E, OFF, BIN, BOUT, XD) EP_RENORM_ALL(E, OFF, BIN, BOUT)
+// Sixteen tables of 4096 four-byte entries would not fit shared memory, so the lookup has two levels.  Shared memory
+// holds, per slot, 16 bits: twice the code of the slot's coordinate value, code = z - zlo (2m - zlo for the m field;
+// the same 128 KB and strides as the one-level tables of b = 11).  The code is all Eq. 5 needs - it goes into the
+// mantissa of 2^22 (bit 0 = the coset's half, bit 1 = one) - and it addresses the second level, one word per (table,
+// code): f << 16 | F.  Entries of the kHotSpan codes around zero sit in shared memory, all of them in global memory.
+// HOFF / COFF = byte offset of the field's table in the hot part / in the complete array.
+#define EP_N1(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "and.b32 u" S ", " X ", 0xFFF;\n\t"
+#define EP_N2(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "mad.lo.u32 t" S ", u" S ", 2, tab" S ";\n\t"
+#define EP_N3(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "ld.shared.u16 " E S ", [t" S "+" OFF "];\n\t"
+/* codes inside the hot window: entry in shared memory; the others: global memory */
+#define EP_N4(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "sub.u32 w" S ", " E S ", " EP_HS2 ";\n\t"
+#define EP_N5(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "setp.lt.u32 pc" S ", w" S ", 1056;\n\t"
+#define EP_N6(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "mad.lo.u32 t" S ", w" S ", 2, hotc" S ";\n\t"
+#define EP_N7(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "mad.wide.u32 ad" S ", " E S ", 2, lc" S ";\n\t"
+#define EP_N8(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) \
+    "@pc" S " ld.shared.u32 w" S ", [t" S "+" HOFF "];\n\t" "@!pc" S " ld.global.nc.u32 w" S ", [ad" S "+" COFF "];\n\t"
+#define EP_N9(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "shr.u32 q" S ", " X ", 12;\n\t"
+#define EP_N10(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "shr.u32 f" S ", w" S ", 16;\n\t"
+#define EP_N11(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "and.b32 bi" S ", w" S ", 0xFFFF;\n\t"
+#define EP_N12(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "sub.u32 bi" S ", u" S ", bi" S ";\n\t"
+#define EP_N13(S, X, AW, BAL, DOFF, CB, E, OFF, BIN, BOUT, HOFF, COFF) "@act" S " mad.lo.u32 " X ", f" S ", q" S ", bi" S ";\n\t"
+#define EP_STEP12_ALL(E, OFF, BIN, BOUT, HOFF, COFF)                                                             \
+    EP_ALL(EP_N1, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N2, E, OFF, BIN, BOUT, HOFF, COFF)                    \
+    EP_ALL(EP_N3, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N4, E, OFF, BIN, BOUT, HOFF, COFF)                    \
+    EP_ALL(EP_N5, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N6, E, OFF, BIN, BOUT, HOFF, COFF)                    \
+    EP_ALL(EP_N7, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N8, E, OFF, BIN, BOUT, HOFF, COFF)                    \
+    EP_ALL(EP_N9, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N10, E, OFF, BIN, BOUT, HOFF, COFF)                   \
+    EP_ALL(EP_N11, E, OFF, BIN, BOUT, HOFF, COFF) EP_ALL(EP_N12, E, OFF, BIN, BOUT, HOFF, COFF)                  \
+    EP_ALL(EP_N13, E, OFF, BIN, BOUT, HOFF, COFF) EP_RENORM_ALL(E, OFF, BIN, BOUT)
 #define EP_C1_12(S, X, AW, BAL, DOFF, CB) "and.b32 u" S ", " X ", 0xFFF;\n\t"
 #define EP_C2_12(S, X, AW, BAL, DOFF, CB) "shr.u32 q" S ", " X ", 12;\n\t"
+/* per coset: 2^22 (+ 1/2) as fp32, the hot part and the complete array of its eight tables */
+#define EP_C8_12(S, X, AW, BAL, DOFF, CB) "selp.b32 cc" S ", d0r, d1r, pc" S ";\n\t"
+#define EP_C9_12(S, X, AW, BAL, DOFF, CB) "selp.b32 hotc" S ", hotb, hotb1, pc" S ";\n\t"
+#define EP_C10_12(S, X, AW, BAL, DOFF, CB) "selp.b64 lc" S ", " EP_L2B ", l2b1, pc" S ";\n\t"
 #define EP_COSET12_ALL                                                                               \
     EP_ALL(EP_C1_12) EP_ALL(EP_C2_12) EP_ALL(EP_C3) EP_ALL(EP_C4) EP_ALL(EP_C5) EP_ALL(EP_C6) EP_ALL(EP_C7)  \
-    EP_RENORM_ALL("", "", BL, NA)
-#define EP_Q1(S, X, AW, BAL, DOFF, CB) "mov.b64 pr" S ", {xa" S ", xb" S "};\n\t"
-#define EP_Q2(S, X, AW, BAL, DOFF, CB) "mul.rn.f32x2 pr" S ", pr" S ", ss" S ";\n\t"
-#define EP_Q3(S, X, AW, BAL, DOFF, CB) "mov.b64 {wl" S ", wh" S "}, pr" S ";\n\t"
-#define EP_PAIR12_ALL EP_ALL(EP_Q1) EP_ALL(EP_Q2) EP_ALL(EP_Q3)
-// z8 = 2m + parity of (z1 + ... + z7): bit 15 of the xor of the first words, added to the m field's coordinate as 1.0
-#define EP_PAR12(S, X, AW, BAL, DOFF, CB)                                \
-    "and.b32 par" S ", par" S ", 0x8000;\n\t"                            \
-    "setp.ne.u32 pc" S ", par" S ", 0;\n\t"                              \
-    "selp.b32 par" S ", 0x3F800000, 0, pc" S ";\n\t"                     \
-    "add.rn.f32 xb" S ", xb" S ", par" S ";\n\t"
+    EP_ALL(EP_C8_12) EP_ALL(EP_C9_12) EP_ALL(EP_C10_12) EP_RENORM_ALL("", "", BL, NA)
+// Eq. 5: 2^22 + code (+ 1/2) as fp32; z8 = 2m + parity of (z1 + ... + z7), the parity from bit 1 of the xor of the
+// looked-up values (zlo is even)
+#define EP_XA12(S, X, AW, BAL, DOFF, CB, E) "or.b32 xa" S ", " E S ", cc" S ";\n\t"
+#define EP_XB12(S, X, AW, BAL, DOFF, CB, E) "or.b32 xb" S ", " E S ", cc" S ";\n\t"
+#define EP_PARX12(S, X, AW, BAL, DOFF, CB) "lop3.b32 par" S ", par" S ", 0x2, cc" S ", 0xEA;\n\t"
+#define EP_X8_12(S, X, AW, BAL, DOFF, CB) "or.b32 xb" S ", e8" S ", par" S ";\n\t"
 // the nine steps and the arithmetic of one group, 2^11-slot and 2^12-slot streams
 #define EP_BODY11(CVT)                                                                                                \
         EP_COSET_ALL                                                                                                  \
@@ -785,14 +766,14 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
         EP_STEP_ALL("e8", "57344", NB, BL) EP_ALL(EP_PARX) EP_ALL(EP_X8) EP_PAIR_ALL EP_ALL(CVT, "3")
 #define EP_BODY12(CVT)                                                                                                \
         EP_COSET12_ALL                                                                                                \
-        EP_STEP12_ALL("e1", "0", NA, NB, "xa")                                                                        \
-        EP_STEP12_ALL("e2", "8192", NB, NA, "xb")  EP_PAIR12_ALL EP_ALL(CVT, "0")                                     \
-        EP_STEP12_ALL("e3", "16384", NA, NB, "xa") EP_ALL(EP_PAR3, "e1", "e2", "e3")                                  \
-        EP_STEP12_ALL("e4", "24576", NB, NA, "xb") EP_PAIR12_ALL EP_ALL(CVT, "1")                                     \
-        EP_STEP12_ALL("e5", "32768", NA, NB, "xa") EP_ALL(EP_PAR3, "par", "e4", "e5")                                 \
-        EP_STEP12_ALL("e6", "40960", NB, NA, "xb") EP_PAIR12_ALL EP_ALL(CVT, "2")                                     \
-        EP_STEP12_ALL("e7", "49152", NA, NB, "xa") EP_ALL(EP_PAR3, "par", "e6", "e7")                                 \
-        EP_STEP12_ALL("e8", "57344", NB, BL, "xb") EP_ALL(EP_PAR12) EP_PAIR12_ALL EP_ALL(CVT, "3")
+        EP_STEP12_ALL("e1", "0", NA, NB, "0", "0")             EP_ALL(EP_XA12, "e1")                                  \
+        EP_STEP12_ALL("e2", "8192", NB, NA, "2112", "16384")   EP_ALL(EP_XB12, "e2") EP_PAIR_ALL EP_ALL(CVT, "0")     \
+        EP_STEP12_ALL("e3", "16384", NA, NB, "4224", "32768")  EP_ALL(EP_PAR3, "e1", "e2", "e3") EP_ALL(EP_XA12, "e3") \
+        EP_STEP12_ALL("e4", "24576", NB, NA, "6336", "49152")  EP_ALL(EP_XB12, "e4") EP_PAIR_ALL EP_ALL(CVT, "1")     \
+        EP_STEP12_ALL("e5", "32768", NA, NB, "8448", "65536")  EP_ALL(EP_PAR3, "par", "e4", "e5") EP_ALL(EP_XA12, "e5") \
+        EP_STEP12_ALL("e6", "40960", NB, NA, "10560", "81920") EP_ALL(EP_XB12, "e6") EP_PAIR_ALL EP_ALL(CVT, "2")     \
+        EP_STEP12_ALL("e7", "49152", NA, NB, "12672", "98304") EP_ALL(EP_PAR3, "par", "e6", "e7") EP_ALL(EP_XA12, "e7") \
+        EP_STEP12_ALL("e8", "57344", NB, BL, "14784", "114688") EP_ALL(EP_PARX12) EP_ALL(EP_X8_12) EP_PAIR_ALL EP_ALL(CVT, "3")
 
 // per output type: CVT(S, j, lo, hi) turns weights 2j, 2j+1 into their stored form, STORE(S) writes the block
 #define EP_CVT_BF16(S, X, AW, BAL, DOFF, CB, J) "cvt.rn.bf16x2.f32 o" J S ", wh" S ", wl" S ";\n\t"
@@ -832,12 +813,12 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     ".reg .b32 o0" S ", o1" S ", o2" S ", o3" S ", ia0" S ", ib0" S ", ia1" S ", ib1" S ", ia2" S ", ib2" S ", ia3" S ", ib3" S ";\n\t" \
     ".reg .b16 h0" S ", h1" S ", h2" S ", h3" S ";\n\t"                                                              \
     ".reg .f32 wl" S ", wh" S ", sg" S ";\n\t"                                                                       \
-    ".reg .b32 lim" S ", wthr" S ";\n\t"                                                                             \
-    ".reg .b64 pr" S ", ss" S ", ad" S ", xw" S ";\n\t"
+    ".reg .b32 lim" S ", wthr" S ", hotc" S ";\n\t"                                                                  \
+    ".reg .b64 pr" S ", ss" S ", ad" S ", xw" S ", lc" S ";\n\t"
 // before the first pass: the cursor leaves its first chunk at ring + chunk size - 2; lim = 0 sends the chain through EP_ROWS
 #define EP_INIT(S, X, AW, BAL, DOFF, CB)                                 \
-    "ld.shared.u32 r0, [" EP_CTX "+" CB "+28];\n\t"                      \
-    "add.u32 wthr" S ", r0, " EP_COFF ";\n\t"                            \
+    "ld.shared.u32 r0, [" EP_CTX "+" CB "+16];\n\t"                      \
+    "add.u32 wthr" S ", r0, 510;\n\t"                                    \
     "mov.u32 lim" S ", 0;\n\t"
 
 #define EP_ADVANCE(S, X, AW, BAL, DOFF, CB, GROUP_BYTES) "add.u32 " DOFF ", " DOFF ", " GROUP_BYTES ";\n\t"
@@ -886,67 +867,50 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     "EP_ROWS_END_" S ":\n\t"
 #define EP_ANY_ACT(S, X, AW, BAL, DOFF, CB) "or.pred pr, pr, act" S ";\n\t"
 
-// the chain's cursor left its chunk: request the chunks up to (slots - 1) ahead of it (one, as a rule), wait for all
-// but the newest, move the addresses back by the ring's length when the cursor's chunk is the one in slot 0 again.
-// The chain's context is read with two 16-byte loads up front: one shared-memory round trip, not six.
+// The chain's cursor left its 512-byte chunk (a group takes at most 448 + 62 bytes, so it is in the next one):
+// request the chunk two ahead of the cursor's new one into the slot that became free, wait for all requests but
+// this newest one, and move every address back by the ring's length when the cursor's chunk is the one in slot 0
+// again.  The context keeps the request state ready to use: source address, bytes left, destination.
 #define EP_SERVICE(S, X, AW, BAL, DOFF, CB)                              \
     "setp.ge.u32 pr, " AW ", wthr" S ";\n\t"                                                                   \
     "vote.sync.any.pred pr, pr, 0xffffffff;\n\t"                                                               \
     "@!pr bra.uni EP_SVC_END_" S ";\n\t"                                                                       \
-    "ld.shared.v4.u32 {r4, r5, r2, r10}, [" EP_CTX "+" CB "+16];\n\t" /* next slot, wbase, -, ring base */    \
-    "ld.shared.v4.u32 {r11, r12, r1, r9}, [" EP_CTX "+" CB "];\n\t"   /* chunk 0 address, room, next chunk */ \
     "shfl.sync.idx.b32 r6, " AW ", 0, 31, 0xffffffff;\n\t"                                                     \
     "popc.b32 r0, " BAL ";\n\t"                                                                                \
     "mad.lo.u32 r6, r0, 2, r6;\n\t"                     /* the cursor's address */                             \
-    "sub.u32 r7, r6, r5;\n\t"                           /* its byte position */                                \
-    "shr.u32 r8, r7, " EP_CSH ";\n\t"                   /* its chunk */                                        \
-    "add.u32 r0, r8, " EP_NSLOT ";\n\t"                                                                        \
-    "sub.s32 r0, r0, r9;\n\t"                           /* chunks the cursor has advanced: requests due */     \
-    "min.s32 r0, r0, " EP_NSLOT ";\n\t"                                                                        \
-    "max.s32 r0, r0, 0;\n\t"                                                                                   \
-    "shl.b32 r8, r0, " EP_CSH ";\n\t"                   /* bytes the cursor's chunk moves on in the ring */    \
-    "setp.eq.u32 pq, r0, 0;\n\t"                                                                               \
-    "@pq bra.uni EP_SVW_" S ";\n\t"                                                                            \
+    "add.u32 r0, wthr" S ", 2;\n\t"                     /* end of the chunk it was in */                       \
+    "setp.lt.u32 pq, r6, r0;\n\t"                                                                              \
+    "@pq bra.uni EP_SVC_END_" S ";\n\t"                 /* (a lane address ran ahead of the cursor: not yet) */ \
+    "ld.shared.v4.u32 {r11, r12, r1, r2}, [" EP_CTX "+" CB "];\n\t"  /* source, bytes left, destination */     \
+    "ld.shared.u32 r10, [" EP_CTX "+" CB "+16];\n\t"    /* ring base */                                        \
     "mov.b64 ra, {r11, r12};\n\t"                                                                              \
-    "setp.lt.u32 pl, " EP_L16 ", " EP_CBYTES ";\n\t"    /* lanes that copy 16 bytes of a chunk */              \
-    "EP_SVL_" S ":\n\t"                                                                                        \
-    "shl.b32 r2, r9, " EP_CSH ";\n\t"                                                                          \
-    "add.u32 r2, r2, " EP_L16 ";\n\t"                   /* this lane's 16 bytes of the chunk */                \
-    "sub.s32 r3, r1, r2;\n\t"                                                                                  \
-    "min.s32 r3, r3, 16;\n\t"                                                                                  \
-    "max.s32 r3, r3, 0;\n\t"                            /* bytes of them inside the payload */                 \
-    "setp.gt.s32 pv, r3, 0;\n\t"                                                                               \
-    "selp.b32 r2, r2, 0, pv;\n\t"                                                                              \
-    "mad.wide.u32 rb, r2, 1, ra;\n\t"                                                                          \
-    "mad.lo.u32 r2, r4, " EP_CBYTES ", r10;\n\t"                                                               \
-    "add.u32 r2, r2, " EP_L16 ";\n\t"                                                                          \
-    "@pl cp.async.cg.shared.global [r2], [rb], 16, r3;\n\t"                                                    \
-    "setp.lt.and.u32 pv, r4, " EP_MSLOT ", pl;\n\t"                                                            \
-    "@pv cp.async.cg.shared.global [r2+" EP_RBYTES "], [rb], 16, r3;\n\t"                                      \
+    "sub.s32 r3, r1, " EP_L16 ";\n\t"                                                                          \
+    "min.s32 r3, r3, 16;\n\t"                           /* bytes of this lane's 16 inside the payload */       \
+    "setp.gt.s32 pv, r3, 0;\n\t"                        /* none: no request (nothing valid reads them) */      \
+    "mad.wide.u32 rb, " EP_L16 ", 1, ra;\n\t"                                                                  \
+    "add.u32 r5, r2, " EP_L16 ";\n\t"                                                                          \
+    "@pv cp.async.cg.shared.global [r5], [rb], 16, r3;\n\t"                                                    \
+    "setp.eq.and.u32 pq, r2, r10, pv;\n\t"              /* slot 0 is written to the mirror as well */          \
+    "@pq cp.async.cg.shared.global [r5+1536], [rb], 16, r3;\n\t"                                               \
     "cp.async.commit_group;\n\t"                                                                               \
-    "add.u32 r9, r9, 1;\n\t"                                                                                   \
-    "add.u32 r4, r4, 1;\n\t"                                                                                   \
-    "setp.eq.u32 pv, r4, " EP_NSLOT ";\n\t"                                                                    \
-    "selp.b32 r4, 0, r4, pv;\n\t"                                                                              \
-    "sub.u32 r0, r0, 1;\n\t"                                                                                   \
-    "setp.ne.u32 pq, r0, 0;\n\t"                                                                               \
-    "@pq bra.uni EP_SVL_" S ";\n\t"                                                                            \
-    "st.shared.u32 [" EP_CTX "+" CB "+12], r9;\n\t"                                                            \
-    "st.shared.u32 [" EP_CTX "+" CB "+16], r4;\n\t"                                                            \
-    "EP_SVW_" S ":\n\t"                                                                                        \
+    "add.cc.u32 r11, r11, 512;\n\t"                                                                            \
+    "addc.u32 r12, r12, 0;\n\t"                                                                                \
+    "sub.s32 r1, r1, 512;\n\t"                                                                                 \
+    "add.u32 r2, r2, 512;\n\t"                                                                                 \
+    "sub.u32 r4, r2, r10;\n\t"                                                                                 \
+    "setp.ge.u32 pv, r4, 1536;\n\t"                                                                            \
+    "selp.b32 r2, r10, r2, pv;\n\t"                                                                            \
+    "st.shared.v4.u32 [" EP_CTX "+" CB "], {r11, r12, r1, r2};\n\t"                                            \
     "cp.async.wait_group 1;\n\t"                                                                               \
     "bar.warp.sync 0xffffffff;\n\t"                                                                            \
-    "sub.u32 r2, wthr" S ", r10;\n\t"                   /* chunk size - 2 + ring offset of the cursor's old chunk */ \
-    "add.u32 r2, r2, r8;\n\t"                                                                                  \
-    "setp.ge.u32 pv, r2, " EP_RWRAP ";\n\t"             /* past the last slot: back to the first */            \
-    "@pv sub.u32 r2, r2, " EP_RBYTES ";\n\t"                                                                   \
-    "add.u32 wthr" S ", r2, r10;\n\t"                                                                          \
-    "and.b32 r3, r7, " EP_CMASK ";\n\t"                                                                        \
-    "add.u32 r2, wthr" S ", r3;\n\t"                                                                           \
-    "sub.u32 r2, r2, " EP_COFF ";\n\t"                  /* the cursor's new address */                         \
-    "sub.u32 r3, r6, r2;\n\t"                                                                                  \
-    "sub.u32 " AW ", " AW ", r3;\n\t"                                                                          \
-    "sub.u32 r5, r5, r3;\n\t"                                                                                  \
+    "add.u32 wthr" S ", wthr" S ", 512;\n\t"            /* the cursor's chunk is the next slot's */            \
+    "sub.u32 r4, wthr" S ", r10;\n\t"                                                                          \
+    "setp.lt.u32 pq, r4, 2046;\n\t"                                                                            \
+    "@pq bra.uni EP_SVC_END_" S ";\n\t"                                                                        \
+    "sub.u32 wthr" S ", wthr" S ", 1536;\n\t"           /* past the third slot: everything back by the ring */ \
+    "sub.u32 " AW ", " AW ", 1536;\n\t"                                                                        \
+    "ld.shared.u32 r5, [" EP_CTX "+" CB "+20];\n\t"                                                            \
+    "sub.u32 r5, r5, 1536;\n\t"                                                                                \
     "st.shared.u32 [" EP_CTX "+" CB "+20], r5;\n\t"                                                            \
     "EP_SVC_END_" S ":\n\t"
 
@@ -970,15 +934,19 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
     asm volatile(                                                                                                     \
         "{\n\t"                                                                                                       \
         EP_ALL(EP_REGS)                                                                                               \
-        ".reg .pred pq, pv, pr, pl;\n\t"                                                                                  \
-        ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, f0c, m21, m11, hotb;\n\t"         \
-        ".reg .b64 ra, rb;\n\t"                                                                                       \
+        ".reg .pred pq, pv, pr;\n\t"                                                                                  \
+        ".reg .b32 r0, r1, r2, r3, r4, r5, r6, r7, r8, r9, r10, r11, r12, c0r, c1r, d0r, d1r, f0c, m21, m11, hotb, hotb1;\n\t" \
+        ".reg .b64 ra, rb, l2b1;\n\t"                                                                                 \
         ".reg .f32 k0f, k1f;\n\t"                                                                                     \
         "mov.b64 {k0f, k1f}, " EP_KK ";\n\t"                                                                          \
         "mov.b32 c0r, 0x45800000;\n\t"                                                                                \
         "mov.b32 c1r, 0x45800400;\n\t"                                                                                \
+        "mov.b32 d0r, 0x4A800000;\n\t"                /* 2^22, 2^22 + 1/2 (2^12-slot streams) */                    \
+        "mov.b32 d1r, 0x4A800001;\n\t"                                                                                \
         "max.u32 f0c, " EP_F0 ", 1;\n\t"                /* frequency used for coset 0: never 0 */                     \
-        "add.u32 hotb, " EP_LUT0 ", " EP_HOTOFF ";\n\t"           /* hot part of the symbol array (2^12-slot streams) */         \
+        "add.u32 hotb, " EP_LUT0 ", " EP_HOTOFF ";\n\t"   /* 2^12-slot streams: hot entries of coset 0, */              \
+        "add.u32 hotb1, hotb, 16896;\n\t"                 /* of coset 1; complete array of coset 1 */                   \
+        "add.s64 l2b1, " EP_L2B ", 131072;\n\t"                                                                       \
         "ld.shared.v2.u32 {m21, m11}, [" EP_CTX "+16];\n\t" /* 2^21, 2^11 */                                          \
         EP_ALL(EP_INIT)                                                                                               \
         "bra.uni EP_RARE;\n\t"                                                                                        \
@@ -1003,7 +971,7 @@ __device__ __forceinline__ void decode_tile_plain(const JobParams &J, uint32_t t
         /* every read-write operand is early-clobber: the loop reads the inputs after it has updated them */         \
         EP_LOOP_OPERANDS                                                                                              \
         : "r"(lt), "r"(lut_addr), "r"(lut_addr + kCosetStride), "r"(ctx), "l"(kk), "l"(out_base), "r"(cf.f0),         \
-          "r"(cf.f1), "r"(lane16), "l"(l2base), "r"(l2max), "n"(kHotBase)                                             \
+          "r"(cf.f1), "r"(lane16), "l"(l2base), "r"(hs2), "n"(kHotBase)                                             \
         : "memory")
 
 // kChains tiles of a tensor whose rows hold at least 32 blocks and whose tables have 2^B slots (B = 11: one-level
@@ -1027,14 +995,13 @@ __device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t f
         const uint32_t rg = ring + c * kRingStride, cctx = ctx + kCtxChain + c * kCtxChainStride;
         const TileSetup T = tile_setup(J, tile, valid[c], lane);
         for (uint32_t k = 0; k < kRingSlots; ++k) ring_issue(rg, T.a0, T.room, k, lane);
-        if (lane == 0) {
-            sts64(cctx + kCcA0, T.a0);
-            sts32(cctx + kCcRoom, T.room);
-            sts32(cctx + kCcNext, kRingSlots);
-            sts32(cctx + kCcNextSlot, 0u);
+        if (lane == 0) {                 // the next request is chunk 3, into slot 0
+            sts64(cctx + kCcSrc, T.a0 + kRingBytes);
+            sts32(cctx + kCcRem, T.room - kRingBytes);
+            sts32(cctx + kCcDst, rg);
+            sts32(cctx + kCcRing, rg);
             sts32(cctx + kCcWbase, rg);
             sts32(cctx + kCcEndo, (T.v0 + T.nv) * BB);
-            sts32(cctx + kCcRing, rg);
         }
         x[c] = T.x; a[c] = rg + T.lead; bal[c] = 0; doff[c] = (T.v0 + lane) * BB;
         off[c] = T.off; end[c] = T.end; lead[c] = T.lead;
@@ -1042,11 +1009,11 @@ __device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t f
     cp_async_wait<1>();           // all but the last chain's third chunk have landed (and the table image, if any)
     __syncwarp();
     if (tables_pending) __syncthreads();
-    const uint32_t k0 = __float_as_uint(float(4096 - J.zlo));
+    const uint32_t k0 = __float_as_uint(float((B == 11 ? 4096 : 4194304) - J.zlo));
     const uint64_t kk = pack64(k0, k0);
     const uint64_t out_base = reinterpret_cast<uint64_t>(J.out);
-    const uint64_t l2base = reinterpret_cast<uint64_t>(J.l2);
-    const uint32_t l2max = J.l2max;
+    const uint64_t l2base = reinterpret_cast<uint64_t>(J.cold);
+    const uint32_t hs2 = J.hs2;
     if constexpr (B == 11) {
         if constexpr (DT == EP_BF16) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_BF16, EP_ST_16, 512);
         else if constexpr (DT == EP_FP16) EP_TILES_LOOP_ASM(EP_BODY11, EP_CVT_FP16, EP_ST_16, 512);
@@ -1180,10 +1147,11 @@ struct GJobParams {
     uint16_t tK[EP_NUM_TABLES];
     uint32_t foff[EP_NUM_TABLES]; // start of table t's frequencies, in u16 units
     // two-level tables of a 2^12-slot stream (ep_build_tables12_kernel only)
-    uint16_t *image;              // 16 x 4096 symbol indices
-    uint2 *hot;                   // 16 x kHotSpan entries: the hot part
-    uint2 *l2;                    // all symbols of the sixteen coordinate tables
-    uint32_t symoff[EP_NUM_TABLES];   // first index of table t's symbols in l2
+    uint16_t *image;              // 16 x 4096 slots: twice the coordinate code
+    uint32_t *hot;                // 16 x kHotSpan entries: the codes hs .. hs + kHotSpan - 1
+    uint32_t *cold;               // 16 x kColdCodes entries: every code
+    int32_t zlo;                  // coordinate value of code 0 (even)
+    uint32_t hs;                  // first code of the hot window
 };
 
 struct GBatchParams {
@@ -1236,75 +1204,65 @@ __global__ void __launch_bounds__(1024) ep_build_tables_kernel(const __grid_cons
     }
 }
 
-// Two-level tables of a 2^12-slot stream (see EP_M1): one CTA per (coordinate table, job).  Prefix sums of the
-// frequencies as above; every symbol writes its entry of the symbol array - and, if it lies within the window of
-// kHotSpan symbols around the table's most frequent one, of the hot part that the decode kernel keeps in shared
-// memory -, every slot finds its symbol by binary search and stores the symbol's index: below kHotEntries an index
-// into the hot part, else kHotEntries plus the index into the whole array.  A frequency is stored as at least 1
-// (a symbol that never occurs owns no slot; the floor only keeps a damaged stream from producing states that take
-// a word in every step).
+// Two-level tables of a 2^12-slot stream (see EP_N1): one CTA per (coordinate table, job).  Prefix sums of the
+// frequencies as above; then every code of the coordinate range gets its entry f << 16 | F in the complete array -
+// and in the hot part, if it lies in the window of kHotSpan codes that the decode kernel keeps in shared memory -,
+// and every slot finds its symbol by binary search and stores twice the symbol's code.  A code no symbol of the
+// table has, and a symbol that never occurs, get f = 1 (they own no slot; the floor only keeps a damaged stream
+// from producing states that take a word in every step).
 __global__ void __launch_bounds__(1024) ep_build_tables12_kernel(const __grid_constant__ GBatchParams P) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint32_t part[1024];
-    __shared__ uint32_t best[1024];
-    __shared__ uint32_t s_lo;
     const GJobParams &J = P.job[blockIdx.y];
     const uint32_t t = blockIdx.x + 1u, tid = threadIdx.x;
     const uint32_t K = J.tK[t];
     constexpr uint32_t M = 4096;
     uint16_t *image = J.image + size_t(t - 1u) * M;
-    uint2 *hot = J.hot + (t - 1u) * kHotSpan;
-    const uint2 unused = make_uint2(1u, 0u);                               // f = 1, F = 0, coordinate 0
-    for (uint32_t k = K + tid; k < kHotSpan; k += blockDim.x) hot[k] = unused;   // the part of the window no symbol fills
+    uint32_t *hot = J.hot + (t - 1u) * kHotSpan;
+    uint32_t *cold = J.cold + (t - 1u) * kColdCodes;
+    const uint32_t unused = 1u << 16;                                 // f = 1, F = 0
+    const bool is_m = ((t - 1u) & 7u) == 7u;                          // the m field: its coordinate is 2m (+ parity)
     if (K == 0) {
-        for (uint32_t u = tid; u < M; u += blockDim.x) image[u] = uint16_t((t - 1u) * kHotSpan);   // never looked up in a valid stream
+        for (uint32_t c = tid; c < kColdCodes; c += blockDim.x) cold[c] = unused;
+        for (uint32_t c = tid; c < kHotSpan; c += blockDim.x) hot[c] = unused;
+        for (uint32_t u = tid; u < M; u += blockDim.x) image[u] = 0;  // never looked up in a valid stream
         return;
     }
     const uint16_t *fq = reinterpret_cast<const uint16_t *>(J.stream + J.off_tables + 8 * EP_NUM_TABLES) + J.foff[t];
     uint16_t *F = reinterpret_cast<uint16_t *>(smem);              // K + 1 entries
     const uint32_t per = (K + blockDim.x - 1) / blockDim.x;
     const uint32_t j0 = min(tid * per, K), j1 = min(j0 + per, K);
-    uint32_t sum = 0, top = 0;                                     // top: (frequency << 16) | (65535 - index): first maximum wins
-    for (uint32_t j = j0; j < j1; ++j) {
-        const uint32_t f = fq[j];
-        sum += f;
-        top = max(top, (f << 16) | (65535u - j));
-    }
+    uint32_t sum = 0;
+    for (uint32_t j = j0; j < j1; ++j) sum += fq[j];
     part[tid] = sum;
-    best[tid] = top;
     __syncthreads();
     if (tid == 0) {
-        uint32_t run = 0, b = 0;
-        for (uint32_t i = 0; i < blockDim.x; ++i) { const uint32_t v = part[i]; part[i] = run; run += v; b = max(b, best[i]); }
+        uint32_t run = 0;
+        for (uint32_t i = 0; i < blockDim.x; ++i) { const uint32_t v = part[i]; part[i] = run; run += v; }
         F[K] = uint16_t(min(run, M));
-        const uint32_t mode = 65535u - (b & 0xFFFFu);
-        const uint32_t last = K > kHotSpan ? K - kHotSpan : 0u;   // the window lies inside the table
-        s_lo = min(mode > kHotSpan / 2 ? mode - kHotSpan / 2 : 0u, last);
     }
     __syncthreads();
-    const uint32_t lo_hot = s_lo;
-    const uint32_t coset = (t - 1u) >> 3, field = (t - 1u) & 7u;          // field 7 is m: its coordinate is 2m (+ parity)
-    uint2 *l2 = J.l2 + J.symoff[t];
     uint32_t run = part[tid];
-    for (uint32_t j = j0; j < j1; ++j) {
-        const uint32_t f = fq[j], Fj = min(run, M - 1u);
-        F[j] = uint16_t(min(run, M));
-        run += f;
-        const int32_t v = J.tmin[t] + int32_t(j);
-        const float coord = float(field == 7u ? 2 * v : v) + 0.5f * float(coset);
-        const uint32_t par = field == 7u ? 0u : uint32_t(v) & 1u;
-        const uint2 e = make_uint2(min(max(f, 1u), 8191u) | (par << 15) | (Fj << 16), __float_as_uint(coord));
-        l2[j] = e;
-        if (j - lo_hot < kHotSpan) hot[j - lo_hot] = e;           // (unsigned: j below the window wraps to a large number)
-    }
+    for (uint32_t j = j0; j < j1; ++j) { F[j] = uint16_t(min(run, M)); run += fq[j]; }
     __syncthreads();
+    for (uint32_t c = tid; c < kColdCodes; c += blockDim.x) {
+        const int32_t z = int32_t(c) + J.zlo;                         // the coordinate value of this code
+        const int32_t j = (is_m ? (z >> 1) : z) - J.tmin[t];          // (z even for the m field: the shift is exact)
+        uint32_t e = unused;
+        if (!(is_m && (z & 1)) && j >= 0 && uint32_t(j) < K)
+            e = (min(max(uint32_t(fq[j]), 1u), M) << 16) | min(uint32_t(F[j]), M - 1u);
+        cold[c] = e;
+        if (c - J.hs < kHotSpan) hot[c - J.hs] = e;                   // (unsigned: a code below the window wraps)
+    }
     for (uint32_t u = tid; u < M; u += blockDim.x) {
         uint32_t lo = 0, hi = K;                                     // largest j with F[j] <= u (F[0] = 0)
         while (hi - lo > 1) {
             const uint32_t mid = (lo + hi) >> 1;
             if (uint32_t(F[mid]) <= u) lo = mid; else hi = mid;
         }
-        image[u] = uint16_t(lo - lo_hot < kHotSpan ? (t - 1u) * kHotSpan + (lo - lo_hot) : kHotEntries + J.symoff[t] + lo);
+        const int32_t z = J.tmin[t] + int32_t(lo);
+        const int32_t code = (is_m ? 2 * z : z) - J.zlo;
+        image[u] = uint16_t(2 * min(max(code, 0), int32_t(kColdCodes) - 1));
     }
 }
 
@@ -1480,19 +1438,24 @@ cudaError_t launch_smem(const BatchParams &P, uint32_t grid, cudaStream_t st) {
 
 size_t large_table_bytes(const ep_info &I) { return size_t(EP_NUM_TABLES) * (size_t(1) << I.b) * 4u; }
 
-// 2^12-slot streams whose symbols can be numbered with 16 bits decode from two-level tables in the hot loop
-uint32_t coord_symbols(const ep_info &I) {
-    uint64_t k = 0;
-    for (int t = 1; t < EP_NUM_TABLES; ++t) k += I.table_K[t];
-    return uint32_t(k < 0xFFFFFFFFull ? k : 0xFFFFFFFFull);
-}
+// 2^12-slot streams whose coordinates span at most kColdCodes values decode from two-level tables in the hot loop
 bool fits_two_level(const ep_info &I) {
-    return kTwoLevelInLoop && I.b == 12 && coord_symbols(I) >= 1 && coord_symbols(I) <= 65535u - kHotEntries;
+    if (!kTwoLevelInLoop || I.b != 12) return false;
+    const Range r = coord_range(I);
+    const int64_t zlo = even_base(r);
+    return r.any && r.hi - zlo < int64_t(kColdCodes) && zlo >= -(int64_t(1) << 20);   // 2^22 - zlo and 2^22 + code: one exponent
 }
-// image, hot part, symbol array, rounded to 256 bytes; the flat tables of the large-table kernel follow at this offset
-size_t two_level_bytes(const ep_info &I) {
-    return (size_t(kLutBytes) + kHotBytes + 8u * size_t(coord_symbols(I)) + 255u) & ~size_t(255);
+// first code of the hot window: kHotSpan codes centred on the coordinate value 0, kept inside the code range
+uint32_t hot_start(const ep_info &I) {
+    const Range r = coord_range(I);
+    const int64_t zlo = even_base(r), codes = (r.any ? r.hi : 0) - zlo + 1;
+    const int64_t last = codes > int64_t(kHotSpan) ? codes - int64_t(kHotSpan) : 0;
+    int64_t hs = -zlo - int64_t(kHotSpan / 2);
+    if (hs < 0) hs = 0;
+    return uint32_t(hs < last ? hs : last);
 }
+// image, hot part, complete array; the flat tables of the large-table kernel follow at this offset
+size_t two_level_bytes(const ep_info &) { return size_t(kLutBytes) + kHotBytes + kColdBytes; }
 // can the hot loop serve this request?  (the field dump and narrow tensors take the plain kernels)
 bool hot_loop_shape(const ep_info &I, int32_t dt) { return dt != EP_FIELDS_I32 && I.C / 8 >= 32u && I.V < (1u << 20); }
 
@@ -1526,10 +1489,10 @@ int fill_large_job(GJobParams &J, const ep_decode_job &jb, uint32_t *lut) {
 // where the two-level tables of a job live inside its table buffer
 void set_two_level(GJobParams &J, const ep_info &I, void *base) {
     J.image = static_cast<uint16_t *>(base);
-    J.hot = reinterpret_cast<uint2 *>(static_cast<uint8_t *>(base) + kLutBytes);
-    J.l2 = reinterpret_cast<uint2 *>(static_cast<uint8_t *>(base) + kLutBytes + kHotBytes);
-    uint32_t acc = 0;
-    for (int t = 1; t < EP_NUM_TABLES; ++t) { J.symoff[t] = acc; acc += I.table_K[t]; }
+    J.hot = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(base) + kLutBytes);
+    J.cold = reinterpret_cast<uint32_t *>(static_cast<uint8_t *>(base) + kLutBytes + kHotBytes);
+    J.zlo = int32_t(even_base(coord_range(I)));
+    J.hs = hot_start(I);
 }
 
 cudaError_t launch_build12(const GBatchParams &P, int n_jobs, cudaStream_t st) {
@@ -1744,8 +1707,8 @@ extern "C" int ep_decode_batch(const ep_decode_job *jobs_in, int32_t n_in, void 
                 set_two_level(G, I, base);
             }
             J.lut_image = static_cast<const uint32_t *>(base);
-            J.l2 = reinterpret_cast<const uint2 *>(static_cast<const uint8_t *>(base) + kLutBytes + kHotBytes);
-            J.l2max = coord_symbols(I) - 1u;
+            J.cold = reinterpret_cast<const uint32_t *>(static_cast<const uint8_t *>(base) + kLutBytes + kHotBytes);
+            J.hs2 = 2u * hot_start(I);
         }
         J.off_payload = I.off_payload;
         J.total_words = uint32_t(I.total_words);
