@@ -995,7 +995,10 @@ __device__ __forceinline__ void decode_tiles_fast(const JobParams &J, uint32_t f
         const uint32_t rg = ring + c * kRingStride, cctx = ctx + kCtxChain + c * kCtxChainStride;
         const TileSetup T = tile_setup(J, tile, valid[c], lane);
         for (uint32_t k = 0; k < kRingSlots; ++k) ring_issue(rg, T.a0, T.room, k, lane);
+        // the record of the tile this chain takes in the CTA's next round (132 bytes: two lines), into L2
+        if (lane < 2u && tile + kTilesPerRound < J.n_tiles) prefetch_l2(J.tile_index + size_t(tile + kTilesPerRound) * 33u + 32u * lane);
         if (lane == 0) {                 // the next request is chunk 3, into slot 0
+            prefetch_l2(J.scales + min(T.v0 / J.per_row, J.row_max));      // the first row scale the loop will ask for
             sts64(cctx + kCcSrc, T.a0 + kRingBytes);
             sts32(cctx + kCcRem, T.room - kRingBytes);
             sts32(cctx + kCcDst, rg);
@@ -1068,15 +1071,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
         const uint32_t r0 = min((a + J.round_cost - 1u) / J.round_cost, J.rounds);
         const uint32_t r1 = min((b + J.round_cost - 1u) / J.round_cost, J.rounds);
         if (r0 >= r1) continue;
-        {   // while the tables are set up, bring this warp's first tile records and the start of their payload into L2
-            const uint32_t t_first = J.tile0 + min(r0 * kTilesPerRound + kChains * warp, J.tile_cnt - 1u);
-            const uint32_t *rec = J.tile_index + size_t(t_first) * 33u;
-            if (lane < kChains + 1u) prefetch_l2(rec + 32u * lane);          // the warp's records span kChains + 1 lines
-            const uint32_t off = min(rec[32], J.total_words);
-            const uint64_t at = 2ull * off + 128u * lane;                      // 4 KB: the rings' first fill and more
-            if (at < 2ull * J.total_words) prefetch_l2(J.stream + J.off_payload + at);
-        }
         if (tables_in_use) __syncthreads();          // every warp is done with the previous job's tables
+        // the table image is requested first: the tiles' records and payload (two dependent reads of memory that no
+        // cache holds yet) are on their way while it arrives
         if (J.lut_image) copy_tables_smem(J.lut_image, lut_addr, J.b == 12u);
         else build_tables_smem(J, lut_addr, warp, lane);
         const CosetFreq cf = load_coset(J);

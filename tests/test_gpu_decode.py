@@ -219,9 +219,9 @@ def test_coordinate_range_up_to_1024_stays_on_the_shared_memory_path():
 
 
 def test_two_level_tables_of_2_to_the_12_slot_streams():
-    # b = 12 (the paper's setting for 8 bpp): slot -> symbol index in shared memory, symbol entries partly in shared
-    # memory (a window around each table's mode), partly in global memory.  Heavy-tailed rows put many symbols
-    # outside the windows; tensors wide enough for the hot loop, all output types, tile ranges, a batch.
+    # b = 12 (the paper's setting for 8 bpp): slot -> coordinate code in shared memory, one entry per (table, code),
+    # those of the 528 codes around zero in shared memory, all of them in global memory.  Heavy-tailed rows put many
+    # coordinates outside the window; tensors wide enough for the hot loop, all output types, tile ranges, a batch.
     W = synth.student_t_rows(192, 4096, 61)
     blob = ep.encode(W, 8.0)
     I = blob.info
@@ -240,14 +240,29 @@ def test_two_level_tables_of_2_to_the_12_slot_streams():
     torch.cuda.synchronize()
     ref = oracle.decode(blob.data, oracle.BF16)[0].reshape(-1)
     assert np.array_equal(_bits(part), ref[3 * I.V * 8:11 * I.V * 8])
-    # more symbols than 16-bit indices can number: the flat tables in global memory serve the stream
     rng = np.random.default_rng(64)
     n = 64 * 512 // 8
+    two = 16 * 4096 * 2 + 16 * 528 * 4 + 16 * 4096 * 4
     fields = np.zeros((n, 9), np.int32)
     fields[:, 0] = rng.integers(0, 2, n)
+    # nearly the widest coordinate range the two levels take (4096 values), uniformly filled: most lookups leave
+    # the window
+    fields[:, 1:8] = rng.integers(-2040, 2040, (n, 7))
+    fields[:, 8] = rng.integers(-1000, 1000, n)
+    full = ep.pack_fields(fields, 64, 512, 12, 64, np.full(64, 0.001, np.float32))
+    assert ep.decode_scratch_bytes(full.info) == two + flat
+    _check_all_types(full.data)
+    # coordinates on one side of zero (the window cannot be centred), one field constant (a lone symbol: f = 2^12)
+    fields[:, 1:8] = rng.integers(0, 1500, (n, 7))
+    fields[:, 3] = 7
+    fields[:, 8] = rng.integers(0, 40, n)
+    onesided = ep.pack_fields(fields, 64, 512, 12, 64, np.full(64, 0.001, np.float32))
+    assert onesided.info.table_K[3] == 1 and ep.decode_scratch_bytes(onesided.info) == two + flat
+    _check_all_types(onesided.data)
+    # a wider range than that: the flat tables in global memory serve the stream
     fields[:, 1:] = rng.integers(-2500, 2500, (n, 8))
     wide = ep.pack_fields(fields, 64, 512, 12, 64, np.full(64, 0.001, np.float32))
-    assert sum(wide.info.table_K[1:]) > 61311 and ep.decode_scratch_bytes(wide.info) == flat
+    assert ep.decode_scratch_bytes(wide.info) == flat
     _check_all_types(wide.data)
     assert ep.last_device_status() == 0
 
