@@ -265,6 +265,21 @@ int ep_decode_batch(const ep_decode_job *jobs, int32_t n_jobs, void *stream);
 int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const void *d_tile_index,
                             const float *d_row_scales, int32_t out_dtype, void *d_out, void *stream);
 
+/* Decode fused into a matrix product, first slice (the paper leaves this as future work, Sec. "Limitations and
+ * future work": its decoder materialises the dense tensor and the product reads it back; the right panel of the
+ * reconstruction-cost experiment shows what that costs at small token counts).  Computes
+ *     y[t, r] = sum_k x[t, k] * W^[r, k],   W^ = the stream decoded to BF16 (Eq. 18, Eq. 5, Eq. 19 with tau = BF16),
+ * with BF16 products accumulated in fp32 by the tensor cores; W^ is never written to global memory.
+ *   d_x   device, T x C bfloat16, row-major, 16-byte aligned (T tokens, 1 <= T <= 32)
+ *   d_y   device, T x R float, row-major, 16-byte aligned; every element is written
+ *   d_tables  device, the prepared lookup tables of the stream (ep_prepare_tables); required
+ * The stream must be laid out for it: one tile per row (V = C / 8), C a multiple of 256, R a multiple of 32, b = 11
+ * with tables that fit shared memory (ep_decode_scratch_bytes(info) == 0).  Anything else returns
+ * EP_ERR_UNSUPPORTED; decode with ep_decode_tensor and multiply separately then.  Asynchronous on `stream`, allocates
+ * nothing.  A wait inside the kernel that does not end raises the integrity word below instead of hanging. */
+int ep_decode_gemm(const ep_info *info, const void *d_stream, const void *d_tile_index, const float *d_row_scales,
+                   const void *d_tables, const void *d_x, uint32_t T, float *d_y, void *stream);
+
 /* Device-side integrity word (no counterpart in the paper; it uses the fact that the encoder of Eq. 17 starts
  * every state at 2^15, so a correct decode of Eq. 18 must end there).  The kernel ORs in a flag when a tile does
  * not end with every state at 2^15 and its word pointer at the next tile's offset (a damaged stream).  There is ONE
@@ -281,7 +296,7 @@ int ep_last_device_status(void *stream);
 const char *ep_strerror(int status);                  /* text of an ep_status value (library convention, not the paper's) */
 uint32_t ep_default_tile_vectors(double target_bpp);  /* V from the paper's tile-size defaults */
 
-/* Tile size for a decoder with `decode_slots` concurrent tile slots (ep_decode_tiles_per_sm() = 48 per SM for this library: 7104 on
+/* Tile size for a decoder with `decode_slots` concurrent tile slots (ep_decode_tiles_per_sm() = 32 per SM for this library: 4736 on
  * a 148-SM B200): the largest V not above the paper's default for the target rate for which the tensor's
  * R*C/8 blocks split into a whole number of rounds of decode_slots tiles (the last round nearly full),
  * rounded up to a multiple of 32 vectors when that stays within the default.
@@ -292,7 +307,7 @@ uint32_t ep_suggest_tile_vectors(uint32_t R, uint32_t C, double target_bpp, uint
 
 /* The same question for tensors that are decoded together by one ep_decode_batch launch (the blocks of a
  * transformer layer): one tile size for all of them, a multiple of 32 not above the paper's default, chosen
- * so that the rounds of all tensors (48 tiles per CTA and round) split over `decode_ctas` CTAs (the SM count:
+ * so that the rounds of all tensors (32 tiles per CTA and round) split over `decode_ctas` CTAs (the SM count:
  * 148 on a B200) with the shortest last round.  R[i] x C[i] are the n tensor shapes. */
 uint32_t ep_suggest_tile_vectors_batch(const uint32_t *R, const uint32_t *C, uint32_t n, double target_bpp,
                                        uint32_t decode_ctas);

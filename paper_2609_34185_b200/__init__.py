@@ -7,5 +7,5 @@ streams.
 from .binding import (  # noqa: F401
     BF16, FP16, FP8_E4M3, INT8, FP32, FP8_E5M2, UINT8, FIELDS_I32, DTYPE_BYTES, EncodeOpts, EncodeReport, Info, DecodeJob, Blob,
     EntroPackError, load, encode, encode_device, pack_fields, blob_info, validate, decode_scratch_bytes, decode_tables_bytes, prepare_tables, decode_tiles_per_sm, decode_tensor,
-    decode_tiles, decode_tile_range, decode_tensor_static, decode_batch, last_device_status, default_tile_vectors, suggest_tile_vectors, suggest_tile_vectors_batch, strerror, DeviceBlob, upload, decode, decode_many,
+    decode_tiles, decode_tile_range, decode_tensor_static, decode_gemm, decode_matmul, decode_batch, last_device_status, default_tile_vectors, suggest_tile_vectors, suggest_tile_vectors_batch, strerror, DeviceBlob, upload, decode, decode_many,
 )

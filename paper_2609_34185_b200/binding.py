@@ -106,6 +106,8 @@ def load():
                                   C.c_void_p, C.c_size_t, C.c_uint32, C.c_uint32, C.c_void_p]
     L.ep_decode_tensor_static.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                           C.c_void_p]
+    L.ep_decode_gemm.argtypes = [C.POINTER(Info), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32,
+                                 C.c_void_p, C.c_void_p]
     L.ep_decode_batch.argtypes = [C.POINTER(DecodeJob), C.c_int32, C.c_void_p]
     L.ep_last_device_status.argtypes = [C.c_void_p]
     L.ep_strerror.restype = C.c_char_p
@@ -280,6 +282,13 @@ def decode_tensor_static(info: Info, d_stream: int, d_tile_index: int, d_row_sca
                                           stream or None), "ep_decode_tensor_static")
 
 
+def decode_gemm(info: Info, d_stream: int, d_tile_index: int, d_row_scales: int, d_tables: int, d_x: int, T: int, d_y: int,
+                stream: int = 0) -> None:
+    """ep_decode_gemm with raw device addresses: y[T, R] (fp32) = x[T, C] (bf16) times the decoded weights, transposed."""
+    _check(load().ep_decode_gemm(C.byref(info), d_stream, d_tile_index, d_row_scales, d_tables, d_x, T, d_y, stream or None),
+           "ep_decode_gemm")
+
+
 def decode_batch(jobs: list[DecodeJob], stream: int = 0) -> None:
     arr = (DecodeJob * len(jobs))(*jobs)
     _check(load().ep_decode_batch(arr, len(jobs), stream or None), "ep_decode_batch")
@@ -388,6 +397,27 @@ def decode_tile_range(dblob: DeviceBlob, tiles: range, out_dtype: int = BF16, ou
                      out.data_ptr() - first * 8 * esize, tiles.start, len(tiles),
                      dblob.scratch.data_ptr() if dblob.scratch is not None else 0,
                      dblob.scratch.numel() if dblob.scratch is not None else 0, _stream_handle(stream))
+    return out
+
+
+def decode_matmul(dblob: DeviceBlob, x, out=None, stream=None):
+    """x [T, C] bfloat16 times the blob's decoded BF16 weights [R, C], transposed: [T, R] float32, the weights going
+    from the stream into the tensor cores without passing through global memory (ep_decode_gemm; at most 32 tokens per
+    launch, more are taken 32 at a time; the stream needs one tile per row, see the header)."""
+    torch = _torch()
+    I = dblob.info
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.shape[1] == I.C and x.is_contiguous()
+    if dblob.tables is None:
+        raise EntroPackError(-7, "decode_matmul needs prepared tables (upload(..., prepare=True))")
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty((T, I.R), dtype=torch.float32, device=x.device)
+    assert out.dtype == torch.float32 and out.shape == (T, I.R) and out.is_contiguous()
+    h = _stream_handle(stream)
+    for t0 in range(0, T, 32):
+        n = min(32, T - t0)
+        decode_gemm(I, dblob.d_stream, dblob.d_tile_index, dblob.d_row_scales, dblob.tables.data_ptr(),
+                    x[t0:t0 + n].data_ptr(), n, out[t0:t0 + n].data_ptr(), h)
     return out
 
 

@@ -1124,6 +1124,197 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
 }
 
 // ======================================================================================================
+// Decode fused into a matrix product (the step the paper leaves as future work, Sec. "Limitations and future
+// work": its decoder still materialises the dense tensor before the product).  First slice: y = x W^T for up
+// to 32 tokens - the regime in which reading the weights dominates a linear layer -, W decoded tile by tile
+// straight into the shared-memory operand of a tcgen05 matrix instruction and never written to global memory.
+//
+// The stream must have one tile per row of W (V = C / 8) and C a multiple of 256.  A CTA takes 32 consecutive rows,
+// one per warp; the 32 warps decode their rows group by group (a group = 32 blocks = 256 columns), so after every
+// group the CTA holds a 32 x 256 slab of W: the B operand (N = 32, K-major, 128-byte swizzle: a lane's 16-byte block
+// is one piece of a swizzled row, so the stores are conflict-free).  The matching 256 columns of x (A operand,
+// M = 128 rows of which the first 16 or 32 are tokens; the others read whatever shared memory follows and produce
+// accumulator rows nobody stores) come in by cp.async, four 64-column tiles.  One thread then issues the sixteen
+// K = 16 instructions of the slab; the fp32 accumulator (128 lanes x 32 columns) stays in tensor memory over the
+// whole row and is read out once per 32 rows.
+//
+// Shared memory: lookup tables, payload rings and context blocks as in the decode kernel, then A (16 KB), B (16 KB)
+// and two mbarriers in the 33 KB the 2^12-slot streams use there.  What bounds the token count: the A tiles of a
+// group must be in flight while the group is decoded (about 1 us), x is re-read by every CTA from L2, and 16 KB is
+// all the landing space there is; 32 tokens need 16 KB per group.
+// Every wait on an mbarrier gives up after kSpinLimit polls, raises the abort word and lets the kernel run to its
+// end (wrong output, status flag set) instead of hanging.
+struct GemmParams {
+    JobParams J;
+    const uint16_t *x;            // [T, C] bf16, row-major
+    float *y;                     // [T, R] fp32, row-major
+    uint32_t T, Tpad;             // tokens; rows of x that are staged (16 or 32)
+    uint32_t R, C;
+    uint32_t row_blocks;          // R / 32
+    uint32_t groups;              // C / 256
+};
+
+constexpr uint32_t kGemmA = kHotBase;                    // A operand: four 64-column tiles of Tpad rows
+constexpr uint32_t kGemmB = kHotBase + 16384;            // B operand: four 64-column tiles of 32 rows
+constexpr uint32_t kGemmBar = kHotBase + 32768;          // mbarriers, tensor-memory address, abort word
+constexpr uint32_t kGemmSmem = kHotBase + 33792;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kGemmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, K-major both, N = 32, M = 128
+static_assert(kHotBase % 1024 == 0, "swizzled operand tiles start on 1024-byte boundaries");
+static_assert(kGemmSmem <= 232448, "more shared memory than an sm_100 CTA can have");
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// waits for the phase of the given parity to complete; false (and the abort word set) if it does not within the limit
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_addr) {
+    if (lds32(abort_addr)) return false;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if ((i & 4095u) == 4095u && lds32(abort_addr)) return false;
+    }
+    sts32(abort_addr, 1u);
+    return false;
+}
+// the mbarrier gets one arrival when the cp.async copies this thread has issued so far have landed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// K-major operand tile with 128-byte swizzle: rows of 128 bytes, groups of eight rows 1024 bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    return uint64_t((smem_addr >> 4) & 0x3FFFu) | (uint64_t(1) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) |
+           (uint64_t(2) << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __grid_constant__ GemmParams P) {
+    extern __shared__ __align__(16) uint8_t smem[];      // (the operand tiles need 1024: checked at run time, see abort word)
+    const JobParams &J = P.J;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
+    const uint32_t ring = lut_addr + kRingBase + warp * (kChains * kRingStride);
+    const uint32_t a_base = lut_addr + kGemmA, b_base = lut_addr + kGemmB;
+    const uint32_t bar_a = lut_addr + kGemmBar, bar_mma = bar_a + 8u, slot = bar_a + 16u, abort_addr = bar_a + 20u;
+    if (tid == 0) {
+        mbar_init(bar_a, kThreads);          // every thread arrives once per group, when its piece of x has landed
+        mbar_init(bar_mma, 1u);              // the commit after a group's matrix instructions
+        sts32(abort_addr, (lut_addr & 1023u) ? 1u : 0u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {                         // 32 columns of tensor memory: the 128 x 32 fp32 accumulator
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(32u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    copy_tables_smem(J.lut_image, lut_addr, false);
+    const CosetFreq cf = load_coset(J);
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = lds32(slot);
+
+    const uint32_t lt = (1u << lane) - 1u, mask = 2047u, b = 11u;
+    const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
+    // where this lane's block of a group goes in B: 64-column tile lane / 8, row = warp, piece lane % 8 of the row
+    const uint32_t b_dst = b_base + (lane >> 3) * 4096u + warp * 128u + (((lane & 7u) ^ (warp & 7u)) << 4);
+    // this thread's 16-byte piece of a group's x columns: tile, row and piece
+    const uint32_t row_shift = P.Tpad == 32u ? 5u : 4u;
+    const bool has_piece = tid < P.Tpad * 32u;
+    const uint32_t a_tile = tid >> (row_shift + 3u), a_row = (tid >> 3) & (P.Tpad - 1u), a_piece = tid & 7u;
+    const uint32_t a_tile_bytes = P.Tpad * 128u;
+    const uint32_t a_dst = a_base + a_tile * a_tile_bytes + a_row * 128u + ((a_piece ^ (a_row & 7u)) << 4);
+    const uint64_t a_src = reinterpret_cast<uint64_t>(P.x) + 2ull * (uint64_t(min(a_row, P.T - 1u)) * P.C + a_tile * 64u + a_piece * 8u);
+    const uint32_t a_bytes = (has_piece && a_row < P.T) ? 16u : 0u;    // rows past the last token are filled with zeros
+    uint32_t n_mma = 0;                      // groups handed to the tensor core so far (the same in every thread)
+    bool bad = false;
+
+    for (uint32_t rb = blockIdx.x; rb < P.row_blocks; rb += gridDim.x) {
+        const uint32_t tile = rb * 32u + warp;                      // = the row of W
+        const TileSetup Tl = tile_setup(J, tile, true, lane);
+        uint32_t x = Tl.x, pos = Tl.lead, threshold = kChunk;
+        for (uint32_t c = 0; c < kRingSlots; ++c) ring_issue(ring, Tl.a0, Tl.room, c, lane);
+        cp_async_wait<1>();
+        __syncwarp();
+        const float sigma = __ldg(J.scales + min(tile, J.row_max));
+        for (uint32_t g = 0; g < P.groups; ++g) {
+            // the tensor core is done with the previous group: A and B may be overwritten
+            if (n_mma) mbar_wait(bar_mma, (n_mma - 1u) & 1u, abort_addr);
+            if (has_piece) cp_async16(a_dst, a_src + 512ull * g, a_bytes);
+            cp_async_arrive(bar_a);
+            if (pos >= threshold) ring_service(ring, Tl.a0, Tl.room, pos, threshold, lane);
+            const uint32_t wa0 = ring + pos % kRingBytes;
+            uint32_t wa = wa0;
+            uint4 blk;
+            decode_group_plain<EP_BF16>(x, wa, lut_addr, cf, mask, b, lt, true, k0_bits, sigma, J.zlo, &blk);
+            pos += wa - wa0;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_dst), "r"(blk.x), "r"(blk.y), "r"(blk.z), "r"(blk.w) : "memory");
+            fence_async_smem();              // the stores above are read through the async proxy
+            __syncthreads();
+            if (tid == 0) {
+                mbar_wait(bar_a, n_mma & 1u, abort_addr);
+                fence_async_smem();
+                tc_fence_after();
+#pragma unroll
+                for (uint32_t c = 0; c < 4; ++c)
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k)                 // 16 columns = 32 bytes further along the swizzled rows
+                        umma_bf16(tmem, umma_desc(a_base + c * a_tile_bytes + 32u * k), umma_desc(b_base + c * 4096u + 32u * k),
+                                  kGemmIdesc, (g | c | k) ? 1u : 0u);
+                umma_commit(bar_mma);
+            }
+            ++n_mma;
+        }
+        // the accumulator of these 32 rows: lanes = tokens, columns = rows of W
+        mbar_wait(bar_mma, (n_mma - 1u) & 1u, abort_addr);
+        tc_fence_after();
+        if (warp < 4u) {
+            uint32_t v[32];
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, "
+                         "%23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                           "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                           "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                         : "r"(tmem + ((warp * 32u) << 16)));
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const uint32_t t = warp * 32u + lane;
+            if (t < P.T) {
+                uint4 *dst = reinterpret_cast<uint4 *>(P.y + size_t(t) * P.R + rb * 32u);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) dst[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+        }
+        tc_fence_before();
+        cp_async_wait<0>();                  // nothing may still be landing in the ring when the next row starts
+        __syncthreads();                     // the accumulator has been read before the next rows overwrite it
+        tc_fence_after();
+        bad |= (x != ep::kStateLow) || (Tl.off + ((pos - Tl.lead) >> 1) != Tl.end);
+    }
+    const bool aborted = lds32(abort_addr) != 0;
+    if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
+    if (aborted && tid == 0) atomicOr(&g_ep_status, 2u);
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32u) : "memory");
+}
+
+// ======================================================================================================
 // Large-table path: b >= 12, a coordinate range above 1024, or a single-symbol table at b = 11.  The
 // seventeen tables (2^b slots of 4 bytes: symbol index << 16 | u - F) are built into caller-provided
 // scratch by one launch and read through L1/L2 by the decode launch that follows on the same stream; a
@@ -1790,6 +1981,61 @@ extern "C" int ep_decode_tensor(const ep_info *info, const void *d_stream, const
                                 size_t scratch_bytes, void *stream) {
     const ep_decode_job jb = one_job(info, d_stream, d_tile_index, d_row_scales, out_dtype, d_out, d_scratch, scratch_bytes);
     return ep_decode_batch(&jb, 1, stream);
+}
+
+extern "C" int ep_decode_gemm(const ep_info *info, const void *d_stream, const void *d_tile_index, const float *d_row_scales,
+                              const void *d_tables, const void *d_x, uint32_t T, float *d_y, void *stream) {
+    if (!info || !d_stream || !d_tile_index || !d_row_scales || !d_tables || !d_x || !d_y || T == 0) return EP_ERR_BAD_ARG;
+    const ep_info &I = *info;
+    if (I.C == 0 || I.C % 8 || I.R == 0 || I.V == 0 || I.b < 9 || I.b > 15 || I.J != ep::kStates) return EP_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_stream) & 3) || (reinterpret_cast<uintptr_t>(d_tile_index) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_x) & 15) || (reinterpret_cast<uintptr_t>(d_y) & 15))
+        return EP_ERR_BAD_ARG;
+    if (reinterpret_cast<uintptr_t>(d_tables) & 255) return EP_ERR_SCRATCH;
+    if (I.table_K[0] == 0 || I.table_min[0] < 0 || int64_t(I.table_min[0]) + I.table_K[0] > 2) return EP_ERR_BAD_STREAM;
+    // one tile per row, whole groups per row, 32 rows per CTA, tables in shared memory, 32 warps of one tile each
+    if (kChains != 1 || kWarps != 32 || I.b != 11 || !fits_smem_tables(I) || I.V != I.C / 8 || I.C % 256 || I.R % 32 || T > 32 ||
+        I.total_words >= (1ull << 30) || uint64_t(I.R) * I.C >= (1ull << 32))
+        return EP_ERR_UNSUPPORTED;
+    const int sms = num_sms();
+    if (sms <= 0) return EP_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GemmParams P;
+    std::memset(&P, 0, sizeof(P));
+    JobParams &J = P.J;
+    J.stream = static_cast<const uint8_t *>(d_stream);
+    J.tile_index = static_cast<const uint32_t *>(d_tile_index);
+    J.scales = d_row_scales;
+    J.lut_image = static_cast<const uint32_t *>(d_tables);
+    J.off_payload = I.off_payload;
+    J.total_words = uint32_t(I.total_words);
+    J.n_vec = uint32_t(uint64_t(I.R) * (I.C / 8));
+    J.per_row = I.C / 8;
+    J.V = I.V;
+    J.n_tiles = I.n_tiles;
+    J.tile_cnt = I.n_tiles;
+    J.row_max = I.R - 1u;
+    fill_table_params(J, I);
+    P.x = static_cast<const uint16_t *>(d_x);
+    P.y = d_y;
+    P.T = T;
+    P.Tpad = T <= 16 ? 16u : 32u;
+    P.R = I.R;
+    P.C = I.C;
+    P.row_blocks = I.R / 32u;
+    P.groups = I.C / 256u;
+    if (I.n_tiles != I.R) return EP_ERR_BAD_ARG;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        if (cudaFuncSetAttribute(ep_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)) != cudaSuccess)
+            return EP_ERR_CUDA;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    const uint32_t grid = P.row_blocks < uint32_t(sms) ? P.row_blocks : uint32_t(sms);
+    ep_decode_gemm_kernel<<<grid, kThreads, kGemmSmem, st>>>(P);
+    return cudaGetLastError() == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
 extern "C" int ep_last_device_status(void *stream) {
