@@ -393,6 +393,58 @@ def decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms):
 
 
 
+def timed_flushed(torch, stream, flush, fn, reps=24, warm=3):
+    """(min, mid-mean) in ms of `reps` runs of fn, each after an L2 flush, CUDA events on `stream`."""
+    for _ in range(warm):
+        fn()
+    ts = []
+    for _ in range(reps):
+        flush.fill_(0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    # event times of one short launch come in steps of about 2 us on this GPU: the mean of the central half of
+    # the sorted times resolves what the median cannot
+    ts.sort()
+    mid = ts[len(ts) // 4: len(ts) - len(ts) // 4]
+    return min(ts), sum(mid) / len(mid)
+
+
+def fused_gemm_record(ep, torch, dev, stream, timed, slots):
+    """The decode fused into the matrix product (ep_decode_gemm) on the 10240 x 3840 layer of the reconstruction-cost
+    experiment: up to 32 tokens, against decoding (with the decode path's own tile size) and multiplying with
+    torch.matmul.  `timed(fn)` returns (min, mid-mean) of flushed repetitions in ms."""
+    from paper_2609_34185_b200 import synth
+    Wl = torch.from_numpy(synth.gaussian_rows(10240, 3840, 77)).to(dev)
+    bl_row = ep.encode_device(Wl, 4.0, tile_vectors=3840 // 8)            # one tile per row: the layout the fused kernel reads
+    bl_dec = ep.encode_device(Wl, 4.0, tile_vectors=ep.suggest_tile_vectors(10240, 3840, 4.0, slots))
+    d_row, d_dec = ep.upload(bl_row, device=dev), ep.upload(bl_dec, device=dev)
+    wbuf = torch.empty((10240, 3840), dtype=torch.bfloat16, device=dev)
+    rows = []
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(78)
+    for tokens in (8, 16, 32):
+        x = torch.randn(tokens, 3840, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        y32 = torch.empty((tokens, 10240), dtype=torch.float32, device=dev)
+        y16 = torch.empty((tokens, 10240), dtype=torch.bfloat16, device=dev)
+
+        def two_kernels():
+            ep.decode(d_dec, ep.BF16, out=wbuf, stream=stream)
+            torch.matmul(x, wbuf.t(), out=y16)
+
+        _, t_two = timed(two_kernels)
+        _, t_fused = timed(lambda: ep.decode_matmul(d_row, x, out=y32, stream=stream))
+        rows.append({"tokens": tokens, "decode_then_matmul_ms": t_two, "fused_ms": t_fused})
+        del x, y32, y16
+    return {"rows": rows, "stored_bpp_fused_layout": bl_row.stored_bpp, "stored_bpp_decode_layout": bl_dec.stored_bpp,
+            "tile_vectors_decode_layout": bl_dec.info.V,
+            "what": "y = x W^T, W a 10240 x 3840 layer at 4 bpp: ep_decode_gemm (weights never written to memory) "
+                    "against ep_decode_batch + torch.matmul"}
+
+
 def peak_info():
     """(HBM GB/s the roofline fractions refer to, where the number comes from)"""
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -408,22 +460,7 @@ def extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak, skip):
     from paper_2609_34185_b200 import synth
 
     def timed(fn, reps=24, warm=3):
-        for _ in range(warm):
-            fn()
-        ts = []
-        for _ in range(reps):
-            flush.fill_(0)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            fn()
-            b.record(stream)
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        # event times of one short launch come in steps of about 2 us on this GPU: the mean of the central half of
-        # the sorted times resolves what the median cannot
-        ts.sort()
-        mid = ts[len(ts) // 4: len(ts) - len(ts) // 4]
-        return min(ts), sum(mid) / len(mid)
+        return timed_flushed(torch, stream, flush, fn, reps, warm)
 
     def record(params, nbytes_in, esize, ms, **more):
         alg = nbytes_in + params * esize
@@ -476,6 +513,7 @@ def extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak, skip):
     out["encode_device_8192x8192_4.0bpp"] = {"ms": enc_ms, "stored_bpp": bl.stored_bpp,
                                              "what": "ep_encode_device call to finished host blob, second call"}
     del W4, buf
+    out["decode_gemm_10240x3840_4.0bpp"] = fused_gemm_record(ep, torch, dev, stream, timed, slots)
     # ---- config 3: the block bundle in its FP8-E4M3 and INT8 containers, 2.5 bpp, one batched launch ----
     if skip != "c3":
         V = ep.suggest_tile_vectors_batch(synth.BLOCK_SHAPES, 2.5, n_sms)
@@ -750,6 +788,8 @@ def main():
     gemm_curve = None
     if args.gemm_curve and rank == 0:
         gemm_curve = decode_then_gemm_curve(ep, torch, dev, stream, flush, n_sms)
+        gemm_curve["fused"] = fused_gemm_record(ep, torch, dev, stream,
+                                                lambda fn: timed_flushed(torch, stream, flush, fn), slots)
 
 
     records = None

@@ -273,10 +273,11 @@ int ep_decode_tensor_static(const ep_info *info, const void *d_stream, const voi
  *   d_x   device, T x C bfloat16, row-major, 16-byte aligned (T tokens, 1 <= T <= 32)
  *   d_y   device, T x R float, row-major, 16-byte aligned; every element is written
  *   d_tables  device, the prepared lookup tables of the stream (ep_prepare_tables); required
- * The stream must be laid out for it: one tile per row (V = C / 8), C a multiple of 256, R a multiple of 32, b = 11
- * with tables that fit shared memory (ep_decode_scratch_bytes(info) == 0).  Anything else returns
+ * The stream must be laid out for it: one tile per row (V = C / 8; ep_encode with tile_vectors = C / 8), C a multiple
+ * of 256, b = 11 with tables that fit shared memory (ep_decode_scratch_bytes(info) == 0).  Anything else returns
  * EP_ERR_UNSUPPORTED; decode with ep_decode_tensor and multiply separately then.  Asynchronous on `stream`, allocates
- * nothing.  A wait inside the kernel that does not end raises the integrity word below instead of hanging. */
+ * nothing (it asks the driver for a tensor-map descriptor of x, a host-side call).  A wait inside the kernel that
+ * does not end raises the integrity word below instead of hanging. */
 int ep_decode_gemm(const ep_info *info, const void *d_stream, const void *d_tile_index, const float *d_row_scales,
                    const void *d_tables, const void *d_x, uint32_t T, float *d_y, void *stream);
 

@@ -20,6 +20,7 @@
 // first 512 bytes of the ring are mirrored behind its end so that the nine steps of a group never have
 // to wrap an address.  (With b <= 11 a lane takes at most seven words in nine steps: a step shortens the
 // state by at most eleven bits, a word adds sixteen.)
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -51,8 +52,7 @@ constexpr uint32_t kCosetStride = 8 * kLutStride;            // the eight tables
 constexpr uint32_t kLutBytes = 16 * kLutStride;              // 131072
 // Payload ring of a chain: three chunks of 512 bytes (one cp.async round of a warp, 16 bytes per lane) plus a mirror
 // of its first 512 bytes.  (Measured and dropped: 64 rings of four 256-byte chunks for two tiles per warp at 32 warps.)
-constexpr uint32_t kChunk = 512, kRingSlots = 3, kMirrorSlots = 1;
-constexpr uint32_t kChunkLanes = kChunk / 16;                // lanes that take part in a chunk's copy
+constexpr uint32_t kChunk = 512, kRingSlots = 3;
 constexpr uint32_t kRingBytes = kRingSlots * kChunk;         // 1536
 constexpr uint32_t kRingMirror = 512;                        // >= 7 words * 32 lanes * 2 bytes + one lane span (62)
 constexpr uint32_t kRingStride = kRingBytes + kRingMirror;   // 2048 per chain
@@ -436,37 +436,40 @@ __device__ __forceinline__ void decode_group_plain(uint32_t &x, uint32_t &wa, ui
 }
 
 // ---- payload ring ------------------------------------------------------------------------------------
-// chunk c of a tile = global bytes [a0 + 512c, a0 + 512c + 512), a0 = tile's first word rounded down to
-// 16 bytes; it lives in ring slot c mod 3, and a chunk in slot 0 is written a second time behind the ring's
-// end.  `room` = bytes from a0 to the end of the payload: nothing beyond it is read (cp.async zero-fills
-// the rest).
+// chunk c of a tile = global bytes [a0 + CHUNK c, a0 + CHUNK (c + 1)), a0 = tile's first word rounded down to
+// 16 bytes; it lives in ring slot c mod SLOTS, and a chunk in one of the slots that make up the ring's first 512
+// bytes is written a second time behind the ring's end.  `room` = bytes from a0 to the end of the payload: nothing
+// beyond it is read (cp.async zero-fills the rest).  The decode kernel's rings are 3 x 512 bytes; the kernel that
+// feeds the tensor cores needs the shared memory for its operands and takes 4 x 256.
+template <uint32_t CHUNK = kChunk, uint32_t SLOTS = kRingSlots>
 __device__ __forceinline__ void ring_issue(uint32_t ring, uint64_t a0, uint32_t room, uint32_t c, uint32_t lane) {
-    if (lane < kChunkLanes) {
-        uint32_t o = kChunk * c + 16u * lane;
+    if (lane < CHUNK / 16u) {
+        uint32_t o = CHUNK * c + 16u * lane;
         uint32_t n = 16;
         if (o + 16u > room) {
             n = o < room ? room - o : 0u;
             if (n == 0) o = 0;                   // nothing is read, but keep the address a valid one
         }
-        const uint32_t slot = c % kRingSlots;
-        const uint32_t dst = ring + kChunk * slot + 16u * lane;
+        const uint32_t slot = c % SLOTS;
+        const uint32_t dst = ring + CHUNK * slot + 16u * lane;
         cp_async16(dst, a0 + o, n);
-        if (slot < kMirrorSlots) cp_async16(dst + kRingBytes, a0 + o, n);
+        if (slot < kRingMirror / CHUNK) cp_async16(dst + CHUNK * SLOTS, a0 + o, n);
     }
     cp_async_commit();
 }
 
-// The cursor entered a new chunk: request chunks up to kRingSlots - 1 ahead of it and wait for all but the
+// The cursor entered a new chunk: request chunks up to SLOTS - 1 ahead of it and wait for all but the
 // newest.  `threshold` = start of the chunk after the cursor's at the previous service; chunks up to
-// threshold / kChunk + kRingSlots - 2 have been requested.  A group touches at most 448 + 62 bytes from its start,
+// threshold / CHUNK + SLOTS - 2 have been requested.  A group touches at most 448 + 62 bytes from its start,
 // which the chunks complete after this call cover (1024 bytes from the cursor's chunk on, or 768).
+template <uint32_t CHUNK = kChunk, uint32_t SLOTS = kRingSlots>
 __device__ __forceinline__ void ring_service(uint32_t ring, uint64_t a0, uint32_t room, uint32_t pos, uint32_t &threshold,
                                              uint32_t lane) {
-    const uint32_t cur = pos / kChunk;
-    for (uint32_t c = threshold / kChunk + kRingSlots - 1u; c < cur + kRingSlots; ++c) ring_issue(ring, a0, room, c, lane);
+    const uint32_t cur = pos / CHUNK;
+    for (uint32_t c = threshold / CHUNK + SLOTS - 1u; c < cur + SLOTS; ++c) ring_issue<CHUNK, SLOTS>(ring, a0, room, c, lane);
     cp_async_wait<1>();
     __syncwarp();
-    threshold = kChunk * (cur + 1u);
+    threshold = CHUNK * (cur + 1u);
 }
 
 // what a chain needs to know about its tile
@@ -1129,19 +1132,22 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
 // to 32 tokens - the regime in which reading the weights dominates a linear layer -, W decoded tile by tile
 // straight into the shared-memory operand of a tcgen05 matrix instruction and never written to global memory.
 //
-// The stream must have one tile per row of W (V = C / 8) and C a multiple of 256.  A CTA takes 32 consecutive rows,
-// one per warp; the 32 warps decode their rows group by group (a group = 32 blocks = 256 columns), so after every
-// group the CTA holds a 32 x 256 slab of W: the B operand (N = 32, K-major, 128-byte swizzle: a lane's 16-byte block
-// is one piece of a swizzled row, so the stores are conflict-free).  The matching 256 columns of x (A operand,
-// M = 128 rows of which the first 16 or 32 are tokens; the others read whatever shared memory follows and produce
-// accumulator rows nobody stores) come in by cp.async, four 64-column tiles.  One thread then issues the sixteen
-// K = 16 instructions of the slab; the fp32 accumulator (128 lanes x 32 columns) stays in tensor memory over the
-// whole row and is read out once per 32 rows.
+// The stream must have one tile per row of W (V = C / 8) and C a multiple of 256.  The rows are spread evenly over
+// the SMs; a CTA takes its range 31 rows at a time, one row per warp: warps 0 .. 30 decode their rows group by group
+// (a group = 32 blocks = 256 columns), so after every group the CTA holds a 31 x 256 slab of W - the B operand
+// (N = 32 with one idle row, K-major, 128-byte swizzle: a lane's 16-byte block is one piece of a swizzled row, so
+// the stores are conflict-free).  Warp 31 decodes nothing: one of its lanes brings the matching 256 columns of x in
+// (A operand, M = 64 rows of which the first 16 or 32 are tokens; the others read whatever shared memory follows
+// and produce accumulator rows nobody stores) with four tensor copies (cp.async.bulk.tensor, the copy engine
+// swizzles), waits until all rows of the slab are stored and issues the slab's sixteen K = 16 instructions.  (A
+// decoding warp cannot do that on the side: whoever issues falls behind by the time it takes, and with two slabs
+// every warp is at most one group ahead of the slowest - measured 138 us against 102 us for the layer below.)  The
+// fp32 accumulator (64 lanes x 32 columns) stays in tensor memory over the whole row and is read out once per step.
 //
-// Shared memory: lookup tables, payload rings and context blocks as in the decode kernel, then A (16 KB), B (16 KB)
-// and two mbarriers in the 33 KB the 2^12-slot streams use there.  What bounds the token count: the A tiles of a
-// group must be in flight while the group is decoded (about 1 us), x is re-read by every CTA from L2, and 16 KB is
-// all the landing space there is; 32 tokens need 16 KB per group.
+// Shared memory: the lookup tables (128 KB), 32 payload rings of 4 x 256 + 512 bytes (48 KB), then A (16 KB: two
+// stages for up to 16 tokens, one for up to 32), B (two slabs of 16 KB: the warps decode the next group while the
+// tensor core reads the last one) and six mbarriers.  What bounds the token count: a group's columns of x must be in
+// flight while the group is decoded (about 1 us), every CTA re-reads x from L2, and 16 KB is the landing space left.
 // Every wait on an mbarrier gives up after kSpinLimit polls, raises the abort word and lets the kernel run to its
 // end (wrong output, status flag set) instead of hanging.
 struct GemmParams {
@@ -1150,41 +1156,42 @@ struct GemmParams {
     float *y;                     // [T, R] fp32, row-major
     uint32_t T, Tpad;             // tokens; rows of x that are staged (16 or 32)
     uint32_t R, C;
-    uint32_t row_blocks;          // R / 32
+    uint32_t rows_per_cta;        // CTA k takes rows [k, k + 1) * rows_per_cta, 31 at a time
     uint32_t groups;              // C / 256
 };
 
-constexpr uint32_t kGemmA = kHotBase;                    // A operand: four 64-column tiles of Tpad rows
-constexpr uint32_t kGemmB = kHotBase + 16384;            // B operand: four 64-column tiles of 32 rows
-constexpr uint32_t kGemmBar = kHotBase + 32768;          // mbarriers, tensor-memory address, abort word
-constexpr uint32_t kGemmSmem = kHotBase + 33792;
-constexpr uint32_t kSpinLimit = 1u << 22;
-constexpr uint32_t kGemmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);   // f32 += bf16 x bf16, K-major both, N = 32, M = 128
-static_assert(kHotBase % 1024 == 0, "swizzled operand tiles start on 1024-byte boundaries");
+constexpr uint32_t kGemmChunk = 256, kGemmSlots = 4;     // payload ring of this kernel
+constexpr uint32_t kGemmRingStride = kGemmChunk * kGemmSlots + kRingMirror;   // 1536
+constexpr uint32_t kGemmA = kRingBase + 32u * kGemmRingStride;   // A operand: per stage four 64-column tiles of Tpad rows
+constexpr uint32_t kGemmB = kGemmA + 16384;              // B operand: two slabs of four 64-column tiles of 32 rows
+constexpr uint32_t kGemmBar = kGemmB + 32768;            // mbarriers, tensor-memory address, abort word, counter
+constexpr uint32_t kGemmSmem = kGemmBar + 64;
+constexpr uint32_t kSpinLimit = 1u << 18;             // attempts of about a microsecond each at most: a quarter of a second
+constexpr uint32_t kGemmRows = 31;                       // rows of W per step: warps 0 .. 30 decode one each, warp 31 feeds the tensor core
+constexpr uint32_t kGemmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((64u >> 4) << 24);   // f32 += bf16 x bf16, K-major both, N = 32, M = 64
+static_assert(kGemmA % 1024 == 0, "swizzled operand tiles start on 1024-byte boundaries");
 static_assert(kGemmSmem <= 232448, "more shared memory than an sm_100 CTA can have");
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+// one attempt: the thread may be suspended by the hardware for up to about a microsecond while the phase is pending
+// (a busy test_wait loop of 32 waiting lanes took half of the kernel's issue slots away from the decoding warps)
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(1000u) : "memory");
     return ok != 0;
 }
 // waits for the phase of the given parity to complete; false (and the abort word set) if it does not within the limit
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_addr) {
     if (lds32(abort_addr)) return false;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_test(bar, parity)) return true;
-        if ((i & 4095u) == 4095u && lds32(abort_addr)) return false;
+        if (mbar_try(bar, parity)) return true;
+        if ((i & 255u) == 255u && lds32(abort_addr)) return false;
     }
     sts32(abort_addr, 1u);
     return false;
-}
-// the mbarrier gets one arrival when the cp.async copies this thread has issued so far have landed
-__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -1203,23 +1210,38 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __grid_constant__ GemmParams P) {
+template <uint32_t TPAD>
+__global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __grid_constant__ GemmParams P,
+                                                                     const __grid_constant__ CUtensorMap x_map) {
     extern __shared__ __align__(16) uint8_t smem[];      // (the operand tiles need 1024: checked at run time, see abort word)
     const JobParams &J = P.J;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
-    const uint32_t ring = lut_addr + kRingBase + warp * (kChains * kRingStride);
+    const uint32_t ring = lut_addr + kRingBase + warp * kGemmRingStride;
     const uint32_t a_base = lut_addr + kGemmA, b_base = lut_addr + kGemmB;
-    const uint32_t bar_a = lut_addr + kGemmBar, bar_mma = bar_a + 8u, slot = bar_a + 16u, abort_addr = bar_a + 20u;
+    // two mbarriers each for: x landed (per stage of A), rows stored (per slab of B), the tensor core's commits (per slab)
+    const uint32_t bar_a = lut_addr + kGemmBar, bar_mma = bar_a + 16u, bar_b = bar_a + 32u, slot = bar_a + 48u,
+                   abort_addr = bar_a + 52u;
+    constexpr uint32_t stages = TPAD == 16u ? 2u : 1u;      // 16 staged rows of x: two groups' worth fit the 16 KB
     if (tid == 0) {
-        mbar_init(bar_a, kThreads);          // every thread arrives once per group, when its piece of x has landed
+        mbar_init(bar_a, 1u);                // the feeding lane's arrival; completes when the tiles of x have landed
+        mbar_init(bar_a + 8u, 1u);
         mbar_init(bar_mma, 1u);              // the commit after a group's matrix instructions
+        mbar_init(bar_mma + 8u, 1u);
+        mbar_init(bar_b, kGemmRows);         // every decoding warp, when its row of the slab is stored
+        mbar_init(bar_b + 8u, kGemmRows);
         sts32(abort_addr, (lut_addr & 1023u) ? 1u : 0u);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {                         // 32 columns of tensor memory: the 128 x 32 fp32 accumulator
+    if (warp == 0) {                         // 32 columns of tensor memory: the 64 x 32 fp32 accumulator
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(32u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // row 31 of both slabs of B belongs to no warp: zero, so that column 31 of the accumulator stays finite
+    if (warp == kGemmRows) {
+        for (uint32_t i = lane; i < 2u * 4u * 8u; i += 32u)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(b_base + (i >> 5) * 16384u + ((i >> 3) & 3u) * 4096u + kGemmRows * 128u + (i & 7u) * 16u), "r"(0u) : "memory");
+        fence_async_smem();
     }
     copy_tables_smem(J.lut_image, lut_addr, false);
     const CosetFreq cf = load_coset(J);
@@ -1229,83 +1251,143 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
     tc_fence_after();
     const uint32_t tmem = lds32(slot);
 
-    const uint32_t lt = (1u << lane) - 1u, mask = 2047u, b = 11u;
-    const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
-    // where this lane's block of a group goes in B: 64-column tile lane / 8, row = warp, piece lane % 8 of the row
-    const uint32_t b_dst = b_base + (lane >> 3) * 4096u + warp * 128u + (((lane & 7u) ^ (warp & 7u)) << 4);
-    // this thread's 16-byte piece of a group's x columns: tile, row and piece
-    const uint32_t row_shift = P.Tpad == 32u ? 5u : 4u;
-    const bool has_piece = tid < P.Tpad * 32u;
-    const uint32_t a_tile = tid >> (row_shift + 3u), a_row = (tid >> 3) & (P.Tpad - 1u), a_piece = tid & 7u;
-    const uint32_t a_tile_bytes = P.Tpad * 128u;
-    const uint32_t a_dst = a_base + a_tile * a_tile_bytes + a_row * 128u + ((a_piece ^ (a_row & 7u)) << 4);
-    const uint64_t a_src = reinterpret_cast<uint64_t>(P.x) + 2ull * (uint64_t(min(a_row, P.T - 1u)) * P.C + a_tile * 64u + a_piece * 8u);
-    const uint32_t a_bytes = (has_piece && a_row < P.T) ? 16u : 0u;    // rows past the last token are filled with zeros
-    uint32_t n_mma = 0;                      // groups handed to the tensor core so far (the same in every thread)
+    const uint32_t row_begin = min(blockIdx.x * P.rows_per_cta, P.R), row_end = min(row_begin + P.rows_per_cta, P.R);
+    const uint32_t steps = (row_end - row_begin + kGemmRows - 1u) / kGemmRows;
+    const uint32_t q_total = steps * P.groups;               // groups this CTA hands to the tensor core
+    // one lane polls, the warp follows
+    auto wait_warp = [&](uint32_t bar, uint32_t parity) {
+        if (lane == 0) mbar_wait(bar, parity, abort_addr);
+        __syncwarp();
+    };
+    constexpr uint32_t a_tile_bytes = TPAD * 128u, a_stage_bytes = 4u * a_tile_bytes;
     bool bad = false;
 
-    for (uint32_t rb = blockIdx.x; rb < P.row_blocks; rb += gridDim.x) {
-        const uint32_t tile = rb * 32u + warp;                      // = the row of W
-        const TileSetup Tl = tile_setup(J, tile, true, lane);
-        uint32_t x = Tl.x, pos = Tl.lead, threshold = kChunk;
-        for (uint32_t c = 0; c < kRingSlots; ++c) ring_issue(ring, Tl.a0, Tl.room, c, lane);
-        cp_async_wait<1>();
-        __syncwarp();
-        const float sigma = __ldg(J.scales + min(tile, J.row_max));
-        for (uint32_t g = 0; g < P.groups; ++g) {
-            // the tensor core is done with the previous group: A and B may be overwritten
-            if (n_mma) mbar_wait(bar_mma, (n_mma - 1u) & 1u, abort_addr);
-            if (has_piece) cp_async16(a_dst, a_src + 512ull * g, a_bytes);
-            cp_async_arrive(bar_a);
-            if (pos >= threshold) ring_service(ring, Tl.a0, Tl.room, pos, threshold, lane);
-            const uint32_t wa0 = ring + pos % kRingBytes;
-            uint32_t wa = wa0;
-            uint4 blk;
-            decode_group_plain<EP_BF16>(x, wa, lut_addr, cf, mask, b, lt, true, k0_bits, sigma, J.zlo, &blk);
-            pos += wa - wa0;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_dst), "r"(blk.x), "r"(blk.y), "r"(blk.z), "r"(blk.w) : "memory");
-            fence_async_smem();              // the stores above are read through the async proxy
-            __syncthreads();
-            if (tid == 0) {
-                mbar_wait(bar_a, n_mma & 1u, abort_addr);
-                fence_async_smem();
+    if (warp == kGemmRows) {
+        // ---- the feeding warp: x into A, matrix instructions, no decoding; one lane does it all ----
+        // group q's 256 columns of x: four tiles of 64 columns x TPAD rows, laid out and swizzled by the copy engine
+        // (rows past the last token lie outside the tensor and arrive as zeros)
+        auto load_a = [&](uint32_t qq) {
+            const uint32_t g = qq % P.groups, st = qq % stages, bar = bar_a + 8u * st;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(a_stage_bytes) : "memory");
+#pragma unroll
+            for (uint32_t t = 0; t < 4; ++t)
+                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                             ::"r"(a_base + st * a_stage_bytes + t * a_tile_bytes), "l"(&x_map), "r"(g * 256u + t * 64u), "r"(0u), "r"(bar)
+                             : "memory");
+        };
+        if (lane == 0) {
+            load_a(0u);
+            if (stages == 2u && q_total > 1u) load_a(1u);
+        }
+        for (uint32_t q = 0; q < q_total; ++q) {
+            const uint32_t st = q % stages, g = q % P.groups;
+            if (lane == 0) {
+                mbar_wait(bar_a + 8u * st, (q / stages) & 1u, abort_addr);
+                mbar_wait(bar_b + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
                 tc_fence_after();
+                // descriptors differ in their address field only: low word + (bytes >> 4)
+                const uint64_t da = umma_desc(a_base + st * a_stage_bytes), db = umma_desc(b_base + 16384u * (q & 1u));
+                const uint32_t da_hi = uint32_t(da >> 32), db_hi = uint32_t(db >> 32), da_lo = uint32_t(da), db_lo = uint32_t(db);
 #pragma unroll
                 for (uint32_t c = 0; c < 4; ++c)
 #pragma unroll
                     for (uint32_t k = 0; k < 4; ++k)                 // 16 columns = 32 bytes further along the swizzled rows
-                        umma_bf16(tmem, umma_desc(a_base + c * a_tile_bytes + 32u * k), umma_desc(b_base + c * 4096u + 32u * k),
-                                  kGemmIdesc, (g | c | k) ? 1u : 0u);
-                umma_commit(bar_mma);
+                        umma_bf16(tmem, pack64(da_lo + ((c * a_tile_bytes + 32u * k) >> 4), da_hi),
+                                  pack64(db_lo + ((c * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc, (g | c | k) ? 1u : 0u);
+                umma_commit(bar_mma + 8u * (q & 1u));
+                if constexpr (stages == 2u) {
+                    // refill the stage the PREVIOUS group used: its instructions were committed a whole group ago and are
+                    // done or nearly so, and the tiles have this group's time to arrive
+                    if (q >= 1u && q + 1u < q_total) {
+                        mbar_wait(bar_mma + 8u * ((q - 1u) & 1u), ((q - 1u) >> 1) & 1u, abort_addr);
+                        load_a(q + 1u);
+                    }
+                } else if (q + 1u < q_total) {   // one stage: it is free when this group's instructions are done
+                    mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
+                    load_a(q + 1u);
+                }
             }
-            ++n_mma;
+            __syncwarp();
+            if (g + 1u == P.groups) {        // a step's last group: the other warps read the accumulator out now
+                tc_fence_before();
+                __syncthreads();
+                tc_fence_after();
+            }
         }
-        // the accumulator of these 32 rows: lanes = tokens, columns = rows of W
-        mbar_wait(bar_mma, (n_mma - 1u) & 1u, abort_addr);
-        tc_fence_after();
-        if (warp < 4u) {
-            uint32_t v[32];
-            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, "
-                         "%23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                           "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                           "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                           "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                         : "r"(tmem + ((warp * 32u) << 16)));
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            const uint32_t t = warp * 32u + lane;
-            if (t < P.T) {
-                uint4 *dst = reinterpret_cast<uint4 *>(P.y + size_t(t) * P.R + rb * 32u);
+    } else {
+        // ---- the decoding warps: one row of W each, group by group into the slabs of B ----
+        const uint32_t lt = (1u << lane) - 1u, mask = 2047u, b = 11u;
+        const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
+        // where this lane's block of a group goes in a slab: 64-column tile lane / 8, row = warp, piece lane % 8 of the row
+        const uint32_t b_dst = b_base + (lane >> 3) * 4096u + warp * 128u + (((lane & 7u) ^ (warp & 7u)) << 4);
+        uint32_t q = 0;
+        for (uint32_t r0 = row_begin; r0 < row_end; r0 += kGemmRows) {
+            const bool active = r0 + warp < row_end;                    // the last rows of the CTA's range may be fewer than 31
+            const uint32_t tile = min(r0 + warp, P.R - 1u);             // = the row of W
+            const TileSetup Tl = tile_setup(J, tile, active, lane);
+            uint32_t x = Tl.x, pos = Tl.lead, threshold = kGemmChunk;
+            if (active) {
+                for (uint32_t c = 0; c < kGemmSlots; ++c) ring_issue<kGemmChunk, kGemmSlots>(ring, Tl.a0, Tl.room, c, lane);
+                cp_async_wait<1>();
+                __syncwarp();
+            }
+            const float sigma = __ldg(J.scales + tile);
+            // the row this warp takes in the next step: its record is asked for now and, a few groups on, the start of
+            // its payload is brought into L2, so that the next step does not begin with two reads from DRAM in a row
+            const bool has_next = r0 + kGemmRows + warp < row_end;
+            const uint32_t *rec_next = J.tile_index + size_t(min(tile + kGemmRows, P.R - 1u)) * 33u;
+            uint32_t off_next = 0;
+            if (has_next) off_next = __ldg(rec_next + 32);
+            if (has_next && lane == 0) prefetch_l2(rec_next);
+            for (uint32_t g = 0; g < P.groups; ++g, ++q) {
+                if (g == 2u && has_next) {
+                    const uint64_t at = 2ull * min(off_next, J.total_words) + 128u * lane;      // 4 KB: the ring's first fill and more
+                    if (at < 2ull * J.total_words) prefetch_l2(J.stream + J.off_payload + at);
+                }
+                uint4 blk = make_uint4(0u, 0u, 0u, 0u);
+                if (active) {
+                    if (pos >= threshold) ring_service<kGemmChunk, kGemmSlots>(ring, Tl.a0, Tl.room, pos, threshold, lane);
+                    const uint32_t wa0 = ring + pos % (kGemmChunk * kGemmSlots);
+                    uint32_t wa = wa0;
+                    decode_group_plain<EP_BF16>(x, wa, lut_addr, cf, mask, b, lt, true, k0_bits, sigma, J.zlo, &blk);
+                    pos += wa - wa0;
+                }
+                // the slab is free: the tensor core is done with the group that used it last, two groups ago
+                if (q >= 2u) wait_warp(bar_mma + 8u * (q & 1u), ((q >> 1) - 1u) & 1u);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_dst + 16384u * (q & 1u)), "r"(blk.x), "r"(blk.y), "r"(blk.z), "r"(blk.w) : "memory");
+                fence_async_smem();          // the stores above are read through the async proxy
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_b + 8u * (q & 1u)) : "memory");
+            }
+            // the accumulator of these rows: with M = 64, token 16 w + l is lane l < 16 of warp w's quarter; columns = rows of W
+            wait_warp(bar_mma + 8u * ((q - 1u) & 1u), ((q - 1u) >> 1) & 1u);
+            tc_fence_after();
+            if (warp < 2u) {
+                uint32_t v[32];
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, "
+                             "%23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                               "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                               "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                               "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                             : "r"(tmem + ((warp * 32u) << 16)));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const uint32_t t = warp * 16u + lane;
+                if (lane < 16u && t < P.T) {
+                    float *dst = P.y + size_t(t) * P.R + r0;
+                    const uint32_t n = min(kGemmRows, row_end - r0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) dst[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    for (uint32_t i = 0; i < kGemmRows; ++i)
+                        if (i < n) dst[i] = __uint_as_float(v[i]);
+                }
             }
+            tc_fence_before();
+            cp_async_wait<0>();              // nothing may still be landing in the ring when the next row starts
+            __syncthreads();                 // the accumulator has been read before the next rows overwrite it
+            tc_fence_after();
+            bad |= active && ((x != ep::kStateLow) || (Tl.off + ((pos - Tl.lead) >> 1) != Tl.end));
         }
-        tc_fence_before();
-        cp_async_wait<0>();                  // nothing may still be landing in the ring when the next row starts
-        __syncthreads();                     // the accumulator has been read before the next rows overwrite it
-        tc_fence_after();
-        bad |= (x != ep::kStateLow) || (Tl.off + ((pos - Tl.lead) >> 1) != Tl.end);
     }
     const bool aborted = lds32(abort_addr) != 0;
     if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(&g_ep_status, 1u);
@@ -1983,6 +2065,12 @@ extern "C" int ep_decode_tensor(const ep_info *info, const void *d_stream, const
     return ep_decode_batch(&jb, 1, stream);
 }
 
+namespace {
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+}
+
 extern "C" int ep_decode_gemm(const ep_info *info, const void *d_stream, const void *d_tile_index, const float *d_row_scales,
                               const void *d_tables, const void *d_x, uint32_t T, float *d_y, void *stream) {
     if (!info || !d_stream || !d_tile_index || !d_row_scales || !d_tables || !d_x || !d_y || T == 0) return EP_ERR_BAD_ARG;
@@ -1994,7 +2082,7 @@ extern "C" int ep_decode_gemm(const ep_info *info, const void *d_stream, const v
     if (reinterpret_cast<uintptr_t>(d_tables) & 255) return EP_ERR_SCRATCH;
     if (I.table_K[0] == 0 || I.table_min[0] < 0 || int64_t(I.table_min[0]) + I.table_K[0] > 2) return EP_ERR_BAD_STREAM;
     // one tile per row, whole groups per row, 32 rows per CTA, tables in shared memory, 32 warps of one tile each
-    if (kChains != 1 || kWarps != 32 || I.b != 11 || !fits_smem_tables(I) || I.V != I.C / 8 || I.C % 256 || I.R % 32 || T > 32 ||
+    if (kChains != 1 || kWarps != 32 || I.b != 11 || !fits_smem_tables(I) || I.V != I.C / 8 || I.C % 256 || T > 32 ||
         I.total_words >= (1ull << 30) || uint64_t(I.R) * I.C >= (1ull << 32))
         return EP_ERR_UNSUPPORTED;
     const int sms = num_sms();
@@ -2022,19 +2110,40 @@ extern "C" int ep_decode_gemm(const ep_info *info, const void *d_stream, const v
     P.Tpad = T <= 16 ? 16u : 32u;
     P.R = I.R;
     P.C = I.C;
-    P.row_blocks = I.R / 32u;
+    // rows spread evenly over the SMs (a CTA takes its range 31 rows at a time; the last, shorter step runs with fewer
+    // warps and ends sooner than a full one)
+    P.rows_per_cta = (I.R + uint32_t(sms) - 1u) / uint32_t(sms);
     P.groups = I.C / 256u;
     if (I.n_tiles != I.R) return EP_ERR_BAD_ARG;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return EP_ERR_CUDA;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        if (cudaFuncSetAttribute(ep_decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)) != cudaSuccess)
+        if (cudaFuncSetAttribute(ep_decode_gemm_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)) != cudaSuccess ||
+            cudaFuncSetAttribute(ep_decode_gemm_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(kGemmSmem)) != cudaSuccess)
             return EP_ERR_CUDA;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    const uint32_t grid = P.row_blocks < uint32_t(sms) ? P.row_blocks : uint32_t(sms);
-    ep_decode_gemm_kernel<<<grid, kThreads, kGemmSmem, st>>>(P);
+    const uint32_t grid = (I.R + P.rows_per_cta - 1u) / P.rows_per_cta;
+    // x as a two-dimensional tensor for the copy engine: boxes of 64 columns (128 bytes, the swizzle span) x Tpad rows
+    static EncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+            qres != cudaDriverEntryPointSuccess)
+            return EP_ERR_CUDA;
+        encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    CUtensorMap x_map;
+    const cuuint64_t dims[2] = {I.C, T}, strides[1] = {cuuint64_t(I.C) * 2u};
+    const cuuint32_t box[2] = {64u, P.Tpad}, estr[2] = {1u, 1u};
+    if (encode(&x_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_x), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return EP_ERR_CUDA;
+    if (P.Tpad == 16u) ep_decode_gemm_kernel<16><<<grid, kThreads, kGemmSmem, st>>>(P, x_map);
+    else ep_decode_gemm_kernel<32><<<grid, kThreads, kGemmSmem, st>>>(P, x_map);
     return cudaGetLastError() == cudaSuccess ? EP_OK : EP_ERR_CUDA;
 }
 
