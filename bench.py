@@ -41,9 +41,9 @@ FALLBACK_HBM_GBS = 6650.0   # earlier measurement on this machine, used only if MEA
 
 # dram bytes (read + write) per launch measured with ncu for the default workload, filled in from
 # profiles/ after a capture; None = not captured for this workload
-NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 39580672 + 76665344,      # dram read + write of one launch
-                     ("c4", 8.0, "fp16"): 68497408 + 80873984,
-                     ("c5", 3.5, "bf16"): 207664896 + 689508608}
+NCU_TRAFFIC_BYTES = {("c4", 4.0, "fp16"): 39581696 + 76114944,      # dram read + write of one launch
+                     ("c4", 8.0, "fp16"): 68460032 + 80646656,
+                     ("c5", 3.5, "bf16"): 207602944 + 686487552}
 
 
 def parse_args():
