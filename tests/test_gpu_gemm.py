@@ -53,6 +53,21 @@ def test_decode_matmul_against_the_oracle(R, C, T, bpp):
     _check(blob, T, R + T)
 
 
+def test_decode_matmul_small_and_ragged_shapes():
+    # hand-packed streams (b = 11, one tile per row): fewer rows than one step of a CTA, a single group per row, row
+    # counts that leave the last step of a CTA ragged, more CTAs' worth of rows than SMs * 31
+    rng = np.random.default_rng(74)
+    for R, C, T in ((1, 256, 1), (5, 256, 32), (33, 512, 16), (157, 768, 3), (148 * 31 + 7, 256, 9)):
+        n = R * C // 8
+        fields = np.zeros((n, 9), np.int32)
+        fields[:, 0] = rng.integers(0, 2, n)
+        fields[:, 1:8] = np.rint(rng.standard_normal((n, 7)) * 6).astype(np.int32)
+        fields[:, 8] = np.rint(rng.standard_normal(n) * 3).astype(np.int32)
+        blob = ep.pack_fields(fields, R, C, 11, C // 8, rng.uniform(0.01, 0.05, R).astype(np.float32))
+        assert blob.info.n_tiles == R
+        _check(blob, T, R + C + T)
+
+
 def test_decode_matmul_more_tokens_than_one_launch_and_repeated_calls():
     W = synth.gaussian_rows(128, 1536, 71)
     blob = ep.encode(W, 4.0, tile_vectors=1536 // 8)
