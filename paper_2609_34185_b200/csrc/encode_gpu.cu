@@ -32,37 +32,61 @@ constexpr int kLocalBins = 512;          // shared-memory window per table, valu
 constexpr int kLocalOrigin = -256;
 constexpr uint32_t kMaxTableSymbols = 40960;   // sum of K over the 17 tables that the tile encoder keeps in shared memory
 
-// ---- Sec. 3.2: row RMS, one thread per row, squares summed in double in index order ---------------
-__global__ void row_rms_kernel(const float *__restrict__ W, uint32_t R, uint32_t C, float *__restrict__ mu) {
-    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= R) return;
-    // the sum is one serial chain (the host's order); the loads are not: eight 16-byte loads are in flight per pass
-    const float4 *x = reinterpret_cast<const float4 *>(W + size_t(r) * C);     // rows start 16-byte aligned: C % 8 == 0
-    const uint32_t n4 = C / 4;
-    double acc = 0.0;
-    uint32_t j = 0;
-    for (; j + 8 <= n4; j += 8) {
-        float4 v[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) v[k] = __ldg(x + j + k);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            acc = __dadd_rn(acc, __dmul_rn(double(v[k].x), double(v[k].x)));
-            acc = __dadd_rn(acc, __dmul_rn(double(v[k].y), double(v[k].y)));
-            acc = __dadd_rn(acc, __dmul_rn(double(v[k].z), double(v[k].z)));
-            acc = __dadd_rn(acc, __dmul_rn(double(v[k].w), double(v[k].w)));
+// ---- rows whose sums run in index order ---------------------------------------------------------------
+// The row RMS (Sec. 3.2) and the refit of Eq. 13 sum over a row in double precision in index order, as the host code
+// does: one serial chain of additions per row, which no reduction tree reproduces bit for bit.  One thread per row
+// reading its own row leaves the GPU waiting for memory (8192 rows = 256 warps with a few KB in flight each: 0.29 ms
+// for the RMS of an 8192 x 8192 tensor).  So a CTA takes kRowsPerCta rows: all its threads stream the rows through
+// shared memory with cp.async, kRowStages chunks ahead, and kRowsPerCta lanes of its first warp run the chains.
+constexpr uint32_t kRowsPerCta = 8, kRowStages = 4, kRowThreads = 256;
+constexpr uint32_t kRmsChunk = 256;                 // floats per row and chunk
+constexpr uint32_t kRmsStride = kRmsChunk + 4;      // padded: the eight lanes read different banks
+
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(uint32_t(__cvta_generic_to_shared(smem_dst))), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit_group() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(kRowThreads) row_rms_kernel(const float *__restrict__ W, uint32_t R, uint32_t C, float *__restrict__ mu) {
+    __shared__ __align__(16) float buf[kRowStages][kRowsPerCta][kRmsStride];
+    const uint32_t tid = threadIdx.x, row0 = blockIdx.x * kRowsPerCta;
+    const uint32_t chunks = (C + kRmsChunk - 1) / kRmsChunk;
+    // chunk c of the CTA's rows: kRowsPerCta x 64 pieces of 16 bytes, two per thread (rows start 16-byte aligned: C % 8 == 0)
+    auto issue = [&](uint32_t c) {
+        if (c < chunks) {
+            for (uint32_t i = tid; i < kRowsPerCta * (kRmsChunk / 4); i += kRowThreads) {
+                const uint32_t r = i / (kRmsChunk / 4), j = i % (kRmsChunk / 4), col = c * kRmsChunk + 4 * j;
+                if (row0 + r < R && col < C) cp_async_16(&buf[c % kRowStages][r][4 * j], W + size_t(row0 + r) * C + col);
+            }
         }
+        cp_async_commit_group();
+    };
+    for (uint32_t c = 0; c + 1 < kRowStages; ++c) issue(c);
+    double acc = 0.0;
+    for (uint32_t c = 0; c < chunks; ++c) {
+        issue(c + kRowStages - 1);
+        cp_async_wait_group<kRowStages - 1>();
+        __syncthreads();
+        if (tid < kRowsPerCta && row0 + tid < R) {
+            const uint32_t n4 = (min(kRmsChunk, C - c * kRmsChunk)) / 4;
+            const float4 *x = reinterpret_cast<const float4 *>(&buf[c % kRowStages][tid][0]);
+            for (uint32_t j = 0; j < n4; ++j) {
+                const float4 v = x[j];
+                acc = __dadd_rn(acc, __dmul_rn(double(v.x), double(v.x)));
+                acc = __dadd_rn(acc, __dmul_rn(double(v.y), double(v.y)));
+                acc = __dadd_rn(acc, __dmul_rn(double(v.z), double(v.z)));
+                acc = __dadd_rn(acc, __dmul_rn(double(v.w), double(v.w)));
+            }
+        }
+        __syncthreads();                     // the stage may be overwritten by the next issue
     }
-    for (; j < n4; ++j) {
-        const float4 v = __ldg(x + j);
-        acc = __dadd_rn(acc, __dmul_rn(double(v.x), double(v.x)));
-        acc = __dadd_rn(acc, __dmul_rn(double(v.y), double(v.y)));
-        acc = __dadd_rn(acc, __dmul_rn(double(v.z), double(v.z)));
-        acc = __dadd_rn(acc, __dmul_rn(double(v.w), double(v.w)));
+    if (tid < kRowsPerCta && row0 + tid < R) {
+        double m = __dsqrt_rn(__ddiv_rn(acc, double(C)));
+        if (!(m > 1e-12)) m = 1e-12;
+        mu[row0 + tid] = __double2float_rn(m);
     }
-    double m = __dsqrt_rn(__ddiv_rn(acc, double(C)));
-    if (!(m > 1e-12)) m = 1e-12;
-    mu[r] = __double2float_rn(m);
 }
 
 // Eq. 3 on one 8-vector: integer point and fp32 residuals of that point
@@ -171,55 +195,98 @@ __global__ void __launch_bounds__(256) quantise_count_kernel(const float *__rest
     }
 }
 
-// Eq. 13, one thread per row, sums in double in index order
-__global__ void refit_kernel(const float *__restrict__ W, uint32_t R, uint32_t C, const int16_t *__restrict__ fields, float s,
-                             const float *__restrict__ mu, float *__restrict__ sigma) {
-    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= R) return;
-    const uint32_t per_row = C / 8;
-    const float4 *x4 = reinterpret_cast<const float4 *>(W + size_t(r) * C);    // rows start 16-byte aligned: C % 8 == 0
-    const int16_t *q = fields + size_t(r) * per_row * 9;
-    double xp = 0.0, pp = 0.0;
-    // two serial chains in the host's order; the loads of four blocks are issued together
-    constexpr int kAhead = 4;
-    for (uint32_t v0 = 0; v0 < per_row; v0 += kAhead) {
-        float xv[kAhead][8];
-        int32_t qv[kAhead][9];
+// Eq. 13: the two sums of a row in double in index order.  One block = 8 weights and its nine fields.
+__device__ __forceinline__ void refit_block(const float *xv, const int16_t *qv, double &xp, double &pp) {
+    const double half = 0.5 * double(qv[0]);
+    int32_t s7 = 0;
 #pragma unroll
-        for (int k = 0; k < kAhead; ++k) {
-            if (v0 + k < per_row) {
-                const float4 a = __ldg(x4 + 2 * (v0 + k)), b = __ldg(x4 + 2 * (v0 + k) + 1);
-                xv[k][0] = a.x; xv[k][1] = a.y; xv[k][2] = a.z; xv[k][3] = a.w;
-                xv[k][4] = b.x; xv[k][5] = b.y; xv[k][6] = b.z; xv[k][7] = b.w;
-#pragma unroll
-                for (int j = 0; j < 9; ++j) qv[k][j] = q[9 * (v0 + k) + j];
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < kAhead; ++k) {
-            if (v0 + k >= per_row) break;
-            const double half = 0.5 * double(qv[k][0]);
-            int32_t s7 = 0;
-#pragma unroll
-            for (int j = 0; j < 7; ++j) {
-                const double p = __dadd_rn(double(qv[k][1 + j]), half);
-                xp = __dadd_rn(xp, __dmul_rn(double(xv[k][j]), p));
-                pp = __dadd_rn(pp, __dmul_rn(p, p));
-                s7 += qv[k][1 + j];
-            }
-            const double p8 = __dadd_rn(double(2 * qv[k][8] + (s7 & 1)), half);   // Eq. 5
-            xp = __dadd_rn(xp, __dmul_rn(double(xv[k][7]), p8));
-            pp = __dadd_rn(pp, __dmul_rn(p8, p8));
-        }
+    for (int j = 0; j < 7; ++j) {
+        const double p = __dadd_rn(double(qv[1 + j]), half);
+        xp = __dadd_rn(xp, __dmul_rn(double(xv[j]), p));
+        pp = __dadd_rn(pp, __dmul_rn(p, p));
+        s7 += qv[1 + j];
     }
+    const double p8 = __dadd_rn(double(2 * qv[8] + (s7 & 1)), half);   // Eq. 5
+    xp = __dadd_rn(xp, __dmul_rn(double(xv[7]), p8));
+    pp = __dadd_rn(pp, __dmul_rn(p8, p8));
+}
+__device__ __forceinline__ float refit_result(double xp, double pp, float s, float mu) {
     double sg;
     if (pp > 0.0) {
         sg = __ddiv_rn(xp, pp);
         if (!(sg > 1e-12)) sg = 1e-12;
     } else {
-        sg = __dmul_rn(double(s), double(mu[r]));
+        sg = __dmul_rn(double(s), double(mu));
     }
-    sigma[r] = __double2float_rn(sg);
+    return __double2float_rn(sg);
+}
+
+// rows streamed through shared memory (see row_rms_kernel); needs 16-byte aligned field rows: C a multiple of 64
+constexpr uint32_t kRefitBlocks = 16;                              // blocks per row and chunk
+constexpr uint32_t kRefitWStride = kRefitBlocks * 8 + 4;           // floats, padded
+constexpr uint32_t kRefitQStride = kRefitBlocks * 9 + 8;           // int16, padded, a multiple of 8
+__global__ void __launch_bounds__(kRowThreads) refit_kernel(const float *__restrict__ W, uint32_t R, uint32_t C,
+                                                            const int16_t *__restrict__ fields, float s,
+                                                            const float *__restrict__ mu, float *__restrict__ sigma) {
+    __shared__ __align__(16) float wbuf[kRowStages][kRowsPerCta][kRefitWStride];
+    __shared__ __align__(16) int16_t qbuf[kRowStages][kRowsPerCta][kRefitQStride];
+    const uint32_t tid = threadIdx.x, row0 = blockIdx.x * kRowsPerCta, per_row = C / 8;
+    const uint32_t chunks = (per_row + kRefitBlocks - 1) / kRefitBlocks;
+    // chunk c of the CTA's rows: per row up to 32 pieces of weights and 18 of fields, 16 bytes each
+    constexpr uint32_t kWPieces = kRefitBlocks * 2, kQPieces = kRefitBlocks * 18 / 16, kPieces = kWPieces + kQPieces;
+    auto issue = [&](uint32_t c) {
+        if (c < chunks) {
+            const uint32_t nb = min(kRefitBlocks, per_row - c * kRefitBlocks);     // blocks in this chunk: 16, or 8 at a row's end
+            for (uint32_t i = tid; i < kRowsPerCta * kPieces; i += kRowThreads) {
+                const uint32_t r = i / kPieces, j = i % kPieces;
+                if (row0 + r >= R) continue;
+                if (j < kWPieces) {
+                    if (j < 2 * nb) cp_async_16(&wbuf[c % kRowStages][r][4 * j], W + size_t(row0 + r) * C + size_t(c) * kRefitBlocks * 8 + 4 * j);
+                } else {
+                    const uint32_t k = j - kWPieces;
+                    if (16 * k < 18 * nb)
+                        cp_async_16(&qbuf[c % kRowStages][r][8 * k], fields + (size_t(row0 + r) * per_row + size_t(c) * kRefitBlocks) * 9 + 8 * k);
+                }
+            }
+        }
+        cp_async_commit_group();
+    };
+    for (uint32_t c = 0; c + 1 < kRowStages; ++c) issue(c);
+    double xp = 0.0, pp = 0.0;
+    for (uint32_t c = 0; c < chunks; ++c) {
+        issue(c + kRowStages - 1);
+        cp_async_wait_group<kRowStages - 1>();
+        __syncthreads();
+        if (tid < kRowsPerCta && row0 + tid < R) {
+            const uint32_t nb = min(kRefitBlocks, per_row - c * kRefitBlocks);
+            const float *xw = &wbuf[c % kRowStages][tid][0];
+            const int16_t *q = &qbuf[c % kRowStages][tid][0];
+            for (uint32_t v = 0; v < nb; ++v) refit_block(xw + 8 * v, q + 9 * v, xp, pp);
+        }
+        __syncthreads();                     // the stage may be overwritten by the next issue
+    }
+    if (tid < kRowsPerCta && row0 + tid < R) sigma[row0 + tid] = refit_result(xp, pp, s, mu[row0 + tid]);
+}
+
+// the same for any C: one thread per row reading its own row
+__global__ void refit_rows_kernel(const float *__restrict__ W, uint32_t R, uint32_t C, const int16_t *__restrict__ fields, float s,
+                                  const float *__restrict__ mu, float *__restrict__ sigma) {
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    const uint32_t per_row = C / 8;
+    const float *x = W + size_t(r) * C;
+    const int16_t *q = fields + size_t(r) * per_row * 9;
+    double xp = 0.0, pp = 0.0;
+    for (uint32_t v = 0; v < per_row; ++v) {
+        float xv[8];
+        int16_t qv[9];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) xv[j] = __ldg(x + 8 * v + j);
+#pragma unroll
+        for (int j = 0; j < 9; ++j) qv[j] = q[9 * v + j];
+        refit_block(xv, qv, xp, pp);
+    }
+    sigma[r] = refit_result(xp, pp, s, mu[r]);
 }
 
 struct EncodeTables {
@@ -388,7 +455,7 @@ public:
     int prepare(const std::vector<uint32_t> &sample) override {
         n_sample_ = uint32_t(sample.size());
         EP_CUDA(cudaMemcpyAsync(w_.rows, sample.data(), 4ull * n_sample_, cudaMemcpyHostToDevice, st_));
-        row_rms_kernel<<<(R_ + 63) / 64, 64, 0, st_>>>(W_, R_, C_, w_.mu);
+        row_rms_kernel<<<(R_ + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, st_>>>(W_, R_, C_, w_.mu);
         EP_CUDA(cudaGetLastError());
         return EP_OK;
     }
@@ -399,7 +466,10 @@ public:
         const uint64_t nvec = uint64_t(R_) * (C_ / 8);
         const uint32_t n_tiles = uint32_t((nvec + V - 1) / V);
         const uint32_t cap = 9u * V;
-        refit_kernel<<<(R_ + 63) / 64, 64, 0, st_>>>(W_, R_, C_, w_.fields, s, w_.mu, w_.sigma);
+        if (C_ % 64 == 0 && (reinterpret_cast<uintptr_t>(w_.fields) & 15) == 0)
+            refit_kernel<<<(R_ + kRowsPerCta - 1) / kRowsPerCta, kRowThreads, 0, st_>>>(W_, R_, C_, w_.fields, s, w_.mu, w_.sigma);
+        else
+            refit_rows_kernel<<<(R_ + 63) / 64, 64, 0, st_>>>(W_, R_, C_, w_.fields, s, w_.mu, w_.sigma);
         EP_CUDA(cudaGetLastError());
         EncodeTables T{};
         std::vector<uint32_t> fF;
