@@ -455,8 +455,9 @@ def peak_info():
 
 def extra_records(ep, torch, dev, stream, flush, slots, n_sms, peak, skip):
     """The stated configurations other than the headline one, each timed as the paper times its codec (CUDA events
-    around the call, three warm-ups, fifteen runs; here with an L2 flush before every run and the median reported).
-    Streams come from the library's GPU encoder (byte-identical to the host encoder's).  Returns a dict of records."""
+    around the call, three warm-ups, then repeated runs; here 24 runs with an L2 flush before each, the mean of the
+    central half reported).  Streams come from the library's GPU encoder (byte-identical to the host encoder's).
+    Returns a dict of records."""
     from paper_2609_34185_b200 import synth
 
     def timed(fn, reps=24, warm=3):
