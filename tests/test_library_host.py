@@ -99,6 +99,18 @@ def test_bad_arguments():
     assert lib.ep_encode(None, 4, 16, 4.0, None, ctypes.byref(h)) == -1
     assert lib.ep_encode(W.ctypes.data, 4, 8, -1.0, None, ctypes.byref(h)) == -1
     assert ep.strerror(-2).startswith("malformed")
+    # the fused decode + matrix product refuses on the host, before any CUDA call, what it cannot serve
+    blob = ep.encode(synth.gaussian_rows(32, 512, 7), 4.0, tile_vectors=64)
+    I = blob.info
+    fake = 4096                                                    # (never dereferenced: the checks come first)
+    assert lib.ep_decode_gemm(None, fake, fake, fake, fake, fake, 4, fake, None) == -1
+    assert lib.ep_decode_gemm(ctypes.byref(I), fake, fake, fake, fake, fake, 0, fake, None) == -1        # no tokens
+    assert lib.ep_decode_gemm(ctypes.byref(I), fake, fake, fake, fake, fake + 2, 4, fake, None) == -1    # misaligned x
+    assert lib.ep_decode_gemm(ctypes.byref(I), fake, fake, fake, fake + 16, fake, 4, fake, None) == -7   # misaligned tables
+    assert lib.ep_decode_gemm(ctypes.byref(I), fake, fake, fake, fake, fake, 33, fake, None) == -3       # more than 32 tokens
+    blob = ep.encode(synth.gaussian_rows(32, 512, 7), 4.0, tile_vectors=50)
+    I = blob.info
+    assert lib.ep_decode_gemm(ctypes.byref(I), fake, fake, fake, fake, fake, 4, fake, None) == -3        # not one tile per row
 
 
 def test_validate_rejects_damaged_structure():
