@@ -68,6 +68,23 @@ def test_decode_matmul_small_and_ragged_shapes():
         _check(blob, T, R + C + T)
 
 
+def test_decode_matmul_random_shapes():
+    # 24 seeded random cases: rows 1 .. 700, 1 .. 12 groups per row, 1 .. 32 tokens, encoder-made streams (row scales,
+    # tables and payload as the encoder leaves them) at 3 .. 6 bpp
+    rng = np.random.default_rng(75)
+    for case in range(24):
+        R = int(rng.integers(1, 700))
+        C = 256 * int(rng.integers(1, 13))
+        T = int(rng.integers(1, 33))
+        bpp = float(rng.choice([3.0, 4.0, 5.0, 6.0]))
+        W = (synth.laplace_rows if case % 2 else synth.gaussian_rows)(R, C, 7600 + case)
+        blob = ep.encode(W, bpp, tile_vectors=C // 8, b_start=11, b_max=11)
+        assert blob.info.b == 11 and blob.info.n_tiles == R
+        if ep.decode_scratch_bytes(blob.info):        # (a coordinate range beyond the shared-memory tables: not this path)
+            continue
+        _check(blob, T, 7700 + case)
+
+
 def test_decode_matmul_more_tokens_than_one_launch_and_repeated_calls():
     W = synth.gaussian_rows(128, 1536, 71)
     blob = ep.encode(W, 4.0, tile_vectors=1536 // 8)
