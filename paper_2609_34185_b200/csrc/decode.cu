@@ -435,6 +435,54 @@ __device__ __forceinline__ void decode_group_plain(uint32_t &x, uint32_t &wa, ui
     }
 }
 
+// ---- the same group with the hot loop's word addressing, for full groups of 2^11-slot streams -------------
+// Every lane keeps its own word address: the words taken in the previous step by this lane and the lanes above it
+// plus those taken in this step by the lanes below are one population count of a bit-select of the two ballots.
+// Used where the loop around the group is C++ (the kernel that feeds the tensor cores); BF16 block returned in `blk`.
+__device__ __forceinline__ void lean_renorm(uint32_t &x, uint32_t &a, uint32_t &bal, uint32_t lt) {
+    const bool need = x < ep::kStateLow;
+    const uint32_t now = __ballot_sync(0xFFFFFFFFu, need);
+    a += 2u * __popc((lt & now) | (~lt & bal));
+    bal = now;
+    if (need) {
+        uint16_t w;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(w) : "r"(a));
+        x = (x << 16) | w;
+    }
+}
+__device__ __forceinline__ uint4 decode_group_lean_bf16(uint32_t &x, uint32_t &wa, uint32_t lut_addr, CosetFreq cf, uint32_t lt,
+                                                        uint32_t k0_bits, float sigma) {
+    uint32_t a = wa, bal = 0, e[9];
+    {   // the coset: slot below f0 -> 0, else 1
+        const uint32_t u = x & 2047u, q = x >> 11;
+        const bool c1 = u >= cf.f0;
+        x = (c1 ? cf.f1 : max(cf.f0, 1u)) * q + (c1 ? u - cf.f0 : u);
+        e[0] = c1 ? 1u : 0u;
+        lean_renorm(x, a, bal, lt);
+    }
+    const uint32_t tab = lut_addr + e[0] * kCosetStride;
+#pragma unroll
+    for (int k = 1; k <= 8; ++k) {
+        const uint32_t q = x >> 11;
+        e[k] = lds32(tab + uint32_t(k - 1) * kLutStride + ((x & 2047u) << 2));
+        x = (e[k] >> 21) * q + (e[k] & 0x7FFu);
+        lean_renorm(x, a, bal, lt);
+    }
+    wa = __shfl_sync(0xFFFFFFFFu, a, 0) + 2u * __popc(bal);      // lane 0's address is the cursor before the last step
+    const uint32_t par = (e[1] ^ e[2] ^ e[3] ^ e[4] ^ e[5] ^ e[6] ^ e[7]) & 0x800u;
+    const uint32_t cc = kExp4096 | (e[0] << 10);
+    const uint64_t kk = pack64(k0_bits, k0_bits);
+    const uint64_t ss = pack64(__float_as_uint(sigma), __float_as_uint(sigma));
+    uint32_t xb[8];
+#pragma unroll
+    for (int k = 1; k <= 7; ++k) xb[k - 1] = (e[k] & kCodeMask) | cc;
+    xb[7] = (e[8] & kCodeMask) | par | cc;
+    float w[8];
+#pragma unroll
+    for (int i = 0; i < 8; i += 2) unpack64(mul2(sub2(pack64(xb[i], xb[i + 1]), kk), ss), w[i], w[i + 1]);
+    return make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]), pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
+}
+
 // ---- payload ring ------------------------------------------------------------------------------------
 // chunk c of a tile = global bytes [a0 + CHUNK c, a0 + CHUNK (c + 1)), a0 = tile's first word rounded down to
 // 16 bytes; it lives in ring slot c mod SLOTS, and a chunk in one of the slots that make up the ring's first 512
@@ -1316,7 +1364,7 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
         }
     } else {
         // ---- the decoding warps: one row of W each, group by group into the slabs of B ----
-        const uint32_t lt = (1u << lane) - 1u, mask = 2047u, b = 11u;
+        const uint32_t lt = (1u << lane) - 1u;
         const uint32_t k0_bits = __float_as_uint(float(4096 - J.zlo));
         // where this lane's block of a group goes in a slab: 64-column tile lane / 8, row = warp, piece lane % 8 of the row
         const uint32_t b_dst = b_base + (lane >> 3) * 4096u + warp * 128u + (((lane & 7u) ^ (warp & 7u)) << 4);
@@ -1349,7 +1397,7 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
                     if (pos >= threshold) ring_service<kGemmChunk, kGemmSlots>(ring, Tl.a0, Tl.room, pos, threshold, lane);
                     const uint32_t wa0 = ring + pos % (kGemmChunk * kGemmSlots);
                     uint32_t wa = wa0;
-                    decode_group_plain<EP_BF16>(x, wa, lut_addr, cf, mask, b, lt, true, k0_bits, sigma, J.zlo, &blk);
+                    blk = decode_group_lean_bf16(x, wa, lut_addr, cf, lt, k0_bits, sigma);
                     pos += wa - wa0;
                 }
                 // the slab is free: the tensor core is done with the group that used it last, two groups ago
