@@ -1215,13 +1215,20 @@ constexpr uint32_t kGemmB = kGemmA + 16384;              // B operand: two slabs
 constexpr uint32_t kGemmBar = kGemmB + 32768;            // mbarriers, tensor-memory address, abort word, counter
 constexpr uint32_t kGemmSmem = kGemmBar + 64;
 constexpr uint32_t kSpinLimit = 1u << 18;             // attempts of about a microsecond each at most: a quarter of a second
-constexpr uint32_t kGemmRows = 31;                       // rows of W per step: warps 0 .. 30 decode one each, warp 31 feeds the tensor core
+constexpr uint32_t kGemmRows = 30;                       // rows of W per step: warps 0 .. 29 decode one each, warp 30 brings x in, warp 31 issues the matrix instructions
 constexpr uint32_t kGemmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((64u >> 4) << 24);   // f32 += bf16 x bf16, K-major both, N = 32, M = 64
 static_assert(kGemmA % 1024 == 0, "swizzled operand tiles start on 1024-byte boundaries");
 static_assert(kGemmSmem <= 232448, "more shared memory than an sm_100 CTA can have");
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+// a test that never waits
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
 }
 // one attempt: the thread may be suspended by the hardware for up to about a microsecond while the phase is pending
 // (a busy test_wait loop of 32 waiting lanes took half of the kernel's issue slots away from the decoding warps)
@@ -1285,10 +1292,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(32u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // row 31 of both slabs of B belongs to no warp: zero, so that column 31 of the accumulator stays finite
-    if (warp == kGemmRows) {
+    if (warp >= kGemmRows) {                 // rows 30 and 31 of both slabs belong to no warp: zero (this warp's row, all its pieces)
         for (uint32_t i = lane; i < 2u * 4u * 8u; i += 32u)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(b_base + (i >> 5) * 16384u + ((i >> 3) & 3u) * 4096u + kGemmRows * 128u + (i & 7u) * 16u), "r"(0u) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(b_base + (i >> 5) * 16384u + ((i >> 3) & 3u) * 4096u + warp * 128u + (i & 7u) * 16u), "r"(0u) : "memory");
         fence_async_smem();
     }
     copy_tables_smem(J.lut_image, lut_addr, false);
@@ -1302,8 +1308,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
     const uint32_t row_begin = min(blockIdx.x * P.rows_per_cta, P.R), row_end = min(row_begin + P.rows_per_cta, P.R);
     const uint32_t steps = (row_end - row_begin + kGemmRows - 1u) / kGemmRows;
     const uint32_t q_total = steps * P.groups;               // groups this CTA hands to the tensor core
-    // one lane polls, the warp follows
+    // usually the phase is long complete: one test by the whole warp; otherwise one lane polls and the warp follows
     auto wait_warp = [&](uint32_t bar, uint32_t parity) {
+        if (mbar_test(bar, parity)) return;
         if (lane == 0) mbar_wait(bar, parity, abort_addr);
         __syncwarp();
     };
@@ -1311,7 +1318,7 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
     bool bad = false;
 
     if (warp == kGemmRows) {
-        // ---- the feeding warp: x into A, matrix instructions, no decoding; one lane does it all ----
+        // ---- the loading warp: one lane brings x into A, nothing else ----
         // group q's 256 columns of x: four tiles of 64 columns x TPAD rows, laid out and swizzled by the copy engine
         // (rows past the last token lie outside the tensor and arrive as zeros)
         auto load_a = [&](uint32_t qq) {
@@ -1328,6 +1335,20 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
             if (stages == 2u && q_total > 1u) load_a(1u);
         }
         for (uint32_t q = 0; q < q_total; ++q) {
+            if (lane == 0 && q + stages < q_total) {   // the stage group q used is free when its instructions are done
+                mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
+                load_a(q + stages);
+            }
+            __syncwarp();
+            if ((q + 1u) % P.groups == 0u) {           // a step's last group: the decoding warps read the accumulator out now
+                tc_fence_before();
+                __syncthreads();
+                tc_fence_after();
+            }
+        }
+    } else if (warp == kGemmRows + 1u) {
+        // ---- the issuing warp: one lane waits for a group's operands and issues its sixteen matrix instructions ----
+        for (uint32_t q = 0; q < q_total; ++q) {
             const uint32_t st = q % stages, g = q % P.groups;
             if (lane == 0) {
                 mbar_wait(bar_a + 8u * st, (q / stages) & 1u, abort_addr);
@@ -1343,20 +1364,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
                         umma_bf16(tmem, pack64(da_lo + ((c * a_tile_bytes + 32u * k) >> 4), da_hi),
                                   pack64(db_lo + ((c * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc, (g | c | k) ? 1u : 0u);
                 umma_commit(bar_mma + 8u * (q & 1u));
-                if constexpr (stages == 2u) {
-                    // refill the stage the PREVIOUS group used: its instructions were committed a whole group ago and are
-                    // done or nearly so, and the tiles have this group's time to arrive
-                    if (q >= 1u && q + 1u < q_total) {
-                        mbar_wait(bar_mma + 8u * ((q - 1u) & 1u), ((q - 1u) >> 1) & 1u, abort_addr);
-                        load_a(q + 1u);
-                    }
-                } else if (q + 1u < q_total) {   // one stage: it is free when this group's instructions are done
-                    mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
-                    load_a(q + 1u);
-                }
             }
             __syncwarp();
-            if (g + 1u == P.groups) {        // a step's last group: the other warps read the accumulator out now
+            if (g + 1u == P.groups) {
                 tc_fence_before();
                 __syncthreads();
                 tc_fence_after();
