@@ -1181,16 +1181,18 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
 // straight into the shared-memory operand of a tcgen05 matrix instruction and never written to global memory.
 //
 // The stream must have one tile per row of W (V = C / 8) and C a multiple of 256.  The rows are spread evenly over
-// the SMs; a CTA takes its range 31 rows at a time, one row per warp: warps 0 .. 30 decode their rows group by group
-// (a group = 32 blocks = 256 columns), so after every group the CTA holds a 31 x 256 slab of W - the B operand
-// (N = 32 with one idle row, K-major, 128-byte swizzle: a lane's 16-byte block is one piece of a swizzled row, so
-// the stores are conflict-free).  Warp 31 decodes nothing: one of its lanes brings the matching 256 columns of x in
-// (A operand, M = 64 rows of which the first 16 or 32 are tokens; the others read whatever shared memory follows
-// and produce accumulator rows nobody stores) with four tensor copies (cp.async.bulk.tensor, the copy engine
-// swizzles), waits until all rows of the slab are stored and issues the slab's sixteen K = 16 instructions.  (A
-// decoding warp cannot do that on the side: whoever issues falls behind by the time it takes, and with two slabs
-// every warp is at most one group ahead of the slowest - measured 138 us against 102 us for the layer below.)  The
-// fp32 accumulator (64 lanes x 32 columns) stays in tensor memory over the whole row and is read out once per step.
+// the SMs; a CTA takes its range 30 rows at a time, one row per warp: warps 0 .. 29 decode their rows group by group
+// (a group = 32 blocks = 256 columns), so after every group the CTA holds a 30 x 256 slab of W - the B operand
+// (N = 32 with two idle rows, K-major, 128-byte swizzle: a lane's 16-byte block is one piece of a swizzled row, so
+// the stores are conflict-free).  Warps 30 and 31 decode nothing.  One lane of warp 30 brings the matching 256
+// columns of x in (A operand, M = 64 rows of which the first 16 or 32 are tokens; the others read whatever shared
+// memory follows and produce accumulator rows nobody stores) with four tensor copies (cp.async.bulk.tensor, the
+// copy engine swizzles).  One lane of warp 31 waits until x has landed and all rows of the slab are stored and
+// issues the slab's sixteen K = 16 instructions.  (A decoding warp cannot do that on the side: whoever issues falls
+// behind by the time it takes, and with two slabs every warp is at most one group ahead of the slowest - measured
+// 138 us for the layer below; one warp for copies and instructions together 90 us, its single instruction stream
+// being the slowest in the CTA; two warps on two schedulers 84 us.)  The fp32 accumulator (64 lanes x 32 columns)
+// stays in tensor memory over the whole row and is read out once per step.
 //
 // Shared memory: the lookup tables (128 KB), 32 payload rings of 4 x 256 + 512 bytes (48 KB), then A (16 KB: two
 // stages for up to 16 tokens, one for up to 32), B (two slabs of 16 KB: the warps decode the next group while the
