@@ -439,16 +439,33 @@ __device__ __forceinline__ void decode_group_plain(uint32_t &x, uint32_t &wa, ui
 // Every lane keeps its own word address: the words taken in the previous step by this lane and the lanes above it
 // plus those taken in this step by the lanes below are one population count of a bit-select of the two ballots.
 // Used where the loop around the group is C++ (the kernel that feeds the tensor cores); BF16 block returned in `blk`.
+// renormalisation: lanes whose state fell below 2^15 take a word each, in lane order (the hot loop's seven instructions)
 __device__ __forceinline__ void lean_renorm(uint32_t &x, uint32_t &a, uint32_t &bal, uint32_t lt) {
-    const bool need = x < ep::kStateLow;
-    const uint32_t now = __ballot_sync(0xFFFFFFFFu, need);
-    a += 2u * __popc((lt & now) | (~lt & bal));
-    bal = now;
-    if (need) {
-        uint16_t w;
-        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(w) : "r"(a));
-        x = (x << 16) | w;
-    }
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 now, t, w;\n\t"
+                 "setp.lt.u32 p, %0, 32768;\n\t"
+                 "vote.sync.ballot.b32 now, p, 0xffffffff;\n\t"
+                 "lop3.b32 t, %3, now, %2, 0xCA;\n\t"          // the lanes below: this step's ballot; this lane and above: the last one's
+                 "popc.b32 t, t;\n\t"
+                 "mad.lo.u32 %1, t, 2, %1;\n\t"
+                 "ld.shared.u16 w, [%1];\n\t"
+                 "@p mad.lo.u32 %0, %0, 65536, w;\n\t"
+                 "mov.b32 %2, now;\n\t}"
+                 : "+r"(x), "+r"(a), "+r"(bal) : "r"(lt) : "memory");
+}
+// one coordinate symbol (Eq. 18) from the table at shared-memory address `table`: returns the entry
+__device__ __forceinline__ uint32_t lean_step(uint32_t &x, uint32_t &a, uint32_t &bal, uint32_t table, uint32_t lt) {
+    uint32_t e;
+    asm volatile("{\n\t.reg .b32 q, u, f, bi;\n\t"
+                 "shr.u32 q, %0, 11;\n\t"
+                 "mad.lo.u32 u, q, 0xFFFFE000, %2;\n\t"        // slot address 4 (x & 2047) + table = 4 x - 8192 (x >> 11) + table
+                 "mad.lo.u32 u, %0, 4, u;\n\t"
+                 "ld.shared.u32 %1, [u];\n\t"
+                 "shr.u32 f, %1, 21;\n\t"
+                 "and.b32 bi, %1, 0x7FF;\n\t"
+                 "mad.lo.u32 %0, f, q, bi;\n\t}"
+                 : "+r"(x), "=r"(e) : "r"(table) : "memory");
+    lean_renorm(x, a, bal, lt);
+    return e;
 }
 __device__ __forceinline__ uint4 decode_group_lean_bf16(uint32_t &x, uint32_t &wa, uint32_t lut_addr, CosetFreq cf, uint32_t lt,
                                                         uint32_t k0_bits, float sigma) {
@@ -462,12 +479,7 @@ __device__ __forceinline__ uint4 decode_group_lean_bf16(uint32_t &x, uint32_t &w
     }
     const uint32_t tab = lut_addr + e[0] * kCosetStride;
 #pragma unroll
-    for (int k = 1; k <= 8; ++k) {
-        const uint32_t q = x >> 11;
-        e[k] = lds32(tab + uint32_t(k - 1) * kLutStride + ((x & 2047u) << 2));
-        x = (e[k] >> 21) * q + (e[k] & 0x7FFu);
-        lean_renorm(x, a, bal, lt);
-    }
+    for (int k = 1; k <= 8; ++k) e[k] = lean_step(x, a, bal, tab + uint32_t(k - 1) * kLutStride, lt);
     wa = __shfl_sync(0xFFFFFFFFu, a, 0) + 2u * __popc(bal);      // lane 0's address is the cursor before the last step
     const uint32_t par = (e[1] ^ e[2] ^ e[3] ^ e[4] ^ e[5] ^ e[6] ^ e[7]) & 0x800u;
     const uint32_t cc = kExp4096 | (e[0] << 10);
