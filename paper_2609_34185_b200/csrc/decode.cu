@@ -1350,8 +1350,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
         }
         for (uint32_t q = 0; q < q_total; ++q) {
             if (lane == 0 && q + stages < q_total) {   // the stage group q used is free when its instructions are done
-                mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
-                load_a(q + stages);
+                // (after a wait that ran out nothing is copied any more: re-arming a barrier whose phase never completed
+                // would overflow its transaction count)
+                if (mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr)) load_a(q + stages);
             }
             __syncwarp();
             if ((q + 1u) % P.groups == 0u) {           // a step's last group: the decoding warps read the accumulator out now
@@ -1365,8 +1366,8 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
         for (uint32_t q = 0; q < q_total; ++q) {
             const uint32_t st = q % stages, g = q % P.groups;
             if (lane == 0) {
-                mbar_wait(bar_a + 8u * st, (q / stages) & 1u, abort_addr);
-                mbar_wait(bar_b + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
+                const bool ready = mbar_wait(bar_a + 8u * st, (q / stages) & 1u, abort_addr) &&
+                                   mbar_wait(bar_b + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
                 tc_fence_after();
                 // descriptors differ in their address field only: low word + (bytes >> 4)
                 const uint64_t da = umma_desc(a_base + st * a_stage_bytes), db = umma_desc(b_base + 16384u * (q & 1u));
@@ -1375,8 +1376,9 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
                 for (uint32_t c = 0; c < 4; ++c)
 #pragma unroll
                     for (uint32_t k = 0; k < 4; ++k)                 // 16 columns = 32 bytes further along the swizzled rows
-                        umma_bf16(tmem, pack64(da_lo + ((c * a_tile_bytes + 32u * k) >> 4), da_hi),
-                                  pack64(db_lo + ((c * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc, (g | c | k) ? 1u : 0u);
+                        if (ready)                                   // (operands that never arrived are not multiplied)
+                            umma_bf16(tmem, pack64(da_lo + ((c * a_tile_bytes + 32u * k) >> 4), da_hi),
+                                      pack64(db_lo + ((c * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc, (g | c | k) ? 1u : 0u);
                 umma_commit(bar_mma + 8u * (q & 1u));
             }
             __syncwarp();
