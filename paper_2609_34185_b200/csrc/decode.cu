@@ -1206,9 +1206,10 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_smem_kernel(const __gri
 // being the slowest in the CTA; two warps on two schedulers 84 us.)  The fp32 accumulator (64 lanes x 32 columns)
 // stays in tensor memory over the whole row and is read out once per step.
 //
-// Shared memory: the lookup tables (128 KB), 32 payload rings of 4 x 256 + 512 bytes (48 KB), then A (16 KB: two
-// stages for up to 16 tokens, one for up to 32), B (two slabs of 16 KB: the warps decode the next group while the
-// tensor core reads the last one) and six mbarriers.  What bounds the token count: a group's columns of x must be in
+// Shared memory: the lookup tables (128 KB), 32 payload rings of 4 x 256 + 512 bytes (48 KB), then A (16 KB: two units
+// of x - a group's 256 columns of up to 16 tokens each, or half a group's of up to 32 -, refilled by the loading warp as
+// soon as the instructions that read a unit are done), B (two slabs of 16 KB: the warps decode the next group while the
+// tensor core reads the last one) and the mbarriers.  What bounds the token count: a group's columns of x must be in
 // flight while the group is decoded (about 1 us), every CTA re-reads x from L2, and 16 KB is the landing space left.
 // Every wait on an mbarrier gives up after kSpinLimit polls, raises the abort word and lets the kernel run to its
 // end (wrong output, status flag set) instead of hanging.
@@ -1227,7 +1228,7 @@ constexpr uint32_t kGemmRingStride = kGemmChunk * kGemmSlots + kRingMirror;   //
 constexpr uint32_t kGemmA = kRingBase + 32u * kGemmRingStride;   // A operand: per stage four 64-column tiles of Tpad rows
 constexpr uint32_t kGemmB = kGemmA + 16384;              // B operand: two slabs of four 64-column tiles of 32 rows
 constexpr uint32_t kGemmBar = kGemmB + 32768;            // mbarriers, tensor-memory address, abort word, counter
-constexpr uint32_t kGemmSmem = kGemmBar + 64;
+constexpr uint32_t kGemmSmem = kGemmBar + 256;
 constexpr uint32_t kSpinLimit = 1u << 18;             // attempts of about a microsecond each at most: a quarter of a second
 constexpr uint32_t kGemmRows = 30;                       // rows of W per step: warps 0 .. 29 decode one each, warp 30 brings x in, warp 31 issues the matrix instructions
 constexpr uint32_t kGemmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((64u >> 4) << 24);   // f32 += bf16 x bf16, K-major both, N = 32, M = 64
@@ -1254,6 +1255,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 // waits for the phase of the given parity to complete; false (and the abort word set) if it does not within the limit
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_addr) {
+    if (mbar_test(bar, parity)) return true;             // usually the phase is long complete
     if (lds32(abort_addr)) return false;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try(bar, parity)) return true;
@@ -1288,13 +1290,17 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
     const uint32_t lut_addr = uint32_t(__cvta_generic_to_shared(smem));
     const uint32_t ring = lut_addr + kRingBase + warp * kGemmRingStride;
     const uint32_t a_base = lut_addr + kGemmA, b_base = lut_addr + kGemmB;
-    // two mbarriers each for: x landed (per stage of A), rows stored (per slab of B), the tensor core's commits (per slab)
-    const uint32_t bar_a = lut_addr + kGemmBar, bar_mma = bar_a + 16u, bar_b = bar_a + 32u, slot = bar_a + 48u,
-                   abort_addr = bar_a + 52u;
-    constexpr uint32_t stages = TPAD == 16u ? 2u : 1u;      // 16 staged rows of x: two groups' worth fit the 16 KB
+    // A holds two units of x, a unit being half of what fits: four tiles of 64 columns x 16 rows (one group's columns), or
+    // two tiles x 32 rows (half a group's).  Per unit one mbarrier "landed" and one "read"; per slab of B one "rows stored"
+    // and one "read".
+    constexpr uint32_t a_tile_bytes = TPAD * 128u, kUnitTiles = 8192u / a_tile_bytes, kUnitsPerGroup = 4u / kUnitTiles;
+    const uint32_t bar_a = lut_addr + kGemmBar, bar_afree = bar_a + 64u, bar_mma = bar_a + 128u, bar_b = bar_a + 144u,
+                   slot = bar_a + 160u, abort_addr = bar_a + 164u;
     if (tid == 0) {
-        mbar_init(bar_a, 1u);                // the feeding lane's arrival; completes when the tiles of x have landed
-        mbar_init(bar_a + 8u, 1u);
+        for (uint32_t i = 0; i < 2u; ++i) {
+            mbar_init(bar_a + 8u * i, 1u);       // the loading lane's arrival; completes when the unit's tiles have landed
+            mbar_init(bar_afree + 8u * i, 1u);   // the commit after the matrix instructions that read the unit
+        }
         mbar_init(bar_mma, 1u);              // the commit after a group's matrix instructions
         mbar_init(bar_mma + 8u, 1u);
         mbar_init(bar_b, kGemmRows);         // every decoding warp, when its row of the slab is stored
@@ -1328,65 +1334,65 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
         if (lane == 0) mbar_wait(bar, parity, abort_addr);
         __syncwarp();
     };
-    constexpr uint32_t a_tile_bytes = TPAD * 128u, a_stage_bytes = 4u * a_tile_bytes;
     bool bad = false;
+    // the end of a step (accumulator read out, next rows may overwrite it) concerns the decoding warps and the issuing
+    // warp; the loading warp runs ahead of them across steps
+    auto step_sync = [&]() {
+        tc_fence_before();
+        asm volatile("bar.sync 1, %0;" ::"n"(kThreads - 32) : "memory");
+        tc_fence_after();
+    };
 
     if (warp == kGemmRows) {
-        // ---- the loading warp: one lane brings x into A, nothing else ----
-        // group q's 256 columns of x: four tiles of 64 columns x TPAD rows, laid out and swizzled by the copy engine
-        // (rows past the last token lie outside the tensor and arrive as zeros)
-        auto load_a = [&](uint32_t qq) {
-            const uint32_t g = qq % P.groups, st = qq % stages, bar = bar_a + 8u * st;
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(a_stage_bytes) : "memory");
-#pragma unroll
-            for (uint32_t t = 0; t < 4; ++t)
-                asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                             ::"r"(a_base + st * a_stage_bytes + t * a_tile_bytes), "l"(&x_map), "r"(g * 256u + t * 64u), "r"(0u), "r"(bar)
-                             : "memory");
-        };
+        // ---- the loading warp: one lane brings x into A, unit after unit, nothing else ----
+        // tile i of the CTA's sequence = columns [64 i, 64 i + 64) of x, counted over all groups (and again from column 0 for
+        // every step); the copy engine lays it out and swizzles it; rows past the last token lie outside the tensor and
+        // arrive as zeros
         if (lane == 0) {
-            load_a(0u);
-            if (stages == 2u && q_total > 1u) load_a(1u);
-        }
-        for (uint32_t q = 0; q < q_total; ++q) {
-            if (lane == 0 && q + stages < q_total) {   // the stage group q used is free when its instructions are done
+            const uint32_t tiles_per_step = 4u * P.groups;
+            for (uint32_t j = 0; j < kUnitsPerGroup * q_total; ++j) {
+                const uint32_t buf = j & 1u;
                 // (after a wait that ran out nothing is copied any more: re-arming a barrier whose phase never completed
                 // would overflow its transaction count)
-                if (mbar_wait(bar_mma + 8u * (q & 1u), (q >> 1) & 1u, abort_addr)) load_a(q + stages);
-            }
-            __syncwarp();
-            if ((q + 1u) % P.groups == 0u) {           // a step's last group: the decoding warps read the accumulator out now
-                tc_fence_before();
-                __syncthreads();
-                tc_fence_after();
+                if (j >= 2u && !mbar_wait(bar_afree + 8u * buf, ((j >> 1) - 1u) & 1u, abort_addr)) break;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a + 8u * buf), "r"(8192u) : "memory");
+#pragma unroll
+                for (uint32_t t = 0; t < kUnitTiles; ++t)
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                                 ::"r"(a_base + buf * 8192u + t * a_tile_bytes), "l"(&x_map),
+                                   "r"(((j * kUnitTiles + t) % tiles_per_step) * 64u), "r"(0u), "r"(bar_a + 8u * buf)
+                                 : "memory");
             }
         }
+        __syncwarp();
     } else if (warp == kGemmRows + 1u) {
-        // ---- the issuing warp: one lane waits for a group's operands and issues its sixteen matrix instructions ----
+        // ---- the issuing warp: one lane waits for a group's rows and, unit by unit, for x, and issues the matrix instructions ----
         for (uint32_t q = 0; q < q_total; ++q) {
-            const uint32_t st = q % stages, g = q % P.groups;
+            const uint32_t g = q % P.groups;
             if (lane == 0) {
-                const bool ready = mbar_wait(bar_a + 8u * st, (q / stages) & 1u, abort_addr) &&
-                                   mbar_wait(bar_b + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
-                tc_fence_after();
+                bool ready = mbar_wait(bar_b + 8u * (q & 1u), (q >> 1) & 1u, abort_addr);
                 // descriptors differ in their address field only: low word + (bytes >> 4)
-                const uint64_t da = umma_desc(a_base + st * a_stage_bytes), db = umma_desc(b_base + 16384u * (q & 1u));
+                const uint64_t da = umma_desc(a_base), db = umma_desc(b_base + 16384u * (q & 1u));
                 const uint32_t da_hi = uint32_t(da >> 32), db_hi = uint32_t(db >> 32), da_lo = uint32_t(da), db_lo = uint32_t(db);
 #pragma unroll
-                for (uint32_t c = 0; c < 4; ++c)
+                for (uint32_t h = 0; h < kUnitsPerGroup; ++h) {
+                    const uint32_t j = kUnitsPerGroup * q + h, buf = j & 1u;
+                    ready = ready && mbar_wait(bar_a + 8u * buf, (j >> 1) & 1u, abort_addr);
+                    tc_fence_after();
 #pragma unroll
-                    for (uint32_t k = 0; k < 4; ++k)                 // 16 columns = 32 bytes further along the swizzled rows
-                        if (ready)                                   // (operands that never arrived are not multiplied)
-                            umma_bf16(tmem, pack64(da_lo + ((c * a_tile_bytes + 32u * k) >> 4), da_hi),
-                                      pack64(db_lo + ((c * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc, (g | c | k) ? 1u : 0u);
+                    for (uint32_t t = 0; t < kUnitTiles; ++t)
+#pragma unroll
+                        for (uint32_t k = 0; k < 4; ++k)             // 16 columns = 32 bytes further along the swizzled rows
+                            if (ready)                               // (operands that never arrived are not multiplied)
+                                umma_bf16(tmem, pack64(da_lo + ((buf * 8192u + t * a_tile_bytes + 32u * k) >> 4), da_hi),
+                                          pack64(db_lo + (((h * kUnitTiles + t) * 4096u + 32u * k) >> 4), db_hi), kGemmIdesc,
+                                          (g | h | t | k) ? 1u : 0u);
+                    umma_commit(bar_afree + 8u * buf);
+                }
                 umma_commit(bar_mma + 8u * (q & 1u));
             }
             __syncwarp();
-            if (g + 1u == P.groups) {
-                tc_fence_before();
-                __syncthreads();
-                tc_fence_after();
-            }
+            if (g + 1u == P.groups) step_sync();
         }
     } else {
         // ---- the decoding warps: one row of W each, group by group into the slabs of B ----
@@ -1456,10 +1462,8 @@ __global__ void __launch_bounds__(kThreads, 1) ep_decode_gemm_kernel(const __gri
                         if (i < n) dst[i] = __uint_as_float(v[i]);
                 }
             }
-            tc_fence_before();
             cp_async_wait<0>();              // nothing may still be landing in the ring when the next row starts
-            __syncthreads();                 // the accumulator has been read before the next rows overwrite it
-            tc_fence_after();
+            step_sync();                     // the accumulator has been read before the next rows overwrite it
             bad |= active && ((x != ep::kStateLow) || (Tl.off + ((pos - Tl.lead) >> 1) != Tl.end));
         }
     }
